@@ -1,0 +1,246 @@
+/*
+ * superoffload.h -- C ABI of the B200 bucketized speculative AdamW library.
+ *
+ * The library implements the optimizer hot path of SuperOffload (arXiv
+ * 2509.21271) on one GPU: model states flattened into fixed-size buckets
+ * (Section 4.3), a mixed-precision AdamW step that runs per bucket *before*
+ * the global gradient check has finished (speculation-then-validation,
+ * Section 4.4), the check itself (global L2 gradient norm + NaN/Inf flag),
+ * commit or bit-exact rollback (Section 4.4, "in-place rollback" and its two
+ * scenarios), and the fp32 -> bf16 parameter cast (Section 4.5).
+ *
+ * General conventions
+ *   - Every function returns an so_status (0 = SO_OK, negative = error) and
+ *     never throws, aborts or prints.  Argument and state errors are detected
+ *     before anything is launched and leave the context untouched.
+ *   - All DEVICE memory is allocated and owned by the caller, in the sizes
+ *     so_layout_init reports; the library keeps host-side metadata only and
+ *     so_destroy frees only that.  Device pointers must be 256-byte aligned.
+ *   - `stream` arguments are cudaStream_t values passed as void* (NULL = the
+ *     legacy default stream).  Calls that launch work enqueue it and return;
+ *     only calls that fill a host struct from device results synchronise that
+ *     stream (stated per function).
+ *   - The device that is current when so_layout_bind is called must be current
+ *     for every later call on that context.  A context is not thread-safe;
+ *     separate contexts are independent.
+ *   - Hyper-parameters are doubles so that host and device see one constant.
+ *
+ * Memory layout (what the caller allocates)
+ *   The flat parameter space [0, N) is the concatenation of the tensors in the
+ *   order given.  Bucket b covers flat [b*B, min((b+1)*B, N)).  Arenas are
+ *   arrays of fixed-size *slots* of `slot_stride_elems` elements (B rounded up
+ *   to a multiple of 64, so every slot starts 256-byte aligned); flat element
+ *   i sits at position (i / B) * slot_stride_elems + (i % B) of the gradient
+ *   and bf16-parameter arenas (identity when B is a multiple of 64).
+ *   The fp32 state arenas (master, m, v) hold n_buckets + undo_slots slots:
+ *   bucket b's committed state lives in slot so_bucket_slot(b) (initially b).
+ *   A speculative step writes the new state of a bucket into a free slot and
+ *   leaves the old one untouched; commit re-points the bucket at the new slot,
+ *   rollback simply drops it.  Nothing is ever copied to undo a step.
+ */
+#ifndef SUPEROFFLOAD_H
+#define SUPEROFFLOAD_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct so_ctx so_ctx;          /* opaque, host-side, library-owned */
+typedef int32_t so_status;
+
+enum {
+    SO_OK = 0,
+    SO_ERR_INVALID_ARG = -1,           /* bad pointer, size, dtype, hyper-parameter  */
+    SO_ERR_STATE = -2,                 /* call not allowed in the current step phase */
+    SO_ERR_CUDA = -3,                  /* a CUDA call failed; see so_last_cuda_error */
+    SO_ERR_UNDO_EXHAUSTED = -4,        /* no free slot for another speculative step  */
+    SO_ERR_NOMEM = -5,                 /* host allocation failed                     */
+    SO_ERR_UNSUPPORTED = -6
+};
+
+enum { SO_GRAD_BF16 = 0, SO_GRAD_FP32 = 1 };
+enum { SO_DECISION_COMMIT = 0, SO_DECISION_SKIP = 1, SO_DECISION_CLIP_RESTEP = 2 };
+#define SO_ALL (-1)
+
+/* AdamW hyper-parameters.  max_grad_norm <= 0 disables clipping. */
+typedef struct {
+    double lr, beta1, beta2, eps, weight_decay, max_grad_norm;
+} so_hparams;
+
+typedef struct {
+    int64_t total_elems;               /* N                                          */
+    int64_t bucket_elems;              /* B                                          */
+    int64_t slot_stride_elems;         /* B rounded up to a multiple of 64           */
+    int64_t last_bucket_elems;         /* elements in the last bucket (0 if N == 0)  */
+    int32_t n_buckets;                 /* ceil(N / B)                                */
+    int32_t n_tensors;
+    int32_t n_state_slots;             /* n_buckets + undo_slots                     */
+    int32_t undo_slots;
+    int32_t grad_dtype;
+    int32_t tile_elems;                /* elements per reduction tile (1024)         */
+    int64_t tiles_per_slot;
+    uint64_t bytes_master, bytes_m, bytes_v;   /* n_state_slots * stride * 4 each    */
+    uint64_t bytes_grad;               /* n_buckets * stride * (2 or 4)              */
+    uint64_t bytes_param_bf16;         /* n_buckets * stride * 2                     */
+    uint64_t bytes_scratch;            /* tile partial sums + per-bucket results     */
+} so_layout_info;
+
+typedef struct {
+    double sumsq;                      /* sum over all gradients of g^2              */
+    double norm;                       /* sqrt(sumsq)                                */
+    double clip_coef;                  /* min(1, max_grad_norm / (norm + 1e-6))      */
+    int32_t nonfinite;                 /* 1 if any gradient is NaN or +-Inf          */
+    int32_t reserved;
+} so_grad_stats;
+
+typedef struct {
+    int32_t decision;                  /* SO_DECISION_*                              */
+    int32_t buckets_speculated;        /* buckets that had been stepped speculatively*/
+    int64_t step_after;                /* committed step count after this call       */
+    so_grad_stats stats;
+} so_step_result;
+
+typedef struct {
+    int64_t commits, skips, clip_resteps;      /* validated iterations by outcome    */
+    int64_t kernel_launches;                   /* kernels this context has launched  */
+    int64_t elems_stepped, elems_checked, elems_cast;  /* work done by those kernels */
+} so_counters;
+
+/*
+ * so_layout_init -- flatten a tensor list into fixed-size buckets
+ * (Section 4.3: model states are divided into buckets, the unit of transfer,
+ * of the optimizer step and of rollback).  Host-only integer arithmetic.
+ *   out          receives a new context (caller frees it with so_destroy)
+ *   n_tensors    number of tensors (>= 0); numel[i] >= 0 elements each (host)
+ *   bucket_elems B, 1 <= B <= 2^30
+ *   grad_dtype   SO_GRAD_BF16 or SO_GRAD_FP32 (dtype of the gradient arena)
+ *   undo_slots   how many buckets may be stepped speculatively per iteration:
+ *                0..n_buckets, or SO_ALL for n_buckets
+ *   info         optional (host): filled with the sizes to allocate
+ * Errors: SO_ERR_INVALID_ARG, SO_ERR_NOMEM.
+ */
+so_status so_layout_init(so_ctx **out, int32_t n_tensors, const int64_t *numel,
+                         int64_t bucket_elems, int32_t grad_dtype, int32_t undo_slots,
+                         so_layout_info *info);
+
+/* Copy of the layout description.  Host-only. */
+so_status so_layout_get_info(const so_ctx *ctx, so_layout_info *info);
+
+/* Where tensor i lives: its flat offset and the first/last bucket it touches
+ * (first > last for an empty tensor).  Host-only. */
+so_status so_layout_tensor(const so_ctx *ctx, int32_t i, int64_t *flat_offset,
+                           int32_t *first_bucket, int32_t *last_bucket);
+
+/*
+ * so_layout_bind -- hand the caller-owned DEVICE arenas to the context.
+ * Sizes as reported by so_layout_init; pointers 256-byte aligned; master, m, v
+ * are fp32, grad is bf16 or fp32 per grad_dtype, param_bf16 is bf16.  The
+ * caller fills master/m/v slot b with bucket b's initial state (m = v = 0 for
+ * a fresh optimizer) and normally calls so_cast_params(SO_ALL) once.  Scratch
+ * needs no initialisation.  Records the current device.  No launch, no sync.
+ */
+so_status so_layout_bind(so_ctx *ctx, void *master, void *m, void *v, void *grad,
+                         void *param_bf16, void *scratch);
+
+/*
+ * so_grad_check -- the global gradient check (Section 4.4: the global
+ * gradient norm needed for clipping and the global NaN/Inf check).
+ *   bucket >= 0 : enqueue the sum of squares + non-finite scan of that bucket's
+ *                 gradients (a bucket that was stepped speculatively already
+ *                 has them: SO_ERR_STATE).  `hp` and `out` are ignored.
+ *   bucket == SO_ALL : scan every bucket not yet covered this iteration, reduce
+ *                 per bucket and over buckets, and fill `out` (host, may be
+ *                 NULL) with sumsq, norm, clip coefficient for
+ *                 hp->max_grad_norm, and the flag.  Synchronises `stream`.
+ * The reduction order is fixed (independent of grid size and of whether the
+ * scan ran inside the fused step), so results repeat bit for bit.
+ */
+so_status so_grad_check(so_ctx *ctx, const so_hparams *hp, int32_t bucket, void *stream,
+                        so_grad_stats *out);
+
+/*
+ * so_adam_step_speculative -- step a bucket before validation has finished
+ * (Section 4.4: the optimizer starts with the gradients available, assuming
+ * finite values and no clipping).  One fused kernel reads bf16/fp32 gradients
+ * and the fp32 master/m/v of the bucket, writes the new fp32 state into a free
+ * slot and the bf16 parameter copy in the same pass, and leaves the tile sums
+ * of g^2 in scratch as a by-product; the old state stays where it is, which is
+ * everything an undo needs.  AdamW with bias correction for step t+1, gradient
+ * scale 1.
+ *   bucket >= 0 : that bucket.  SO_ERR_STATE if already covered this iteration,
+ *                 SO_ERR_UNDO_EXHAUSTED if no slot is free (check it with
+ *                 so_grad_check instead; validation then steps it in place).
+ *   bucket == SO_ALL : every uncovered bucket, in index order, for as long as
+ *                 slots are free (batched launches); never UNDO_EXHAUSTED.
+ * All speculative steps of one iteration must use equal hyper-parameters.
+ * Enqueues only; no synchronisation.
+ */
+so_status so_adam_step_speculative(so_ctx *ctx, const so_hparams *hp, int32_t bucket,
+                                   void *stream);
+
+/*
+ * so_validate_commit_or_rollback -- end the iteration (Section 4.4: after
+ * validation, either keep the speculative update, skip the iteration when a
+ * NaN/Inf was found, or revert it and re-execute with clipped gradients).
+ * Completes the gradient check if so_grad_check(SO_ALL) has not run
+ * (synchronises `stream`), then
+ *   nonfinite          -> SKIP: speculative slots are dropped, the bf16 copy of
+ *                         those buckets is re-derived from the untouched master,
+ *                         the step count does not advance;
+ *   else clip_coef < 1 -> CLIP_RESTEP: every bucket is stepped from its
+ *                         untouched prior state with gradients scaled by
+ *                         clip_coef (same step index), then committed;
+ *   else               -> COMMIT: speculated buckets are re-pointed at their new
+ *                         slot (no device work); buckets that were only checked
+ *                         are stepped in place with scale 1.
+ * `hp` must equal the hyper-parameters of this iteration's speculative steps.
+ * `out` (host, may be NULL) receives the decision, statistics and step count.
+ * Follow-up kernels are enqueued on `stream`; the call does not wait for them.
+ */
+so_status so_validate_commit_or_rollback(so_ctx *ctx, const so_hparams *hp, void *stream,
+                                         so_step_result *out);
+
+/*
+ * so_cast_params -- fp32 master -> bf16 parameter copy, round to nearest even
+ * (Section 4.5: the cast runs on the GPU).  bucket >= 0 or SO_ALL.  Only
+ * between iterations (SO_ERR_STATE while buckets are covered).  Enqueues only.
+ */
+so_status so_cast_params(so_ctx *ctx, int32_t bucket, void *stream);
+
+/* Slot of the state arenas that holds bucket b's committed master/m/v. */
+so_status so_bucket_slot(const so_ctx *ctx, int32_t bucket, int32_t *slot);
+
+/* Committed step count t (starts at 0); so_set_step restores it on resume
+ * (only between iterations). */
+so_status so_get_step(const so_ctx *ctx, int64_t *t);
+so_status so_set_step(so_ctx *ctx, int64_t t);
+
+/* Number of buckets not yet covered (stepped or checked) this iteration. */
+so_status so_pending_buckets(const so_ctx *ctx, int32_t *n);
+
+so_status so_get_counters(const so_ctx *ctx, so_counters *out);
+
+/* Raw cudaError_t of the last failing CUDA call on this context (0 if none). */
+int32_t so_last_cuda_error(const so_ctx *ctx);
+
+const char *so_strerror(so_status s);
+
+/* Frees the host-side context.  Never touches device memory. */
+void so_destroy(so_ctx *ctx);
+
+/*
+ * Host-logic test hooks.  In dry-run mode no CUDA call is made: launches are
+ * only counted, and the per-bucket check results come from
+ * so_debug_set_bucket_stats instead of the device.  This lets the slot map and
+ * the per-iteration state machine be exercised on a machine without a GPU.
+ */
+so_status so_debug_set_dry_run(so_ctx *ctx, int32_t on);
+so_status so_debug_set_bucket_stats(so_ctx *ctx, int32_t bucket, double sumsq,
+                                    int32_t nonfinite);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SUPEROFFLOAD_H */

@@ -1,0 +1,386 @@
+// Device code of the bucketized speculative AdamW library (sm_100a).
+//
+// Everything here is a streaming, HBM-bound pass: no reuse, no contraction, no
+// tensor cores.  The design rules are the ones that matter for such passes on
+// B200: perfectly coalesced 128-bit (fp32) and 64-bit (bf16) accesses, enough
+// independent bytes in flight per SM to cover DRAM latency, streaming cache
+// policy (nothing is read twice), a persistent grid sized from the SM count,
+// and no block-level synchronisation at all (the reduction is per warp).
+//
+// Work decomposition.  A bucket is cut into *tiles* of 1024 consecutive
+// elements; one warp owns one tile at a time (tiles are dealt round-robin to
+// all warps of the grid).  Inside a tile a warp sweeps 8 *rows* of 128
+// elements; lane l owns the *quad* of elements [4l, 4l+4) of each row, so a
+// warp-wide fp32 access is one contiguous 512-byte line set and a bf16 access
+// one contiguous 256-byte one.  The sum of squares of a tile is accumulated
+// per lane in row order, then folded across lanes with an xor-shuffle tree and
+// stored as one double per tile; a second tiny kernel folds the tiles of each
+// bucket in a fixed order.  The summation order therefore depends on nothing
+// but the data and the bucket geometry: the same bits come out whatever the
+// grid size, and whether the sums were produced by the fused step kernel or by
+// the stand-alone check kernel.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace so {
+
+constexpr int kTileElems = 1024;          // elements per warp tile
+constexpr int kRowElems = 128;            // 32 lanes x 4 elements
+constexpr int kRowsPerTile = kTileElems / kRowElems;
+constexpr int kThreads = 256;             // threads per block (8 warps)
+constexpr int kWarpsPerBlock = kThreads / 32;
+constexpr int kMaxBatch = 128;            // buckets per launch
+constexpr int kReduceThreads = 512;
+
+struct Geometry {
+    int64_t stride;                       // elements between slots
+    uint32_t tiles_per_slot;
+    uint32_t bucket_elems;
+    uint32_t last_elems;                  // elements in the last bucket
+    int32_t last_bucket;                  // its index (-1 if none)
+};
+
+// Per-step constants, all derived on the host in double precision.
+struct AdamScalars {
+    double beta1, omb1;                   // beta1, 1 - beta1
+    double beta2, omb2;
+    double rsqrt_bc2;                     // 1 / sqrt(1 - beta2^t)
+    double step_size;                     // lr / (1 - beta1^t)
+    double decay;                         // 1 - lr * wd
+    double eps;
+    double scale;                         // gradient scale (clip coefficient)
+};
+
+struct BucketEntry { int32_t bucket, src_slot, dst_slot; };
+
+struct StepArgs {
+    const void *grad;
+    float *master, *mom, *var;
+    uint16_t *param_bf16;
+    double *partials;
+    Geometry geo;
+    AdamScalars k;
+    int32_t n_entries;
+    BucketEntry e[kMaxBatch];
+};
+
+struct CheckArgs {
+    const void *grad;
+    double *partials;
+    Geometry geo;
+    int32_t n_entries;
+    int32_t bucket[kMaxBatch];
+};
+
+struct CastArgs {
+    const float *master;
+    uint16_t *param_bf16;
+    Geometry geo;
+    int32_t n_entries;
+    BucketEntry e[kMaxBatch];             // dst_slot unused
+};
+
+struct BucketStats { double sumsq; int32_t nonfinite; int32_t pad; };
+
+// ---------------------------------------------------------------------------
+// streaming loads / stores of one quad (4 consecutive elements)
+// ---------------------------------------------------------------------------
+
+__device__ __forceinline__ void load_quad(const float *base, uint32_t idx, uint32_t n, float (&x)[4])
+{
+    if (idx + 4 <= n) {
+        const float4 q = __ldcs(reinterpret_cast<const float4 *>(base + idx));
+        x[0] = q.x; x[1] = q.y; x[2] = q.z; x[3] = q.w;
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) x[j] = (idx + j < n) ? __ldcs(base + idx + j) : 0.0f;
+    }
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }
+
+__device__ __forceinline__ void load_quad(const uint16_t *base, uint32_t idx, uint32_t n, float (&x)[4])
+{
+    if (idx + 4 <= n) {
+        const uint2 q = __ldcs(reinterpret_cast<const uint2 *>(base + idx));
+        x[0] = __uint_as_float(q.x << 16);
+        x[1] = __uint_as_float(q.x & 0xFFFF0000u);
+        x[2] = __uint_as_float(q.y << 16);
+        x[3] = __uint_as_float(q.y & 0xFFFF0000u);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            x[j] = (idx + j < n) ? bf16_bits_to_float(__ldcs(base + idx + j)) : 0.0f;
+    }
+}
+
+__device__ __forceinline__ void store_quad(float *base, uint32_t idx, uint32_t n, const float (&x)[4])
+{
+    if (idx + 4 <= n) {
+        __stcs(reinterpret_cast<float4 *>(base + idx), make_float4(x[0], x[1], x[2], x[3]));
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (idx + j < n) __stcs(base + idx + j, x[j]);
+    }
+}
+
+// fp32 pair -> packed bf16 pair, round to nearest even (hardware cvt; NaN maps
+// to the canonical quiet NaN, denormals are kept).  `lo` lands in bits 0..15.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+__device__ __forceinline__ void store_quad_bf16(uint16_t *base, uint32_t idx, uint32_t n,
+                                                const float (&x)[4])
+{
+    const uint32_t w0 = pack_bf16x2(x[0], x[1]);
+    const uint32_t w1 = pack_bf16x2(x[2], x[3]);
+    if (idx + 4 <= n) {
+        __stcs(reinterpret_cast<uint2 *>(base + idx), make_uint2(w0, w1));
+    } else {
+        const uint16_t h[4] = {(uint16_t)(w0 & 0xFFFFu), (uint16_t)(w0 >> 16),
+                               (uint16_t)(w1 & 0xFFFFu), (uint16_t)(w1 >> 16)};
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (idx + j < n) __stcs(base + idx + j, h[j]);
+    }
+}
+
+// Fold a per-lane double across the warp with a fixed xor tree.
+__device__ __forceinline__ double warp_fold(double x)
+{
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1)
+        x = __dadd_rn(x, __shfl_xor_sync(0xFFFFFFFFu, x, off));
+    return x;
+}
+
+// ---------------------------------------------------------------------------
+// AdamW on one element, in double (Kingma & Ba Alg. 1 + decoupled decay)
+// ---------------------------------------------------------------------------
+//
+//   g~ = scale*g;  m' = b1*m + (1-b1)*g~;  v' = b2*v + (1-b2)*g~^2
+//   p' = p*(1 - lr*wd) - (lr/bc1) * m' / (sqrt(v')/sqrt(bc2) + eps)
+//
+// m' and v' are formed with separately rounded products and one add (no fused
+// multiply-add): with decimal betas the exact value often sits on an fp32
+// rounding tie, and only this evaluation order reproduces the reference
+// rounding of the stored moments bit for bit.  The parameter update hoists the
+// bias corrections into per-step scalars (one division and one square root per
+// element); it agrees with the textbook order to a few 1e-16 relative.
+template <bool kScaled>
+__device__ __forceinline__ void adamw_element(float g, float &p, float &m, float &v,
+                                              const AdamScalars &k, double &sumsq)
+{
+    const double gd = (double)g;
+    const double gs = kScaled ? __dmul_rn(gd, k.scale) : gd;
+    const double sq = __dmul_rn(gs, gs);
+    if (!kScaled) sumsq = __dadd_rn(sumsq, sq);
+    const double m64 = __dadd_rn(__dmul_rn(k.beta1, (double)m), __dmul_rn(k.omb1, gs));
+    const double v64 = __dadd_rn(__dmul_rn(k.beta2, (double)v), __dmul_rn(k.omb2, sq));
+    const double denom = __fma_rn(__dsqrt_rn(v64), k.rsqrt_bc2, k.eps);
+    const double u = __dmul_rn(k.step_size, __ddiv_rn(m64, denom));
+    const double p64 = __fma_rn((double)p, k.decay, -u);
+    p = __double2float_rn(p64);
+    m = __double2float_rn(m64);
+    v = __double2float_rn(v64);
+}
+
+// ---------------------------------------------------------------------------
+// fused step: g, p, m, v in -> p', m', v', bf16(p') out (+ tile sums of g^2)
+// ---------------------------------------------------------------------------
+//
+// kSpec = true : speculative step (scale 1, tile sums written).
+// kSpec = false: step with a known scale (re-step after a clip, or the in-place
+//                step of a bucket that was only checked); no sums.
+// Source and destination slots may be the same slot (in-place): every element
+// is read and written by the same thread, reads first.
+template <typename GradT, bool kSpec, int kRowsInFlight>
+__global__ void __launch_bounds__(kThreads, 2) adamw_step_kernel(const __grid_constant__ StepArgs a)
+{
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t warp = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
+    const uint32_t tps = a.geo.tiles_per_slot;
+    const uint32_t total_tiles = (uint32_t)a.n_entries * tps;
+
+    for (uint32_t tile = warp; tile < total_tiles; tile += n_warps) {
+        const uint32_t j = tile / tps;
+        const uint32_t lt = tile - j * tps;
+        const BucketEntry e = a.e[j];
+        const uint32_t n = (e.bucket == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
+        const uint32_t base = lt * kTileElems;
+        if (base >= n) continue;
+
+        const GradT *g = static_cast<const GradT *>(a.grad) + (int64_t)e.bucket * a.geo.stride;
+        const int64_t src = (int64_t)e.src_slot * a.geo.stride;
+        const int64_t dst = (int64_t)e.dst_slot * a.geo.stride;
+        const float *p_in = a.master + src, *m_in = a.mom + src, *v_in = a.var + src;
+        float *p_out = a.master + dst, *m_out = a.mom + dst, *v_out = a.var + dst;
+        uint16_t *pb = a.param_bf16 + (int64_t)e.bucket * a.geo.stride;
+
+        double acc = 0.0;
+#pragma unroll 1
+        for (int r0 = 0; r0 < kRowsPerTile; r0 += kRowsInFlight) {
+            if (base + r0 * kRowElems >= n) break;
+            float gq[kRowsInFlight][4], pq[kRowsInFlight][4], mq[kRowsInFlight][4],
+                vq[kRowsInFlight][4];
+#pragma unroll
+            for (int u = 0; u < kRowsInFlight; ++u) {
+                const uint32_t idx = base + (r0 + u) * kRowElems + lane * 4;
+                load_quad(g, idx, n, gq[u]);
+                load_quad(p_in, idx, n, pq[u]);
+                load_quad(m_in, idx, n, mq[u]);
+                load_quad(v_in, idx, n, vq[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < kRowsInFlight; ++u) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    adamw_element<!kSpec>(gq[u][q], pq[u][q], mq[u][q], vq[u][q], a.k, acc);
+                const uint32_t idx = base + (r0 + u) * kRowElems + lane * 4;
+                if (idx < n) {
+                    store_quad(p_out, idx, n, pq[u]);
+                    store_quad(m_out, idx, n, mq[u]);
+                    store_quad(v_out, idx, n, vq[u]);
+                    store_quad_bf16(pb, idx, n, pq[u]);
+                }
+            }
+        }
+        if (kSpec) {
+            acc = warp_fold(acc);
+            if (lane == 0) a.partials[(int64_t)e.bucket * tps + lt] = acc;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// stand-alone gradient scan: tile sums of g^2 (same order as the fused kernel)
+// ---------------------------------------------------------------------------
+template <typename GradT>
+__global__ void __launch_bounds__(kThreads) grad_check_kernel(const __grid_constant__ CheckArgs a)
+{
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t warp = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
+    const uint32_t tps = a.geo.tiles_per_slot;
+    const uint32_t total_tiles = (uint32_t)a.n_entries * tps;
+
+    for (uint32_t tile = warp; tile < total_tiles; tile += n_warps) {
+        const uint32_t j = tile / tps;
+        const uint32_t lt = tile - j * tps;
+        const int32_t b = a.bucket[j];
+        const uint32_t n = (b == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
+        const uint32_t base = lt * kTileElems;
+        if (base >= n) continue;
+        const GradT *g = static_cast<const GradT *>(a.grad) + (int64_t)b * a.geo.stride;
+
+        float gq[kRowsPerTile][4];
+#pragma unroll
+        for (int r = 0; r < kRowsPerTile; ++r) {
+            const uint32_t idx = base + r * kRowElems + lane * 4;
+            if (idx < n) {
+                load_quad(g, idx, n, gq[r]);
+            } else {
+                gq[r][0] = gq[r][1] = gq[r][2] = gq[r][3] = 0.0f;
+            }
+        }
+        double acc = 0.0;
+#pragma unroll
+        for (int r = 0; r < kRowsPerTile; ++r) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const double gd = (double)gq[r][q];
+                acc = __dadd_rn(acc, __dmul_rn(gd, gd));
+            }
+        }
+        acc = warp_fold(acc);
+        if (lane == 0) a.partials[(int64_t)b * tps + lt] = acc;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// per-bucket fold of the tile sums (fixed order) + non-finite flag
+// ---------------------------------------------------------------------------
+//
+// g^2 is formed in double, so it cannot overflow for a finite fp32/bf16 input,
+// and a sum of non-negative finite doubles this long cannot overflow either: a
+// tile sum is Inf or NaN exactly when the tile holds a NaN or an infinity.
+__global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(const double *partials,
+                                                                      BucketStats *stats,
+                                                                      Geometry geo)
+{
+    __shared__ double s_sum[kReduceThreads];
+    __shared__ int s_bad[kReduceThreads];
+    const int32_t b = blockIdx.x;
+    const uint32_t n = (b == geo.last_bucket) ? geo.last_elems : geo.bucket_elems;
+    const uint32_t n_tiles = (n + kTileElems - 1) / kTileElems;
+    const double *src = partials + (int64_t)b * geo.tiles_per_slot;
+
+    double acc = 0.0;
+    int bad = 0;
+    for (uint32_t i = threadIdx.x; i < n_tiles; i += kReduceThreads) {
+        const double x = src[i];
+        const uint32_t hi = (uint32_t)__double2hiint(x);
+        bad |= ((hi & 0x7FF00000u) == 0x7FF00000u);
+        acc = __dadd_rn(acc, x);
+    }
+    s_sum[threadIdx.x] = acc;
+    s_bad[threadIdx.x] = bad;
+    __syncthreads();
+    for (int s = kReduceThreads / 2; s > 0; s >>= 1) {
+        if ((int)threadIdx.x < s) {
+            s_sum[threadIdx.x] = __dadd_rn(s_sum[threadIdx.x], s_sum[threadIdx.x + s]);
+            s_bad[threadIdx.x] |= s_bad[threadIdx.x + s];
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        stats[b].sumsq = s_sum[0];
+        stats[b].nonfinite = s_bad[0];
+        stats[b].pad = 0;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// stand-alone cast: fp32 master (slot src) -> bf16 copy of the bucket
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) cast_params_kernel(const __grid_constant__ CastArgs a)
+{
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t warp = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
+    const uint32_t tps = a.geo.tiles_per_slot;
+    const uint32_t total_tiles = (uint32_t)a.n_entries * tps;
+
+    for (uint32_t tile = warp; tile < total_tiles; tile += n_warps) {
+        const uint32_t j = tile / tps;
+        const uint32_t lt = tile - j * tps;
+        const BucketEntry e = a.e[j];
+        const uint32_t n = (e.bucket == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
+        const uint32_t base = lt * kTileElems;
+        if (base >= n) continue;
+        const float *p = a.master + (int64_t)e.src_slot * a.geo.stride;
+        uint16_t *pb = a.param_bf16 + (int64_t)e.bucket * a.geo.stride;
+
+        float pq[kRowsPerTile][4];
+#pragma unroll
+        for (int r = 0; r < kRowsPerTile; ++r) {
+            const uint32_t idx = base + r * kRowElems + lane * 4;
+            if (idx < n) load_quad(p, idx, n, pq[r]);
+        }
+#pragma unroll
+        for (int r = 0; r < kRowsPerTile; ++r) {
+            const uint32_t idx = base + r * kRowElems + lane * 4;
+            if (idx < n) store_quad_bf16(pb, idx, n, pq[r]);
+        }
+    }
+}
+
+}  // namespace so

@@ -1,0 +1,679 @@
+// Host side of the bucketized speculative AdamW library: layout arithmetic,
+// the slot map, the per-iteration state machine, and the kernel launches.
+// The C ABI is documented in include/superoffload.h.
+#include "superoffload.h"
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "so_kernels.cuh"
+
+using namespace so;
+
+namespace {
+
+enum Phase { kIdle = 0, kOpen = 1, kChecked = 2 };
+enum Cover : uint8_t { kNone = 0, kCheckedOnly = 1, kSpeculated = 2 };
+
+}  // namespace
+
+struct so_ctx {
+    // ---- layout (immutable after init) ----
+    std::vector<int64_t> numel, offsets;
+    int64_t total = 0, bucket_elems = 0, stride = 0, last_elems = 0, tiles_per_slot = 0;
+    int32_t n_buckets = 0, undo_slots = 0, n_slots = 0, grad_dtype = SO_GRAD_BF16;
+    // ---- binding ----
+    bool bound = false;
+    int device = -1, num_sms = 0;
+    float *master = nullptr, *mom = nullptr, *var = nullptr;
+    void *grad = nullptr;
+    uint16_t *param_bf16 = nullptr;
+    double *d_partials = nullptr;
+    BucketStats *d_stats = nullptr;
+    BucketStats *h_stats = nullptr;
+    bool h_stats_pinned = false;
+    int occ_step = 0, occ_check = 0, occ_cast = 0;
+    // ---- slot map ----
+    std::vector<int32_t> slot_of;       // committed slot of each bucket
+    std::vector<int32_t> spec_slot;     // slot holding the speculative result, or -1
+    std::vector<int32_t> free_slots;
+    // ---- iteration state ----
+    int phase = kIdle;
+    std::vector<uint8_t> cover;
+    int32_t n_covered = 0, n_speculated = 0;
+    bool have_hp = false;
+    so_hparams hp_iter{};
+    so_grad_stats stats{};
+    int64_t t = 0;
+    // ---- bookkeeping ----
+    so_counters counters{};
+    int32_t last_cuda_error = 0;
+    bool dry_run = false;
+    std::vector<BucketStats> injected;
+};
+
+namespace {
+
+Geometry geometry_of(const so_ctx *c)
+{
+    Geometry g;
+    g.stride = c->stride;
+    g.tiles_per_slot = (uint32_t)c->tiles_per_slot;
+    g.bucket_elems = (uint32_t)c->bucket_elems;
+    g.last_elems = (uint32_t)c->last_elems;
+    g.last_bucket = c->n_buckets - 1;
+    return g;
+}
+
+int64_t elems_of(const so_ctx *c, int32_t b)
+{
+    return b == c->n_buckets - 1 ? c->last_elems : c->bucket_elems;
+}
+
+so_status cuda_fail(so_ctx *c, cudaError_t e)
+{
+    c->last_cuda_error = (int32_t)e;
+    return SO_ERR_CUDA;
+}
+
+bool hparams_ok(const so_hparams *hp)
+{
+    if (!hp) return false;
+    const double vals[] = {hp->lr, hp->beta1, hp->beta2, hp->eps, hp->weight_decay,
+                           hp->max_grad_norm};
+    for (double x : vals)
+        if (!std::isfinite(x)) return false;
+    return hp->lr >= 0.0 && hp->beta1 >= 0.0 && hp->beta1 < 1.0 && hp->beta2 >= 0.0 &&
+           hp->beta2 < 1.0 && hp->eps >= 0.0 && hp->weight_decay >= 0.0;
+}
+
+bool hparams_equal(const so_hparams &a, const so_hparams &b)
+{
+    return std::memcmp(&a, &b, sizeof(so_hparams)) == 0;
+}
+
+AdamScalars scalars_for(const so_hparams &hp, int64_t step_index, double scale)
+{
+    const double bc1 = 1.0 - std::pow(hp.beta1, (double)step_index);
+    const double bc2 = 1.0 - std::pow(hp.beta2, (double)step_index);
+    AdamScalars k;
+    k.beta1 = hp.beta1;
+    k.omb1 = 1.0 - hp.beta1;
+    k.beta2 = hp.beta2;
+    k.omb2 = 1.0 - hp.beta2;
+    k.rsqrt_bc2 = 1.0 / std::sqrt(bc2);
+    k.step_size = hp.lr / bc1;
+    k.decay = 1.0 - hp.lr * hp.weight_decay;
+    k.eps = hp.eps;
+    k.scale = scale;
+    return k;
+}
+
+double clip_coef_of(double norm, double max_norm)
+{
+    if (!(max_norm > 0.0)) return 1.0;
+    const double c = max_norm / (norm + 1e-6);
+    return c < 1.0 ? c : 1.0;
+}
+
+// Persistent grid: enough blocks to fill every SM at the kernel's occupancy,
+// never more than there are tiles to hand out.
+unsigned grid_for(const so_ctx *c, int64_t total_tiles, int blocks_per_sm)
+{
+    int64_t want = (total_tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    int64_t cap = (int64_t)c->num_sms * (blocks_per_sm > 0 ? blocks_per_sm : 1);
+    if (want > cap) want = cap;
+    if (want < 1) want = 1;
+    return (unsigned)want;
+}
+
+so_status after_launch(so_ctx *c)
+{
+    c->counters.kernel_launches += 1;
+    if (c->dry_run) return SO_OK;
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? SO_OK : cuda_fail(c, e);
+}
+
+// ---- launches --------------------------------------------------------------
+
+// Step the listed buckets (src slot -> dst slot).  speculative: scale 1 and
+// tile sums written; otherwise the given scale and no sums.
+so_status launch_steps(so_ctx *c, const std::vector<BucketEntry> &entries, const so_hparams &hp,
+                       bool speculative, double scale, cudaStream_t stream)
+{
+    const Geometry geo = geometry_of(c);
+    for (size_t first = 0; first < entries.size(); first += kMaxBatch) {
+        const int n = (int)std::min<size_t>(kMaxBatch, entries.size() - first);
+        StepArgs a;
+        a.grad = c->grad;
+        a.master = c->master;
+        a.mom = c->mom;
+        a.var = c->var;
+        a.param_bf16 = c->param_bf16;
+        a.partials = c->d_partials;
+        a.geo = geo;
+        a.k = scalars_for(hp, c->t + 1, scale);
+        a.n_entries = n;
+        for (int i = 0; i < n; ++i) {
+            a.e[i] = entries[first + i];
+            c->counters.elems_stepped += elems_of(c, a.e[i].bucket);
+        }
+        for (int i = n; i < kMaxBatch; ++i) a.e[i] = BucketEntry{0, 0, 0};
+        if (!c->dry_run) {
+            const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_step);
+            const bool bf16 = c->grad_dtype == SO_GRAD_BF16;
+            if (speculative) {
+                if (bf16) adamw_step_kernel<uint16_t, true, 4><<<grid, kThreads, 0, stream>>>(a);
+                else adamw_step_kernel<float, true, 4><<<grid, kThreads, 0, stream>>>(a);
+            } else {
+                if (bf16) adamw_step_kernel<uint16_t, false, 4><<<grid, kThreads, 0, stream>>>(a);
+                else adamw_step_kernel<float, false, 4><<<grid, kThreads, 0, stream>>>(a);
+            }
+        }
+        const so_status s = after_launch(c);
+        if (s != SO_OK) return s;
+    }
+    return SO_OK;
+}
+
+so_status launch_checks(so_ctx *c, const std::vector<int32_t> &buckets, cudaStream_t stream)
+{
+    const Geometry geo = geometry_of(c);
+    for (size_t first = 0; first < buckets.size(); first += kMaxBatch) {
+        const int n = (int)std::min<size_t>(kMaxBatch, buckets.size() - first);
+        CheckArgs a;
+        a.grad = c->grad;
+        a.partials = c->d_partials;
+        a.geo = geo;
+        a.n_entries = n;
+        for (int i = 0; i < n; ++i) {
+            a.bucket[i] = buckets[first + i];
+            c->counters.elems_checked += elems_of(c, a.bucket[i]);
+        }
+        for (int i = n; i < kMaxBatch; ++i) a.bucket[i] = 0;
+        if (!c->dry_run) {
+            const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_check);
+            if (c->grad_dtype == SO_GRAD_BF16)
+                grad_check_kernel<uint16_t><<<grid, kThreads, 0, stream>>>(a);
+            else
+                grad_check_kernel<float><<<grid, kThreads, 0, stream>>>(a);
+        }
+        const so_status s = after_launch(c);
+        if (s != SO_OK) return s;
+    }
+    return SO_OK;
+}
+
+so_status launch_casts(so_ctx *c, const std::vector<BucketEntry> &entries, cudaStream_t stream)
+{
+    const Geometry geo = geometry_of(c);
+    for (size_t first = 0; first < entries.size(); first += kMaxBatch) {
+        const int n = (int)std::min<size_t>(kMaxBatch, entries.size() - first);
+        CastArgs a;
+        a.master = c->master;
+        a.param_bf16 = c->param_bf16;
+        a.geo = geo;
+        a.n_entries = n;
+        for (int i = 0; i < n; ++i) {
+            a.e[i] = entries[first + i];
+            c->counters.elems_cast += elems_of(c, a.e[i].bucket);
+        }
+        for (int i = n; i < kMaxBatch; ++i) a.e[i] = BucketEntry{0, 0, 0};
+        if (!c->dry_run) {
+            const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_cast);
+            cast_params_kernel<<<grid, kThreads, 0, stream>>>(a);
+        }
+        const so_status s = after_launch(c);
+        if (s != SO_OK) return s;
+    }
+    return SO_OK;
+}
+
+// Finish the gradient check: scan what is still uncovered, fold per bucket on
+// the device, bring the per-bucket results to the host, fold over buckets in
+// index order, derive norm and clip coefficient.  Synchronises the stream.
+so_status finalize_check(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
+{
+    std::vector<int32_t> todo;
+    for (int32_t b = 0; b < c->n_buckets; ++b)
+        if (c->cover[b] == kNone) todo.push_back(b);
+    if (!todo.empty()) {
+        const so_status s = launch_checks(c, todo, stream);
+        if (s != SO_OK) return s;
+        for (int32_t b : todo) c->cover[b] = kCheckedOnly;
+        c->n_covered = c->n_buckets;
+    }
+    if (c->n_buckets > 0) {
+        if (!c->dry_run) {
+            bucket_reduce_kernel<<<(unsigned)c->n_buckets, kReduceThreads, 0, stream>>>(
+                c->d_partials, c->d_stats, geometry_of(c));
+        }
+        so_status s = after_launch(c);
+        if (s != SO_OK) return s;
+        if (!c->dry_run) {
+            cudaError_t e = cudaMemcpyAsync(c->h_stats, c->d_stats,
+                                            sizeof(BucketStats) * (size_t)c->n_buckets,
+                                            cudaMemcpyDeviceToHost, stream);
+            if (e != cudaSuccess) return cuda_fail(c, e);
+            e = cudaStreamSynchronize(stream);
+            if (e != cudaSuccess) return cuda_fail(c, e);
+        } else {
+            for (int32_t b = 0; b < c->n_buckets; ++b) c->h_stats[b] = c->injected[b];
+        }
+    }
+    double sumsq = 0.0;
+    int32_t nonfinite = 0;
+    for (int32_t b = 0; b < c->n_buckets; ++b) {
+        sumsq += c->h_stats[b].sumsq;
+        nonfinite |= (c->h_stats[b].nonfinite != 0);
+    }
+    c->stats.sumsq = sumsq;
+    c->stats.norm = std::sqrt(sumsq);
+    c->stats.clip_coef = clip_coef_of(c->stats.norm, hp.max_grad_norm);
+    c->stats.nonfinite = nonfinite;
+    c->stats.reserved = 0;
+    c->phase = kChecked;
+    return SO_OK;
+}
+
+void end_iteration(so_ctx *c)
+{
+    std::fill(c->cover.begin(), c->cover.end(), (uint8_t)kNone);
+    std::fill(c->spec_slot.begin(), c->spec_slot.end(), -1);
+    c->n_covered = 0;
+    c->n_speculated = 0;
+    c->have_hp = false;
+    c->phase = kIdle;
+}
+
+so_status note_hparams(so_ctx *c, const so_hparams *hp)
+{
+    if (!hparams_ok(hp)) return SO_ERR_INVALID_ARG;
+    if (c->have_hp && !hparams_equal(c->hp_iter, *hp)) return SO_ERR_INVALID_ARG;
+    return SO_OK;
+}
+
+}  // namespace
+
+// ============================================================================
+// C ABI
+// ============================================================================
+
+extern "C" {
+
+so_status so_layout_init(so_ctx **out, int32_t n_tensors, const int64_t *numel,
+                         int64_t bucket_elems, int32_t grad_dtype, int32_t undo_slots,
+                         so_layout_info *info)
+{
+    if (!out || n_tensors < 0 || (n_tensors > 0 && !numel)) return SO_ERR_INVALID_ARG;
+    if (bucket_elems < 1 || bucket_elems > ((int64_t)1 << 30)) return SO_ERR_INVALID_ARG;
+    if (grad_dtype != SO_GRAD_BF16 && grad_dtype != SO_GRAD_FP32) return SO_ERR_INVALID_ARG;
+    int64_t total = 0;
+    for (int32_t i = 0; i < n_tensors; ++i) {
+        if (numel[i] < 0 || numel[i] > ((int64_t)1 << 46)) return SO_ERR_INVALID_ARG;
+        total += numel[i];
+        if (total > ((int64_t)1 << 46)) return SO_ERR_INVALID_ARG;
+    }
+    const int64_t nb64 = (total + bucket_elems - 1) / bucket_elems;
+    if (nb64 > (1 << 24)) return SO_ERR_INVALID_ARG;
+    const int32_t nb = (int32_t)nb64;
+    if (undo_slots == SO_ALL) undo_slots = nb;
+    if (undo_slots < 0 || undo_slots > nb) return SO_ERR_INVALID_ARG;
+
+    so_ctx *c = new (std::nothrow) so_ctx();
+    if (!c) return SO_ERR_NOMEM;
+    try {
+        c->numel.assign(numel, numel + n_tensors);
+        c->offsets.resize(n_tensors);
+        int64_t off = 0;
+        for (int32_t i = 0; i < n_tensors; ++i) { c->offsets[i] = off; off += numel[i]; }
+        c->total = total;
+        c->bucket_elems = bucket_elems;
+        c->stride = (bucket_elems + 63) / 64 * 64;
+        c->n_buckets = nb;
+        c->last_elems = nb == 0 ? 0 : total - (int64_t)(nb - 1) * bucket_elems;
+        c->tiles_per_slot = (c->stride + kTileElems - 1) / kTileElems;
+        c->undo_slots = undo_slots;
+        c->n_slots = nb + undo_slots;
+        c->grad_dtype = grad_dtype;
+        c->slot_of.resize(nb);
+        for (int32_t b = 0; b < nb; ++b) c->slot_of[b] = b;
+        c->spec_slot.assign(nb, -1);
+        for (int32_t s = c->n_slots - 1; s >= nb; --s) c->free_slots.push_back(s);
+        c->cover.assign(nb, (uint8_t)kNone);
+        c->injected.assign(nb, BucketStats{0.0, 0, 0});
+    } catch (...) {
+        delete c;
+        return SO_ERR_NOMEM;
+    }
+    *out = c;
+    if (info) so_layout_get_info(c, info);
+    return SO_OK;
+}
+
+so_status so_layout_get_info(const so_ctx *c, so_layout_info *info)
+{
+    if (!c || !info) return SO_ERR_INVALID_ARG;
+    std::memset(info, 0, sizeof(*info));
+    info->total_elems = c->total;
+    info->bucket_elems = c->bucket_elems;
+    info->slot_stride_elems = c->stride;
+    info->last_bucket_elems = c->last_elems;
+    info->n_buckets = c->n_buckets;
+    info->n_tensors = (int32_t)c->numel.size();
+    info->n_state_slots = c->n_slots;
+    info->undo_slots = c->undo_slots;
+    info->grad_dtype = c->grad_dtype;
+    info->tile_elems = kTileElems;
+    info->tiles_per_slot = c->tiles_per_slot;
+    const uint64_t state = (uint64_t)c->n_slots * (uint64_t)c->stride * 4u;
+    info->bytes_master = info->bytes_m = info->bytes_v = state;
+    info->bytes_grad = (uint64_t)c->n_buckets * (uint64_t)c->stride *
+                       (c->grad_dtype == SO_GRAD_BF16 ? 2u : 4u);
+    info->bytes_param_bf16 = (uint64_t)c->n_buckets * (uint64_t)c->stride * 2u;
+    const uint64_t partial_bytes = (uint64_t)c->n_buckets * (uint64_t)c->tiles_per_slot * 8u;
+    const uint64_t stats_bytes = (uint64_t)c->n_buckets * sizeof(BucketStats);
+    info->bytes_scratch = (partial_bytes + 255u) / 256u * 256u + stats_bytes + 256u;
+    return SO_OK;
+}
+
+so_status so_layout_tensor(const so_ctx *c, int32_t i, int64_t *flat_offset,
+                           int32_t *first_bucket, int32_t *last_bucket)
+{
+    if (!c || i < 0 || i >= (int32_t)c->numel.size()) return SO_ERR_INVALID_ARG;
+    const int64_t off = c->offsets[i], n = c->numel[i];
+    if (flat_offset) *flat_offset = off;
+    const int32_t fb = (int32_t)(off / c->bucket_elems);
+    const int32_t lb = n > 0 ? (int32_t)((off + n - 1) / c->bucket_elems) : fb - 1;
+    if (first_bucket) *first_bucket = fb;
+    if (last_bucket) *last_bucket = lb;
+    return SO_OK;
+}
+
+so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
+                         void *param_bf16, void *scratch)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (c->phase != kIdle) return SO_ERR_STATE;
+    void *ptrs[] = {master, m, v, grad, param_bf16, scratch};
+    for (void *p : ptrs) {
+        if (c->n_buckets > 0 && !p) return SO_ERR_INVALID_ARG;
+        if ((reinterpret_cast<uintptr_t>(p) & 255u) != 0) return SO_ERR_INVALID_ARG;
+    }
+    if (!c->dry_run) {
+        cudaError_t e = cudaGetDevice(&c->device);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, c->device);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        const bool bf16 = c->grad_dtype == SO_GRAD_BF16;
+        e = bf16 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                       &c->occ_step, adamw_step_kernel<uint16_t, true, 4>, kThreads, 0)
+                 : cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                       &c->occ_step, adamw_step_kernel<float, true, 4>, kThreads, 0);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        e = bf16 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                       &c->occ_check, grad_check_kernel<uint16_t>, kThreads, 0)
+                 : cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                       &c->occ_check, grad_check_kernel<float>, kThreads, 0);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_cast, cast_params_kernel,
+                                                          kThreads, 0);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+    } else {
+        c->num_sms = 148;
+        c->occ_step = c->occ_check = c->occ_cast = 2;
+    }
+    if (!c->h_stats) {
+        const size_t bytes = sizeof(BucketStats) * (size_t)(c->n_buckets > 0 ? c->n_buckets : 1);
+        if (!c->dry_run && cudaMallocHost(reinterpret_cast<void **>(&c->h_stats), bytes) ==
+                               cudaSuccess) {
+            c->h_stats_pinned = true;
+        } else {
+            if (!c->dry_run) cudaGetLastError();      // clear the failed pinned allocation
+            c->h_stats = static_cast<BucketStats *>(std::malloc(bytes));
+            if (!c->h_stats) return SO_ERR_NOMEM;
+        }
+    }
+    c->master = static_cast<float *>(master);
+    c->mom = static_cast<float *>(m);
+    c->var = static_cast<float *>(v);
+    c->grad = grad;
+    c->param_bf16 = static_cast<uint16_t *>(param_bf16);
+    c->d_partials = static_cast<double *>(scratch);
+    const uint64_t partial_bytes = (uint64_t)c->n_buckets * (uint64_t)c->tiles_per_slot * 8u;
+    c->d_stats = reinterpret_cast<BucketStats *>(static_cast<char *>(scratch) +
+                                                 (partial_bytes + 255u) / 256u * 256u);
+    c->bound = true;
+    return SO_OK;
+}
+
+so_status so_grad_check(so_ctx *c, const so_hparams *hp, int32_t bucket, void *stream,
+                        so_grad_stats *out)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (!c->bound) return SO_ERR_STATE;
+    if (c->phase == kChecked) return SO_ERR_STATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (bucket == SO_ALL) {
+        so_status s = note_hparams(c, hp);
+        if (s != SO_OK) return s;
+        s = finalize_check(c, *hp, st);
+        if (s != SO_OK) return s;
+        if (!c->have_hp) { c->hp_iter = *hp; c->have_hp = true; }
+        if (out) *out = c->stats;
+        return SO_OK;
+    }
+    if (bucket < 0 || bucket >= c->n_buckets) return SO_ERR_INVALID_ARG;
+    if (c->cover[bucket] != kNone) return SO_ERR_STATE;
+    const so_status s = launch_checks(c, std::vector<int32_t>{bucket}, st);
+    if (s != SO_OK) return s;
+    c->cover[bucket] = kCheckedOnly;
+    c->n_covered += 1;
+    c->phase = kOpen;
+    return SO_OK;
+}
+
+so_status so_adam_step_speculative(so_ctx *c, const so_hparams *hp, int32_t bucket, void *stream)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (!c->bound) return SO_ERR_STATE;
+    if (c->phase == kChecked) return SO_ERR_STATE;
+    so_status s = note_hparams(c, hp);
+    if (s != SO_OK) return s;
+    if (bucket != SO_ALL && (bucket < 0 || bucket >= c->n_buckets)) return SO_ERR_INVALID_ARG;
+
+    std::vector<BucketEntry> entries;
+    if (bucket == SO_ALL) {
+        size_t free_left = c->free_slots.size();
+        for (int32_t b = 0; b < c->n_buckets && free_left > 0; ++b)
+            if (c->cover[b] == kNone) {
+                entries.push_back(BucketEntry{b, c->slot_of[b], c->free_slots[free_left - 1]});
+                --free_left;
+            }
+    } else {
+        if (c->cover[bucket] != kNone) return SO_ERR_STATE;
+        if (c->free_slots.empty()) return SO_ERR_UNDO_EXHAUSTED;
+        entries.push_back(BucketEntry{bucket, c->slot_of[bucket], c->free_slots.back()});
+    }
+    if (entries.empty()) return SO_OK;
+    s = launch_steps(c, entries, *hp, /*speculative=*/true, 1.0, static_cast<cudaStream_t>(stream));
+    if (s != SO_OK) return s;
+    for (const BucketEntry &e : entries) {
+        c->free_slots.pop_back();
+        c->spec_slot[e.bucket] = e.dst_slot;
+        c->cover[e.bucket] = kSpeculated;
+    }
+    c->n_covered += (int32_t)entries.size();
+    c->n_speculated += (int32_t)entries.size();
+    if (!c->have_hp) { c->hp_iter = *hp; c->have_hp = true; }
+    c->phase = kOpen;
+    return SO_OK;
+}
+
+so_status so_validate_commit_or_rollback(so_ctx *c, const so_hparams *hp, void *stream,
+                                         so_step_result *out)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (!c->bound) return SO_ERR_STATE;
+    so_status s = note_hparams(c, hp);
+    if (s != SO_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (c->phase != kChecked) {
+        s = finalize_check(c, *hp, st);
+        if (s != SO_OK) return s;
+    }
+    // the coefficient always follows the hyper-parameters given here
+    c->stats.clip_coef = clip_coef_of(c->stats.norm, hp->max_grad_norm);
+
+    int32_t decision;
+    if (c->stats.nonfinite) decision = SO_DECISION_SKIP;
+    else if (c->stats.clip_coef < 1.0) decision = SO_DECISION_CLIP_RESTEP;
+    else decision = SO_DECISION_COMMIT;
+
+    const int32_t n_spec = c->n_speculated;
+    if (decision == SO_DECISION_SKIP) {
+        // drop the speculative slots; the bf16 copy of those buckets was
+        // overwritten by the speculative step and is re-derived from the old master
+        std::vector<BucketEntry> recast;
+        for (int32_t b = 0; b < c->n_buckets; ++b)
+            if (c->cover[b] == kSpeculated) recast.push_back(BucketEntry{b, c->slot_of[b], 0});
+        if (!recast.empty()) {
+            s = launch_casts(c, recast, st);
+            if (s != SO_OK) return s;
+        }
+        for (int32_t b = 0; b < c->n_buckets; ++b)
+            if (c->cover[b] == kSpeculated) c->free_slots.push_back(c->spec_slot[b]);
+        c->counters.skips += 1;
+    } else {
+        const bool clip = decision == SO_DECISION_CLIP_RESTEP;
+        // buckets to (re-)step with the validated scale: all of them after a
+        // clip, only the never-speculated ones after a commit
+        std::vector<BucketEntry> work;
+        for (int32_t b = 0; b < c->n_buckets; ++b) {
+            if (c->cover[b] == kSpeculated) {
+                if (clip) work.push_back(BucketEntry{b, c->slot_of[b], c->spec_slot[b]});
+            } else {
+                work.push_back(BucketEntry{b, c->slot_of[b], c->slot_of[b]});
+            }
+        }
+        if (!work.empty()) {
+            s = launch_steps(c, work, *hp, /*speculative=*/false,
+                             clip ? c->stats.clip_coef : 1.0, st);
+            if (s != SO_OK) return s;
+        }
+        for (int32_t b = 0; b < c->n_buckets; ++b)
+            if (c->cover[b] == kSpeculated) {
+                c->free_slots.push_back(c->slot_of[b]);
+                c->slot_of[b] = c->spec_slot[b];
+            }
+        c->t += 1;
+        if (clip) c->counters.clip_resteps += 1; else c->counters.commits += 1;
+    }
+    if (out) {
+        out->decision = decision;
+        out->buckets_speculated = n_spec;
+        out->step_after = c->t;
+        out->stats = c->stats;
+    }
+    end_iteration(c);
+    return SO_OK;
+}
+
+so_status so_cast_params(so_ctx *c, int32_t bucket, void *stream)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (!c->bound || c->phase != kIdle) return SO_ERR_STATE;
+    if (bucket != SO_ALL && (bucket < 0 || bucket >= c->n_buckets)) return SO_ERR_INVALID_ARG;
+    std::vector<BucketEntry> entries;
+    if (bucket == SO_ALL) {
+        for (int32_t b = 0; b < c->n_buckets; ++b)
+            entries.push_back(BucketEntry{b, c->slot_of[b], 0});
+    } else {
+        entries.push_back(BucketEntry{bucket, c->slot_of[bucket], 0});
+    }
+    if (entries.empty()) return SO_OK;
+    return launch_casts(c, entries, static_cast<cudaStream_t>(stream));
+}
+
+so_status so_bucket_slot(const so_ctx *c, int32_t bucket, int32_t *slot)
+{
+    if (!c || !slot || bucket < 0 || bucket >= c->n_buckets) return SO_ERR_INVALID_ARG;
+    *slot = c->slot_of[bucket];
+    return SO_OK;
+}
+
+so_status so_get_step(const so_ctx *c, int64_t *t)
+{
+    if (!c || !t) return SO_ERR_INVALID_ARG;
+    *t = c->t;
+    return SO_OK;
+}
+
+so_status so_set_step(so_ctx *c, int64_t t)
+{
+    if (!c || t < 0) return SO_ERR_INVALID_ARG;
+    if (c->phase != kIdle) return SO_ERR_STATE;
+    c->t = t;
+    return SO_OK;
+}
+
+so_status so_pending_buckets(const so_ctx *c, int32_t *n)
+{
+    if (!c || !n) return SO_ERR_INVALID_ARG;
+    *n = c->n_buckets - c->n_covered;
+    return SO_OK;
+}
+
+so_status so_get_counters(const so_ctx *c, so_counters *out)
+{
+    if (!c || !out) return SO_ERR_INVALID_ARG;
+    *out = c->counters;
+    return SO_OK;
+}
+
+int32_t so_last_cuda_error(const so_ctx *c) { return c ? c->last_cuda_error : 0; }
+
+const char *so_strerror(so_status s)
+{
+    switch (s) {
+        case SO_OK: return "ok";
+        case SO_ERR_INVALID_ARG: return "invalid argument";
+        case SO_ERR_STATE: return "call not allowed in the current phase of the iteration";
+        case SO_ERR_CUDA: return "CUDA error (see so_last_cuda_error)";
+        case SO_ERR_UNDO_EXHAUSTED: return "no free slot for another speculative step";
+        case SO_ERR_NOMEM: return "host allocation failed";
+        case SO_ERR_UNSUPPORTED: return "unsupported";
+        default: return "unknown status";
+    }
+}
+
+void so_destroy(so_ctx *c)
+{
+    if (!c) return;
+    if (c->h_stats) {
+        if (c->h_stats_pinned) cudaFreeHost(c->h_stats);
+        else std::free(c->h_stats);
+    }
+    delete c;
+}
+
+so_status so_debug_set_dry_run(so_ctx *c, int32_t on)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (c->bound) return SO_ERR_STATE;
+    c->dry_run = on != 0;
+    return SO_OK;
+}
+
+so_status so_debug_set_bucket_stats(so_ctx *c, int32_t bucket, double sumsq, int32_t nonfinite)
+{
+    if (!c || bucket < 0 || bucket >= c->n_buckets) return SO_ERR_INVALID_ARG;
+    c->injected[bucket] = BucketStats{sumsq, nonfinite, 0};
+    return SO_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,143 @@
+"""Lock-step comparison of the CUDA path with the CPU oracle.
+
+Each iteration starts from the device's own pre-step state (copied to the
+host), runs the whole path on the GPU through the C ABI, replays the same
+iteration in the oracle, and compares element by element.  The clip
+coefficient feeds every element of a re-step at full precision, so the
+oracle's replay uses the coefficient the device found (compared separately
+against the oracle's own, to the norm tolerance)."""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+import torch
+
+import oracle
+from helpers import bf16_bits_to_f32, ulp_distance
+from paper_2509_21271_b200 import binding as B
+from paper_2509_21271_b200 import workloads as W
+from paper_2509_21271_b200.optimizer import BucketedAdamW
+
+# tolerances of the parity contract
+MAX_ULP_STATE = 2            # fp32 master / m / v, per element per step
+NORM_RTOL = 1e-5             # global norm vs the fp64 oracle
+
+
+def hparams_of(w: W.Workload) -> oracle.HParams:
+    return oracle.HParams(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
+                          weight_decay=w.weight_decay, max_grad_norm=w.max_grad_norm)
+
+
+def grads_to_numpy(g: torch.Tensor) -> np.ndarray:
+    """Device/host gradient tensor -> what the oracle takes (bits or fp32)."""
+    if g.dtype == torch.bfloat16:
+        return g.view(torch.int16).cpu().numpy().view(np.uint16)
+    return g.cpu().numpy()
+
+
+def bf16_to_numpy(t: torch.Tensor) -> np.ndarray:
+    return t.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+@dataclass
+class Report:
+    decisions: list = field(default_factory=list)
+    max_ulp: dict = field(default_factory=lambda: {"p": 0, "m": 0, "v": 0})
+    n_diff: dict = field(default_factory=lambda: {"p": 0, "m": 0, "v": 0})
+    n_elems: int = 0
+    max_norm_rel: float = 0.0
+    bf16_mismatch: int = 0
+
+
+def assert_bf16_consistent(pb_dev: np.ndarray, p_dev: np.ndarray, pb_orc: np.ndarray,
+                           p_orc: np.ndarray, rep: Report) -> None:
+    """The bf16 copy must be the RNE cast of the device's own master (bit
+    exact), hence equal to the oracle's wherever the masters agree and within
+    one bf16 ulp elsewhere."""
+    want = oracle.bf16_rne(p_dev)
+    assert np.array_equal(pb_dev, want), "bf16 copy is not the RNE cast of the device master"
+    same = p_dev.view(np.uint32) == p_orc.view(np.uint32)
+    assert np.array_equal(pb_dev[same], pb_orc[same])
+    if not same.all():
+        a = bf16_bits_to_f32(pb_dev[~same]).view(np.int32).astype(np.int64) >> 16
+        b = bf16_bits_to_f32(pb_orc[~same]).view(np.int32).astype(np.int64) >> 16
+        assert np.abs(a - b).max() <= 1
+        rep.bf16_mismatch += int((a != b).sum())
+
+
+def compare_state(dev, orc, rep: Report) -> None:
+    for name, a, b in zip(("p", "m", "v"), dev, orc):
+        d = ulp_distance(a, b)
+        mx = int(d.max()) if d.size else 0
+        assert mx <= MAX_ULP_STATE, f"{name}: {mx} ulp from the oracle"
+        rep.max_ulp[name] = max(rep.max_ulp[name], mx)
+        rep.n_diff[name] += int((d != 0).sum())
+    rep.n_elems += dev[0].size
+
+
+def check_stats(stats, orc_res, max_grad_norm: float, rep: Report) -> None:
+    """Device norm / coefficient / flag against the oracle's own."""
+    assert stats.nonfinite == orc_res.nonfinite
+    if orc_res.nonfinite:
+        return
+    assert np.isfinite(stats.norm)
+    rel = abs(stats.norm - orc_res.norm) / max(orc_res.norm, 1e-300)
+    assert rel <= NORM_RTOL, f"norm off by {rel:.3e}"
+    rep.max_norm_rel = max(rep.max_norm_rel, rel)
+    own_coef = oracle.clip_coef(orc_res.norm, max_grad_norm)
+    assert abs(stats.clip_coef - own_coef) <= NORM_RTOL * own_coef
+    assert (stats.clip_coef < 1.0) == (own_coef < 1.0)
+
+
+def run_lockstep(w: W.Workload, steps: int, undo_slots: int = B.SO_ALL,
+                 speculative: bool = True, guard_bands: bool = True):
+    """Full element-by-element parity over `steps` iterations of workload w."""
+    hp = hparams_of(w)
+    stream = torch.cuda.current_stream()
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, undo_slots,
+                        guard_bands=guard_bands)
+    p0 = W.initial_master(w, device="cuda")
+    opt.load_state(p0)
+    opt.cast_params(stream=stream)
+    torch.cuda.synchronize()
+
+    p = p0.cpu().numpy()
+    m = np.zeros_like(p)
+    v = np.zeros_like(p)
+    pb = bf16_to_numpy(opt.gather_param_bf16())
+    assert np.array_equal(pb, oracle.bf16_rne(p)), "initial cast differs from the oracle"
+    rep = Report()
+    t = 0
+    for step in range(1, steps + 1):
+        g = W.gradients(w, step, device="cuda")
+        opt.load_grads(g)
+        g_host = grads_to_numpy(g)
+        res = opt.iteration(hp, stream=stream, speculative=speculative)
+        torch.cuda.synchronize()
+
+        # oracle replay from the device's pre-step state
+        forced = res.stats.clip_coef if res.decision == B.SO_DECISION_CLIP_RESTEP else None
+        orc_res = oracle.iteration_stv(p, m, v, pb, g_host, w.bucket_elems, t, hp,
+                                       forced_coef=forced)
+        own_coef = oracle.clip_coef(orc_res.norm, hp.max_grad_norm)
+        own_decision = oracle.decision(orc_res.nonfinite, own_coef)
+        assert res.decision == own_decision == orc_res.decision, (step, res.decision, own_decision)
+        check_stats(res.stats, orc_res, hp.max_grad_norm, rep)
+        t = orc_res.step_after
+        assert res.step_after == t == opt.step_count
+        rep.decisions.append(res.decision)
+
+        dev = [x.cpu().numpy() for x in opt.gather_state()]
+        pb_dev = bf16_to_numpy(opt.gather_param_bf16())
+        compare_state(dev, (p, m, v), rep)
+        assert_bf16_consistent(pb_dev, dev[0], pb, p, rep)
+        if res.decision == B.SO_DECISION_SKIP:
+            for a, b in zip(dev, (p, m, v)):
+                assert a.tobytes() == b.tobytes(), "SKIP did not restore the state bit for bit"
+            assert pb_dev.tobytes() == pb.tobytes()
+        # next iteration starts from the device's state
+        p, m, v, pb = dev[0], dev[1], dev[2], pb_dev
+    if guard_bands:
+        assert opt.guard_bands_intact(), "a kernel wrote outside its arena"
+    return rep, opt

@@ -1,0 +1,263 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle
+on the same seeded inputs.  Tolerances: fp32 master/m/v within 2 ulp per
+element per step; global norm within 1e-5 relative; the bf16 copy is the exact
+RNE cast of the device master; flags, decisions and rollbacks bit-exact."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_harness import (Report, bf16_to_numpy, grads_to_numpy, hparams_of, run_lockstep)
+from helpers import is_bf16_nan
+from paper_2509_21271_b200 import binding as B
+from paper_2509_21271_b200 import build as so_build
+from paper_2509_21271_b200 import workloads as W
+from paper_2509_21271_b200.optimizer import BucketedAdamW
+
+pytestmark = pytest.mark.gpu
+
+C, S, R = B.SO_DECISION_COMMIT, B.SO_DECISION_SKIP, B.SO_DECISION_CLIP_RESTEP
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    so_build.build_library()
+    assert torch.cuda.is_available()
+    torch.cuda.set_device(0)
+
+
+def _state_bytes(opt):
+    return [x.cpu().numpy().tobytes() for x in opt.gather_state()] + \
+        [bf16_to_numpy(opt.gather_param_bf16()).tobytes()]
+
+
+# ---------------------------------------------------------------------------
+# config "tiny": 1 Mi parameters, 4 buckets, clip every step, +inf on step 7
+# ---------------------------------------------------------------------------
+
+def test_tiny_ten_steps_lockstep():
+    rep, opt = run_lockstep(W.tiny(), steps=10)
+    assert rep.decisions == [R] * 6 + [S] + [R] * 3
+    assert opt.step_count == 9
+    c = opt.counters()
+    assert (c.commits, c.skips, c.clip_resteps) == (0, 1, 9)
+    # the moments follow the oracle's evaluation order: expected bit-identical
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+    assert rep.n_diff["p"] <= 1e-5 * rep.n_elems
+
+
+def test_tiny_ragged_tensors_and_odd_bucket_size():
+    """Odd tensor sizes, a bucket size that is not a multiple of the vector
+    width (slot stride != bucket size, partial quads and a partial tile)."""
+    rep, opt = run_lockstep(W.tiny_ragged(), steps=8)
+    assert rep.decisions[6] == S and set(rep.decisions) == {R, S}
+    assert opt.info.slot_stride_elems != opt.info.bucket_elems
+
+
+def test_tiny_without_clipping_commits():
+    w = W.tiny()
+    w.max_grad_norm = 0.0
+    w.faults = ()
+    rep, opt = run_lockstep(w, steps=4)
+    assert rep.decisions == [C] * 4
+    assert opt.counters().elems_checked == 0          # sums came from the fused step
+
+
+def test_tiny_fp32_gradients():
+    w = W.tiny()
+    w.grad_dtype = "fp32"
+    rep, _ = run_lockstep(w, steps=8)
+    assert rep.decisions[6] == S
+
+
+@pytest.mark.parametrize("n,bucket", [(1, 64), (3, 1), (5, 7), (1023, 1024), (1025, 1024),
+                                      (4096, 1024), (130_001, 2048), (70_000, 70_000)])
+def test_small_and_degenerate_sizes(n, bucket):
+    w = W.Workload(name="small", numel=[n], bucket_elems=bucket, sigma_g=1e-2, steps=3)
+    rep, _ = run_lockstep(w, steps=3)
+    assert len(rep.decisions) == 3
+
+
+def test_empty_model_on_the_device():
+    opt = BucketedAdamW([], 1024)
+    hp = oracle.HParams()
+    res = opt.iteration(hp, stream=torch.cuda.current_stream())
+    assert res.decision == C and res.stats.norm == 0.0 and opt.step_count == 1
+
+
+# ---------------------------------------------------------------------------
+# exactness of speculation (Section 4.4) and of the rollback
+# ---------------------------------------------------------------------------
+
+def _run_device_only(w, steps, undo_slots, speculative, bucket_order=None):
+    hp = hparams_of(w)
+    stream = torch.cuda.current_stream()
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, undo_slots)
+    opt.load_state(W.initial_master(w, device="cuda"))
+    opt.cast_params(stream=stream)
+    trace = []
+    for step in range(1, steps + 1):
+        opt.load_grads(W.gradients(w, step, device="cuda"))
+        if speculative and bucket_order is not None:
+            for b in bucket_order:
+                try:
+                    opt.step_speculative(hp, b, stream)
+                except B.SuperOffloadError as e:
+                    assert e.status == B.SO_ERR_UNDO_EXHAUSTED
+            res = opt.validate(hp, stream)
+        else:
+            res = opt.iteration(hp, stream=stream, speculative=speculative)
+        trace.append((res.decision, res.stats.sumsq, res.stats.norm, res.stats.clip_coef,
+                      res.stats.nonfinite, res.step_after))
+    torch.cuda.synchronize()
+    return trace, _state_bytes(opt)
+
+
+@pytest.mark.parametrize("name", ["tiny", "tiny_ragged"])
+def test_speculative_flow_is_bitwise_the_check_first_flow(name):
+    """STV must reach exactly the result of synchronise-then-execute: state,
+    bf16 copy, norm, coefficient and decisions, bit for bit -- whatever subset
+    of buckets was speculated and in whatever order."""
+    w = W.by_name(name)
+    ref = _run_device_only(w, 9, undo_slots=0, speculative=False)
+    full = _run_device_only(w, 9, undo_slots=B.SO_ALL, speculative=True)
+    windowed = _run_device_only(w, 9, undo_slots=2, speculative=True)
+    shuffled = _run_device_only(w, 9, undo_slots=3, speculative=True,
+                                bucket_order=[3, 0, 2, 1] if name == "tiny" else [4, 1, 0, 3, 2])
+    assert ref[0] == full[0] == windowed[0] == shuffled[0]
+    assert ref[1] == full[1] == windowed[1] == shuffled[1]
+
+
+def test_repeat_runs_are_bitwise_identical():
+    a = _run_device_only(W.tiny(), 5, B.SO_ALL, True)
+    b = _run_device_only(W.tiny(), 5, B.SO_ALL, True)
+    assert a == b
+
+
+def test_elementwise_result_does_not_depend_on_bucket_size():
+    outs = []
+    for bucket in (262_144, 100_000, 1 << 20, 4096):
+        w = W.tiny()
+        w.bucket_elems, w.max_grad_norm, w.faults = bucket, 0.0, ()
+        outs.append(_run_device_only(w, 3, B.SO_ALL, True)[1])
+    assert all(o == outs[0] for o in outs)
+
+
+@pytest.mark.parametrize("kind", ["inf", "-inf", "nan"])
+@pytest.mark.parametrize("where", ["first", "last", "middle"])
+def test_rollback_restores_the_prior_state_bit_for_bit(kind, where):
+    w = W.tiny_ragged()
+    w.faults = ()
+    hp = hparams_of(w)
+    stream = torch.cuda.current_stream()
+    opt = BucketedAdamW(w.numel, w.bucket_elems, guard_bands=True)
+    opt.load_state(W.initial_master(w, device="cuda"))
+    opt.cast_params(stream=stream)
+    opt.load_grads(W.gradients(w, 1, device="cuda"))
+    assert opt.iteration(hp, stream=stream).decision == R       # some non-trivial m, v
+    before = _state_bytes(opt)
+    slots = [B.so_bucket_slot(opt.ctx, b) for b in range(opt.n_buckets)]
+    g = W.gradients(w, 2, device="cuda")
+    idx = {"first": 0, "last": w.total - 1, "middle": w.total // 2 + 1}[where]
+    g[idx] = {"inf": float("inf"), "-inf": float("-inf"), "nan": float("nan")}[kind]
+    opt.load_grads(g)
+    opt.step_speculative(hp, B.SO_ALL, stream)
+    torch.cuda.synchronize()
+    during = bf16_to_numpy(opt.gather_param_bf16()).tobytes()
+    assert during != before[3]                                  # the speculative copy is live
+    res = opt.validate(hp, stream)
+    torch.cuda.synchronize()
+    assert res.decision == S and res.stats.nonfinite == 1 and res.step_after == 1
+    assert _state_bytes(opt) == before
+    assert [B.so_bucket_slot(opt.ctx, b) for b in range(opt.n_buckets)] == slots
+    assert opt.guard_bands_intact()
+
+
+# ---------------------------------------------------------------------------
+# the gradient check alone
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_grad_check_against_the_oracle_norm(dtype):
+    n, bucket = 3_000_017, 500_000
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    z = torch.randn(n, generator=gen, device="cuda")
+    # wide dynamic range, including magnitudes whose square leaves fp32
+    expo = torch.randint(-40, 41, (n,), generator=gen, device="cuda").float()
+    g = z * torch.pow(torch.tensor(2.0, device="cuda"), expo)
+    g[17] = 3.0e38
+    g[n - 1] = 1.0e-40
+    g = g.to(torch.bfloat16 if dtype == "bf16" else torch.float32)
+    opt = BucketedAdamW([n], bucket, grad_dtype=dtype, undo_slots=0)
+    opt.load_grads(g)
+    hp = oracle.HParams(max_grad_norm=1.0)
+    stats = opt.grad_check(hp, stream=torch.cuda.current_stream())
+    s, nrm, flag = oracle.global_grad_check(grads_to_numpy(g), bucket)
+    assert flag == 0 and stats.nonfinite == 0                   # finite in, finite out
+    assert stats.sumsq == pytest.approx(s, rel=1e-12)
+    assert stats.norm == pytest.approx(nrm, rel=1e-12)
+    assert stats.clip_coef == pytest.approx(oracle.clip_coef(nrm, 1.0), rel=1e-12)
+    opt.validate(hp, torch.cuda.current_stream())
+
+
+def test_nonfinite_flag_for_every_special_bf16_pattern_and_position():
+    n, bucket = 5000, 1024
+    specials = [0x7F80, 0xFF80, 0x7F81, 0x7FC0, 0xFFFF, 0x7FFF]
+    finite_extremes = [0x7F7F, 0xFF7F, 0x0001, 0x8001, 0x0000, 0x8000]
+    hp = oracle.HParams()
+    opt = BucketedAdamW([n], bucket, undo_slots=0)
+    base = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    for pos in (0, 1023, 1024, 4095, 4096, 4999):
+        for pat, want in [(p, 1) for p in specials] + [(p, 0) for p in finite_extremes]:
+            g = base.clone()
+            g.view(torch.int16)[pos] = np.array(pat, dtype=np.uint16).view(np.int16).item()
+            opt.load_grads(g)
+            stats = opt.grad_check(hp, stream=torch.cuda.current_stream())
+            assert stats.nonfinite == want, (hex(pat), pos)
+            _, flag = oracle.grad_check_range(grads_to_numpy(g), 0, n)
+            assert flag == want
+            res = opt.validate(hp, torch.cuda.current_stream())
+            assert res.decision == (S if want else C)
+
+
+# ---------------------------------------------------------------------------
+# the cast alone: every fp32 bit pattern
+# ---------------------------------------------------------------------------
+
+def test_cast_is_rne_for_all_2_to_32_patterns():
+    chunk = 1 << 26
+    opt = BucketedAdamW([chunk], 1 << 24, undo_slots=0)
+    stream = torch.cuda.current_stream()
+    for c in range((1 << 32) // chunk):
+        pats = torch.arange(c * chunk, (c + 1) * chunk, dtype=torch.int64, device="cuda")
+        bits = pats.to(torch.int32) if c < 32 else (pats - (1 << 32)).to(torch.int32)
+        opt.master[:chunk].copy_(bits.view(torch.float32))
+        opt.cast_params(stream=stream)
+        got = opt.param_bf16[:chunk].view(torch.int16)
+        host_in = bits.view(torch.float32).cpu().numpy()
+        want = oracle.bf16_rne(host_in)
+        want_t = torch.from_numpy(want.view(np.int16)).cuda()
+        nan = torch.from_numpy(np.isnan(host_in)).cuda()
+        assert torch.equal(got[~nan], want_t[~nan]), f"chunk {c}"
+        if nan.any():
+            got_nan = got[nan].cpu().numpy().view(np.uint16)
+            assert is_bf16_nan(got_nan).all(), f"chunk {c}: NaN lost"
+
+
+# ---------------------------------------------------------------------------
+# GPT-2-small-shaped list: 124M parameters in 25M-element buckets
+# ---------------------------------------------------------------------------
+
+def test_gpt2_small_commit_path_lockstep():
+    rep, opt = run_lockstep(W.gpt2_small(clip=False), steps=4, guard_bands=False)
+    assert rep.decisions == [C] * 4
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+    assert rep.max_norm_rel < 1e-12
+
+
+def test_gpt2_small_clip_path_lockstep():
+    rep, opt = run_lockstep(W.gpt2_small(clip=True), steps=3, guard_bands=False)
+    assert rep.decisions == [R] * 3
+    assert rep.max_ulp["p"] <= 2
