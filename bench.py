@@ -1,0 +1,344 @@
+#!/usr/bin/env python
+"""Benchmark of the bucketized speculative AdamW step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A "step" is one pass of the whole hot path over one synthetic gradient batch:
+speculative fused AdamW+cast step of every bucket, the global gradient check
+(finalised from the tile sums the step left behind), and the validation
+decision with whatever it entails (a commit on this workload).  Prints one JSON
+line: optimizer params/s over all GPUs (`value`, inputs resident in HBM), the
+same through the host-buffer entry point (`e2e`), the HBM roofline of the
+fused step kernel, and the CPU oracle timed on a bounded sample.
+
+With N > 1 (launched by torchrun) every rank runs an independent replica of
+the workload on its own GPU -- the path has no exchange step on one node --
+and the value is N x params / max-over-ranks time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "optimizer_params_per_sec"
+UNIT = "params/s"
+BYTES_PER_PARAM = {"bf16": 28, "fp32": 30}      # algorithmic HBM bytes of the fused step
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per parameter of the fused step
+# kernel, from the ncu capture summarised under profiles/ (None until measured)
+NCU_TRAFFIC_BYTES_PER_PARAM = None
+
+
+def _measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while timing."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) == 6:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        if self.thread:
+            self.thread.join(timeout=2)
+        sm, mx, reasons = [], None, set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+            except ValueError:
+                continue
+            for name, val in zip(names, r[2:]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        med = sm[len(sm) // 2] if sm else None
+        return {"sm_mhz": med, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _hparams(w, oracle_mod=None):
+    from paper_2509_21271_b200.binding import so_hparams
+    return so_hparams(w.lr, w.beta1, w.beta2, w.eps, w.weight_decay, w.max_grad_norm)
+
+
+def _oracle_sample(w, steps, warmup):
+    """The CPU oracle, as it stands, on the first bucket of the workload."""
+    import numpy as np
+    import torch
+
+    import oracle
+    from paper_2509_21271_b200 import workloads as W
+
+    n = min(w.bucket_elems, w.total)
+    sample = W.Workload(name=w.name + "_sample", numel=[n], bucket_elems=n, sigma_g=w.sigma_g,
+                        seed=w.seed, max_grad_norm=w.max_grad_norm, grad_dtype=w.grad_dtype)
+    hp = oracle.HParams(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
+                        weight_decay=w.weight_decay, max_grad_norm=w.max_grad_norm)
+    p = W.initial_master(sample).numpy()
+    m, v = np.zeros_like(p), np.zeros_like(p)
+    pb = oracle.bf16_rne(p)
+    g = W.gradients(sample, 1)
+    g = g.view(torch.int16).numpy().view(np.uint16) if g.dtype == torch.bfloat16 else g.numpy()
+    t = 0
+    for _ in range(warmup):
+        t = oracle.iteration_ste(p, m, v, pb, g, n, t, hp).step_after
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        t = oracle.iteration_ste(p, m, v, pb, g, n, t, hp).step_after
+    dt = time.perf_counter() - t0
+    return {"value": n * steps / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"first bucket ({n} params) of {w.name}, {steps} steps of check+AdamW+cast, "
+                      f"single thread, {dt:.1f} s"}, dt / steps, n
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    base, per_step, n = _oracle_sample(w, args.steps, max(args.warmup, 1))
+    line = {"impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "sample_params": n, "bucket_elems": w.bucket_elems},
+            "cpu_baseline": base,
+            "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="gpt2_small")
+    ap.add_argument("--undo-slots", type=int, default=-1)
+    ap.add_argument("--per-bucket", action="store_true",
+                    help="one speculative-step call per bucket instead of one batched call")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--step-variant", type=int, default=0,
+                    help="0: bulk-copy pipeline (default), 1: register-only step kernel")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+
+    from paper_2509_21271_b200 import workloads as W
+    w = W.by_name(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+
+    from paper_2509_21271_b200 import binding as B
+    from paper_2509_21271_b200 import build as so_build
+    from paper_2509_21271_b200.optimizer import BucketedAdamW
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        so_build.build_library()
+    if dist is not None:
+        dist.barrier()
+
+    hp = _hparams(w)
+    stream = torch.cuda.current_stream()
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, args.undo_slots,
+                        step_variant=args.step_variant)
+    opt.load_state(W.initial_master(w, device="cuda"))
+    opt.cast_params(stream=stream)
+    g = W.gradients(w, 1, device="cuda")
+    opt.load_grads(g)
+    torch.cuda.synchronize()
+    N = w.total
+    nb = opt.n_buckets
+
+    def one_step(ev=None):
+        if args.per_bucket:
+            for b in range(nb):
+                try:
+                    B.so_adam_step_speculative(opt.ctx, hp, b, stream)
+                except B.SuperOffloadError as e:
+                    if e.status != B.SO_ERR_UNDO_EXHAUSTED:
+                        raise
+        else:
+            if ev is not None:
+                ev[0].record(stream)
+            B.so_adam_step_speculative(opt.ctx, hp, B.SO_ALL, stream)
+            if ev is not None:
+                ev[1].record(stream)
+        return B.so_validate_commit_or_rollback(opt.ctx, hp, stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident timing ------------------------------------------
+    for _ in range(args.warmup):
+        one_step()
+    kernel_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                     for _ in range(args.steps)]
+    launches0 = opt.counters().kernel_launches
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    decisions = set()
+    t_start.record(stream)
+    for k in range(args.steps):
+        decisions.add(one_step(kernel_events[k]).decision)
+    t_end.record(stream)
+    barrier()
+    elapsed_ms = t_start.elapsed_time(t_end)
+    launches = opt.counters().kernel_launches - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    spec_buckets = min(nb, opt.info.undo_slots)
+    spec_params = sum(opt.bucket_range(b)[1] - opt.bucket_range(b)[0] for b in range(spec_buckets))
+    kernel_ms = None
+    if not args.per_bucket:
+        times = [a.elapsed_time(b) for a, b in kernel_events]
+        kernel_ms = sum(times) / len(times)
+
+    # ---- end to end through the host-buffer entry point -------------------
+    e2e = None
+    if not args.no_e2e:
+        gsz = 2 if w.grad_dtype == "bf16" else 4
+        host_g = torch.empty(N, dtype=opt.grad_torch_dtype, pin_memory=True)
+        host_g.copy_(g)
+        host_p = torch.empty(N, dtype=torch.bfloat16, pin_memory=True)
+        for _ in range(3):
+            B.so_iteration_host(opt.ctx, hp, host_g.data_ptr(), host_p.data_ptr(), stream)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_e2e = max(3, min(args.steps, 10))
+        e0.record(stream)
+        for _ in range(n_e2e):
+            B.so_iteration_host(opt.ctx, hp, host_g.data_ptr(), host_p.data_ptr(), stream)
+        e1.record(stream)
+        barrier()
+        e2e_ms = e0.elapsed_time(e1) / n_e2e
+        e2e = {"ms": e2e_ms, "h2d": N * gsz, "d2h": N * 2 + 40}
+
+    # ---- max over ranks ----------------------------------------------------
+    if dist is not None:
+        vals = torch.tensor([elapsed_ms, e2e["ms"] if e2e else 0.0], device="cuda",
+                            dtype=torch.float64)
+        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(vals[0])
+        if e2e:
+            e2e["ms"] = float(vals[1])
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    ms_per_step = elapsed_ms / args.steps
+    value = world * N / (ms_per_step * 1e-3)
+    peak, peak_kind = _measured_peak()
+    bpp = BYTES_PER_PARAM[w.grad_dtype]
+    roofline = None
+    if kernel_ms:
+        achieved = bpp * spec_params / (kernel_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "adamw_step_kernel (fused speculative step+cast)",
+                    "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}",
+                    "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": (NCU_TRAFFIC_BYTES_PER_PARAM * spec_params
+                                if NCU_TRAFFIC_BYTES_PER_PARAM else None),
+                    "bytes_per_param": bpp, "params_per_launch": spec_params,
+                    "kernel_ms": kernel_ms}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "params": N, "tensors": len(w.numel),
+                   "bucket_elems": w.bucket_elems, "n_buckets": nb,
+                   "undo_slots": opt.info.undo_slots, "grad_dtype": w.grad_dtype,
+                   "max_grad_norm": w.max_grad_norm,
+                   "decisions": sorted(B.DECISION_NAMES[d] for d in decisions),
+                   "launch_mode": "per_bucket" if args.per_bucket else "batched",
+                   "step_kernel": "bulk_copy_pipeline" if args.step_variant == 0 else "registers",
+                   "parallelism": "replicas" if world > 1 else "single",
+                   "l2": f"working set {16 * N / 1e6:.0f} MB resident + undo slots, "
+                         "larger than the 126 MB L2; no flush"},
+        "hbm_gbs_whole_step": world * bpp * N / (ms_per_step * 1e-3) / 1e9,
+        "gpu_launches": launches,
+        "clocks": clocks,
+    }
+    if roofline:
+        line["roofline"] = roofline
+    if e2e:
+        line["e2e"] = {"value": world * N / (e2e["ms"] * 1e-3), "unit": UNIT,
+                       "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                       "ms_per_step": e2e["ms"]}
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = _oracle_sample(w, 20, 1)[0]
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -57,7 +57,8 @@ enum {
     SO_ERR_CUDA = -3,                  /* a CUDA call failed; see so_last_cuda_error */
     SO_ERR_UNDO_EXHAUSTED = -4,        /* no free slot for another speculative step  */
     SO_ERR_NOMEM = -5,                 /* host allocation failed                     */
-    SO_ERR_UNSUPPORTED = -6
+    SO_ERR_UNSUPPORTED = -6,
+    SO_ERR_TIMEOUT = -7                /* a kernel's bounded wait on its own copies ran out */
 };
 
 enum { SO_GRAD_BF16 = 0, SO_GRAD_FP32 = 1 };
@@ -209,6 +210,25 @@ so_status so_validate_commit_or_rollback(so_ctx *ctx, const so_hparams *hp, void
  */
 so_status so_cast_params(so_ctx *ctx, int32_t bucket, void *stream);
 
+/*
+ * so_iteration_host -- one whole iteration fed from and drained to HOST memory,
+ * pipelined per bucket the way Section 4.3 overlaps bucket transfers with
+ * compute: the gradient bucket b is copied host -> device while bucket b-1 is
+ * being stepped speculatively and the bf16 parameters of bucket b-2 travel
+ * device -> host (Section 4.5: only low-precision data crosses the link, the
+ * casts run on the GPU).  Then validation as in
+ * so_validate_commit_or_rollback; after a SKIP or CLIP_RESTEP the bf16
+ * parameters are sent again.
+ *   host_grad        flat gradient of N elements in grad_dtype, parameter order
+ *                    (pinned host memory for asynchronous copies)
+ *   host_param_bf16  flat bf16 output of N elements, or NULL for none
+ * Buckets beyond the undo capacity are scanned instead of stepped and receive
+ * their step inside validation.  Uses two internal copy streams created on
+ * first use.  Returns after all copies have completed (synchronises).
+ */
+so_status so_iteration_host(so_ctx *ctx, const so_hparams *hp, const void *host_grad,
+                            void *host_param_bf16, void *stream, so_step_result *out);
+
 /* Slot of the state arenas that holds bucket b's committed master/m/v. */
 so_status so_bucket_slot(const so_ctx *ctx, int32_t bucket, int32_t *slot);
 
@@ -239,6 +259,11 @@ void so_destroy(so_ctx *ctx);
 so_status so_debug_set_dry_run(so_ctx *ctx, int32_t on);
 so_status so_debug_set_bucket_stats(so_ctx *ctx, int32_t bucket, double sumsq,
                                     int32_t nonfinite);
+
+/* Which implementation of the fused step runs: 0 (default) stages bulk copies
+ * through shared memory, 1 keeps everything in registers.  Both produce the
+ * same bits; the switch exists for measurements and for testing both. */
+so_status so_debug_set_step_variant(so_ctx *ctx, int32_t variant);
 
 #ifdef __cplusplus
 }

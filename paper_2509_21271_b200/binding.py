@@ -15,6 +15,7 @@ from .build import LIB_PATH
 SO_OK = 0
 SO_ERR_INVALID_ARG, SO_ERR_STATE, SO_ERR_CUDA = -1, -2, -3
 SO_ERR_UNDO_EXHAUSTED, SO_ERR_NOMEM, SO_ERR_UNSUPPORTED = -4, -5, -6
+SO_ERR_TIMEOUT = -7
 SO_GRAD_BF16, SO_GRAD_FP32 = 0, 1
 SO_DECISION_COMMIT, SO_DECISION_SKIP, SO_DECISION_CLIP_RESTEP = 0, 1, 2
 SO_ALL = -1
@@ -69,9 +70,10 @@ _lib = None
 
 EXPORTS = ["so_layout_init", "so_layout_get_info", "so_layout_tensor", "so_layout_bind",
            "so_grad_check", "so_adam_step_speculative", "so_validate_commit_or_rollback",
-           "so_cast_params", "so_bucket_slot", "so_get_step", "so_set_step",
+           "so_cast_params", "so_iteration_host", "so_bucket_slot", "so_get_step", "so_set_step",
            "so_pending_buckets", "so_get_counters", "so_last_cuda_error", "so_strerror",
-           "so_destroy", "so_debug_set_dry_run", "so_debug_set_bucket_stats"]
+           "so_destroy", "so_debug_set_dry_run", "so_debug_set_bucket_stats",
+           "so_debug_set_step_variant"]
 
 
 def lib() -> C.CDLL:
@@ -95,6 +97,7 @@ def lib() -> C.CDLL:
         "so_adam_step_speculative": [vp, P(so_hparams), i32, vp],
         "so_validate_commit_or_rollback": [vp, P(so_hparams), vp, P(so_step_result)],
         "so_cast_params": [vp, i32, vp],
+        "so_iteration_host": [vp, P(so_hparams), vp, vp, vp, P(so_step_result)],
         "so_bucket_slot": [vp, i32, P(i32)],
         "so_get_step": [vp, P(i64)],
         "so_set_step": [vp, i64],
@@ -102,6 +105,7 @@ def lib() -> C.CDLL:
         "so_get_counters": [vp, P(so_counters)],
         "so_debug_set_dry_run": [vp, i32],
         "so_debug_set_bucket_stats": [vp, i32, dbl, i32],
+        "so_debug_set_step_variant": [vp, i32],
     }
     for name, argtypes in sig.items():
         fn = getattr(L, name)
@@ -208,6 +212,15 @@ def so_cast_params(ctx, bucket: int = SO_ALL, stream=None) -> None:
     _ok(ctx, lib().so_cast_params(ctx, bucket, _stream(stream)), "so_cast_params")
 
 
+def so_iteration_host(ctx, hp, host_grad: int, host_param_bf16: int, stream=None) -> so_step_result:
+    """Host addresses (pinned memory); ``host_param_bf16`` may be 0 for no output."""
+    h = _hp(hp)
+    out = so_step_result()
+    _ok(ctx, lib().so_iteration_host(ctx, C.byref(h), host_grad, host_param_bf16 or None,
+                                     _stream(stream), C.byref(out)), "so_iteration_host")
+    return out
+
+
 def so_bucket_slot(ctx, bucket: int) -> int:
     s = C.c_int32()
     _ok(ctx, lib().so_bucket_slot(ctx, bucket, C.byref(s)), "so_bucket_slot")
@@ -247,3 +260,7 @@ def so_debug_set_dry_run(ctx, on: bool) -> None:
 def so_debug_set_bucket_stats(ctx, bucket: int, sumsq: float, nonfinite: int) -> None:
     _ok(ctx, lib().so_debug_set_bucket_stats(ctx, bucket, sumsq, nonfinite),
         "so_debug_set_bucket_stats")
+
+
+def so_debug_set_step_variant(ctx, variant: int) -> None:
+    _ok(ctx, lib().so_debug_set_step_variant(ctx, variant), "so_debug_set_step_variant")

@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "so_kernels.cuh"
+#include "so_step_tma.cuh"
 
 using namespace so;
 
@@ -32,7 +33,10 @@ struct so_ctx {
     void *grad = nullptr;
     uint16_t *param_bf16 = nullptr;
     double *d_partials = nullptr;
-    BucketStats *d_stats = nullptr;
+    BucketStats *d_stats = nullptr;     // n_buckets results, then one record whose first
+                                        // word is the device status (0 = fine)
+    int32_t *d_status = nullptr;
+    int step_variant = 0;               // 0: bulk-copy pipeline, 1: register path
     BucketStats *h_stats = nullptr;
     bool h_stats_pinned = false;
     int occ_step = 0, occ_check = 0, occ_cast = 0;
@@ -53,6 +57,9 @@ struct so_ctx {
     int32_t last_cuda_error = 0;
     bool dry_run = false;
     std::vector<BucketStats> injected;
+    // ---- host-fed iteration: copy streams and ordering events (lazy) ----
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    std::vector<cudaEvent_t> events;
 };
 
 namespace {
@@ -87,7 +94,7 @@ bool hparams_ok(const so_hparams *hp)
     for (double x : vals)
         if (!std::isfinite(x)) return false;
     return hp->lr >= 0.0 && hp->beta1 >= 0.0 && hp->beta1 < 1.0 && hp->beta2 >= 0.0 &&
-           hp->beta2 < 1.0 && hp->eps >= 0.0 && hp->weight_decay >= 0.0;
+           hp->beta2 < 1.0 && hp->eps >= 2.3e-308 && hp->weight_decay >= 0.0;
 }
 
 bool hparams_equal(const so_hparams &a, const so_hparams &b)
@@ -140,6 +147,69 @@ so_status after_launch(so_ctx *c)
 
 // ---- launches --------------------------------------------------------------
 
+// Shapes of the bulk-copy pipeline (rows per chunk, warps per block, input
+// stages, output stages).  Variant 0 is the default.
+using ShapeDefault = PipeShape<2, 12, 3, 1>;
+using ShapeA = PipeShape<2, 8, 4, 2>;
+using ShapeB = PipeShape<1, 16, 4, 2>;
+using ShapeC = PipeShape<1, 24, 3, 2>;
+using ShapeD = PipeShape<1, 32, 3, 1>;
+using ShapeE = PipeShape<2, 16, 2, 1>;
+
+template <typename S>
+void launch_tma(so_ctx *c, const StepArgs &a, int n, bool speculative, cudaStream_t stream)
+{
+    int64_t blocks = ((int64_t)n * a.geo.tiles_per_slot + S::kWarps - 1) / S::kWarps;
+    if (blocks > c->num_sms) blocks = c->num_sms;
+    const unsigned grid = (unsigned)(blocks < 1 ? 1 : blocks);
+    if (c->grad_dtype == SO_GRAD_BF16) {
+        const size_t sm = TmaLayout<uint16_t, S>::kSmemBytes;
+        if (speculative)
+            adamw_step_tma_kernel<uint16_t, true, S><<<grid, S::kThreads, sm, stream>>>(a, c->d_status);
+        else
+            adamw_step_tma_kernel<uint16_t, false, S><<<grid, S::kThreads, sm, stream>>>(a, c->d_status);
+    } else {
+        const size_t sm = TmaLayout<float, S>::kSmemBytes;
+        if (speculative)
+            adamw_step_tma_kernel<float, true, S><<<grid, S::kThreads, sm, stream>>>(a, c->d_status);
+        else
+            adamw_step_tma_kernel<float, false, S><<<grid, S::kThreads, sm, stream>>>(a, c->d_status);
+    }
+}
+
+void launch_tma_variant(so_ctx *c, const StepArgs &a, int n, bool speculative, cudaStream_t stream)
+{
+    switch (c->step_variant) {
+        case 10: launch_tma<ShapeA>(c, a, n, speculative, stream); break;
+        case 11: launch_tma<ShapeB>(c, a, n, speculative, stream); break;
+        case 12: launch_tma<ShapeC>(c, a, n, speculative, stream); break;
+        case 13: launch_tma<ShapeD>(c, a, n, speculative, stream); break;
+        case 14: launch_tma<ShapeE>(c, a, n, speculative, stream); break;
+        default: launch_tma<ShapeDefault>(c, a, n, speculative, stream); break;
+    }
+}
+
+// The bulk-copy kernels stage through more than 48 KB of shared memory.
+template <typename S>
+cudaError_t allow_smem()
+{
+    const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    cudaError_t e = cudaFuncSetAttribute(adamw_step_tma_kernel<uint16_t, true, S>, attr,
+                                         TmaLayout<uint16_t, S>::kSmemBytes);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(adamw_step_tma_kernel<uint16_t, false, S>, attr,
+                                 TmaLayout<uint16_t, S>::kSmemBytes);
+    if constexpr (TmaLayout<float, S>::kSmemBytes <= 227 * 1024) {
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(adamw_step_tma_kernel<float, true, S>, attr,
+                                     TmaLayout<float, S>::kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(adamw_step_tma_kernel<float, false, S>, attr,
+                                     TmaLayout<float, S>::kSmemBytes);
+    }
+    return e;
+}
+
 // Step the listed buckets (src slot -> dst slot).  speculative: scale 1 and
 // tile sums written; otherwise the given scale and no sums.
 so_status launch_steps(so_ctx *c, const std::vector<BucketEntry> &entries, const so_hparams &hp,
@@ -164,12 +234,15 @@ so_status launch_steps(so_ctx *c, const std::vector<BucketEntry> &entries, const
         }
         for (int i = n; i < kMaxBatch; ++i) a.e[i] = BucketEntry{0, 0, 0};
         if (!c->dry_run) {
-            const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_step);
             const bool bf16 = c->grad_dtype == SO_GRAD_BF16;
-            if (speculative) {
+            if (c->step_variant != 1) {
+                launch_tma_variant(c, a, n, speculative, stream);
+            } else if (speculative) {
+                const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_step);
                 if (bf16) adamw_step_kernel<uint16_t, true, 4><<<grid, kThreads, 0, stream>>>(a);
                 else adamw_step_kernel<float, true, 4><<<grid, kThreads, 0, stream>>>(a);
             } else {
+                const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_step);
                 if (bf16) adamw_step_kernel<uint16_t, false, 4><<<grid, kThreads, 0, stream>>>(a);
                 else adamw_step_kernel<float, false, 4><<<grid, kThreads, 0, stream>>>(a);
             }
@@ -256,11 +329,16 @@ so_status finalize_check(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
         if (s != SO_OK) return s;
         if (!c->dry_run) {
             cudaError_t e = cudaMemcpyAsync(c->h_stats, c->d_stats,
-                                            sizeof(BucketStats) * (size_t)c->n_buckets,
+                                            sizeof(BucketStats) * (size_t)(c->n_buckets + 1),
                                             cudaMemcpyDeviceToHost, stream);
             if (e != cudaSuccess) return cuda_fail(c, e);
             e = cudaStreamSynchronize(stream);
             if (e != cudaSuccess) return cuda_fail(c, e);
+            if (c->h_stats[c->n_buckets].nonfinite != 0 || c->h_stats[c->n_buckets].pad != 0) {
+                // a kernel gave up waiting for one of its own copies
+                cudaMemsetAsync(c->d_status, 0, sizeof(BucketStats), stream);
+                return SO_ERR_TIMEOUT;
+            }
         } else {
             for (int32_t b = 0; b < c->n_buckets; ++b) c->h_stats[b] = c->injected[b];
         }
@@ -376,7 +454,7 @@ so_status so_layout_get_info(const so_ctx *c, so_layout_info *info)
                        (c->grad_dtype == SO_GRAD_BF16 ? 2u : 4u);
     info->bytes_param_bf16 = (uint64_t)c->n_buckets * (uint64_t)c->stride * 2u;
     const uint64_t partial_bytes = (uint64_t)c->n_buckets * (uint64_t)c->tiles_per_slot * 8u;
-    const uint64_t stats_bytes = (uint64_t)c->n_buckets * sizeof(BucketStats);
+    const uint64_t stats_bytes = (uint64_t)(c->n_buckets + 1) * sizeof(BucketStats);
     info->bytes_scratch = (partial_bytes + 255u) / 256u * 256u + stats_bytes + 256u;
     return SO_OK;
 }
@@ -423,12 +501,19 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_cast, cast_params_kernel,
                                                           kThreads, 0);
         if (e != cudaSuccess) return cuda_fail(c, e);
+        e = allow_smem<ShapeDefault>();
+        if (e == cudaSuccess) e = allow_smem<ShapeA>();
+        if (e == cudaSuccess) e = allow_smem<ShapeB>();
+        if (e == cudaSuccess) e = allow_smem<ShapeC>();
+        if (e == cudaSuccess) e = allow_smem<ShapeD>();
+        if (e == cudaSuccess) e = allow_smem<ShapeE>();
+        if (e != cudaSuccess) return cuda_fail(c, e);
     } else {
         c->num_sms = 148;
         c->occ_step = c->occ_check = c->occ_cast = 2;
     }
     if (!c->h_stats) {
-        const size_t bytes = sizeof(BucketStats) * (size_t)(c->n_buckets > 0 ? c->n_buckets : 1);
+        const size_t bytes = sizeof(BucketStats) * (size_t)(c->n_buckets + 1);
         if (!c->dry_run && cudaMallocHost(reinterpret_cast<void **>(&c->h_stats), bytes) ==
                                cudaSuccess) {
             c->h_stats_pinned = true;
@@ -447,6 +532,12 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
     const uint64_t partial_bytes = (uint64_t)c->n_buckets * (uint64_t)c->tiles_per_slot * 8u;
     c->d_stats = reinterpret_cast<BucketStats *>(static_cast<char *>(scratch) +
                                                  (partial_bytes + 255u) / 256u * 256u);
+    c->d_status = reinterpret_cast<int32_t *>(c->d_stats + c->n_buckets);
+    if (!c->dry_run) {
+        // the status record is the only part of scratch that must start at zero
+        const cudaError_t e = cudaMemset(c->d_status, 0, sizeof(BucketStats));
+        if (e != cudaSuccess) return cuda_fail(c, e);
+    }
     c->bound = true;
     return SO_OK;
 }
@@ -599,6 +690,92 @@ so_status so_cast_params(so_ctx *c, int32_t bucket, void *stream)
     return launch_casts(c, entries, static_cast<cudaStream_t>(stream));
 }
 
+so_status so_iteration_host(so_ctx *c, const so_hparams *hp, const void *host_grad,
+                            void *host_param_bf16, void *stream, so_step_result *out)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (!c->bound || c->phase != kIdle) return SO_ERR_STATE;
+    if (!hparams_ok(hp) || (c->n_buckets > 0 && !host_grad)) return SO_ERR_INVALID_ARG;
+    if (c->dry_run) return SO_ERR_UNSUPPORTED;
+    cudaStream_t main = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if (!c->copy_in) {
+        e = cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        e = cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+    }
+    while ((int32_t)c->events.size() < 2 * c->n_buckets + 1) {
+        cudaEvent_t ev;
+        e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        c->events.push_back(ev);
+    }
+    const size_t gsz = c->grad_dtype == SO_GRAD_BF16 ? 2 : 4;
+    const char *hg = static_cast<const char *>(host_grad);
+    char *hp_out = static_cast<char *>(host_param_bf16);
+    char *dgrad = static_cast<char *>(c->grad);
+    cudaEvent_t start = c->events[2 * c->n_buckets];
+
+    // the copy streams start after whatever the caller queued on `stream`
+    e = cudaEventRecord(start, main);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    cudaStreamWaitEvent(c->copy_in, start, 0);
+    cudaStreamWaitEvent(c->copy_out, start, 0);
+
+    for (int32_t b = 0; b < c->n_buckets; ++b) {
+        const size_t n = (size_t)elems_of(c, b);
+        e = cudaMemcpyAsync(dgrad + (size_t)b * (size_t)c->stride * gsz,
+                            hg + (size_t)b * (size_t)c->bucket_elems * gsz, n * gsz,
+                            cudaMemcpyHostToDevice, c->copy_in);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        cudaEventRecord(c->events[2 * b], c->copy_in);
+        cudaStreamWaitEvent(main, c->events[2 * b], 0);
+        so_status s;
+        bool speculated = false;
+        if (!c->free_slots.empty()) {
+            s = so_adam_step_speculative(c, hp, b, stream);
+            speculated = true;
+        } else {
+            s = so_grad_check(c, hp, b, stream, nullptr);
+        }
+        if (s != SO_OK) return s;
+        if (speculated && hp_out) {
+            cudaEventRecord(c->events[2 * b + 1], main);
+            cudaStreamWaitEvent(c->copy_out, c->events[2 * b + 1], 0);
+            e = cudaMemcpyAsync(hp_out + (size_t)b * (size_t)c->bucket_elems * 2,
+                                c->param_bf16 + (size_t)b * (size_t)c->stride, n * 2,
+                                cudaMemcpyDeviceToHost, c->copy_out);
+            if (e != cudaSuccess) return cuda_fail(c, e);
+        }
+    }
+    std::vector<uint8_t> was_speculated(c->cover.begin(), c->cover.end());
+    so_step_result res;
+    so_status s = so_validate_commit_or_rollback(c, hp, stream, &res);
+    if (s != SO_OK) return s;
+    if (hp_out) {
+        // whatever validation (re)wrote after the speculative copies went out
+        cudaEventRecord(start, main);
+        cudaStreamWaitEvent(c->copy_out, start, 0);
+        for (int32_t b = 0; b < c->n_buckets; ++b) {
+            const bool sent = was_speculated[b] == kSpeculated;
+            if (sent && res.decision == SO_DECISION_COMMIT) continue;
+            if (!sent && res.decision == SO_DECISION_SKIP) continue;   // never changed
+            const size_t n = (size_t)elems_of(c, b);
+            e = cudaMemcpyAsync(hp_out + (size_t)b * (size_t)c->bucket_elems * 2,
+                                c->param_bf16 + (size_t)b * (size_t)c->stride, n * 2,
+                                cudaMemcpyDeviceToHost, c->copy_out);
+            if (e != cudaSuccess) return cuda_fail(c, e);
+        }
+    }
+    e = cudaStreamSynchronize(c->copy_out);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    e = cudaStreamSynchronize(main);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    if (out) *out = res;
+    return SO_OK;
+}
+
 so_status so_bucket_slot(const so_ctx *c, int32_t bucket, int32_t *slot)
 {
     if (!c || !slot || bucket < 0 || bucket >= c->n_buckets) return SO_ERR_INVALID_ARG;
@@ -647,6 +824,7 @@ const char *so_strerror(so_status s)
         case SO_ERR_UNDO_EXHAUSTED: return "no free slot for another speculative step";
         case SO_ERR_NOMEM: return "host allocation failed";
         case SO_ERR_UNSUPPORTED: return "unsupported";
+        case SO_ERR_TIMEOUT: return "a kernel gave up waiting for one of its own copies";
         default: return "unknown status";
     }
 }
@@ -654,6 +832,9 @@ const char *so_strerror(so_status s)
 void so_destroy(so_ctx *c)
 {
     if (!c) return;
+    for (cudaEvent_t ev : c->events) cudaEventDestroy(ev);
+    if (c->copy_in) cudaStreamDestroy(c->copy_in);
+    if (c->copy_out) cudaStreamDestroy(c->copy_out);
     if (c->h_stats) {
         if (c->h_stats_pinned) cudaFreeHost(c->h_stats);
         else std::free(c->h_stats);
@@ -666,6 +847,14 @@ so_status so_debug_set_dry_run(so_ctx *c, int32_t on)
     if (!c) return SO_ERR_INVALID_ARG;
     if (c->bound) return SO_ERR_STATE;
     c->dry_run = on != 0;
+    return SO_OK;
+}
+
+so_status so_debug_set_step_variant(so_ctx *c, int32_t variant)
+{
+    if (!c || variant < 0 || variant > 14) return SO_ERR_INVALID_ARG;
+    if (c->phase != kIdle) return SO_ERR_STATE;
+    c->step_variant = variant;
     return SO_OK;
 }
 

@@ -24,10 +24,13 @@ class BucketedAdamW:
     GUARD = 4096            # bytes of sentinel before and after every arena
 
     def __init__(self, numel: Sequence[int], bucket_elems: int, grad_dtype: str = "bf16",
-                 undo_slots: int = B.SO_ALL, device: str = "cuda", guard_bands: bool = False):
+                 undo_slots: int = B.SO_ALL, device: str = "cuda", guard_bands: bool = False,
+                 step_variant: int = 0):
         self.device = torch.device(device)
         gd = B.SO_GRAD_BF16 if grad_dtype == "bf16" else B.SO_GRAD_FP32
         self.ctx, self.info = B.so_layout_init(list(numel), bucket_elems, gd, undo_slots)
+        if step_variant:
+            B.so_debug_set_step_variant(self.ctx, step_variant)
         self.grad_torch_dtype = torch.bfloat16 if gd == B.SO_GRAD_BF16 else torch.float32
         self.guard_bands = guard_bands
         i = self.info

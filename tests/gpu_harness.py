@@ -91,12 +91,12 @@ def check_stats(stats, orc_res, max_grad_norm: float, rep: Report) -> None:
 
 
 def run_lockstep(w: W.Workload, steps: int, undo_slots: int = B.SO_ALL,
-                 speculative: bool = True, guard_bands: bool = True):
+                 speculative: bool = True, guard_bands: bool = True, step_variant: int = 0):
     """Full element-by-element parity over `steps` iterations of workload w."""
     hp = hparams_of(w)
     stream = torch.cuda.current_stream()
     opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, undo_slots,
-                        guard_bands=guard_bands)
+                        guard_bands=guard_bands, step_variant=step_variant)
     p0 = W.initial_master(w, device="cuda")
     opt.load_state(p0)
     opt.cast_params(stream=stream)

@@ -56,6 +56,15 @@ def test_tiny_ragged_tensors_and_odd_bucket_size():
     assert opt.info.slot_stride_elems != opt.info.bucket_elems
 
 
+@pytest.mark.parametrize("name", ["tiny", "tiny_ragged"])
+def test_register_variant_of_the_step_lockstep(name):
+    """The step kernel that keeps everything in registers (no shared-memory
+    staging) against the oracle."""
+    rep, _ = run_lockstep(W.by_name(name), steps=8, step_variant=1)
+    assert rep.decisions[6] == S
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+
+
 def test_tiny_without_clipping_commits():
     w = W.tiny()
     w.max_grad_norm = 0.0
@@ -91,10 +100,11 @@ def test_empty_model_on_the_device():
 # exactness of speculation (Section 4.4) and of the rollback
 # ---------------------------------------------------------------------------
 
-def _run_device_only(w, steps, undo_slots, speculative, bucket_order=None):
+def _run_device_only(w, steps, undo_slots, speculative, bucket_order=None, step_variant=0):
     hp = hparams_of(w)
     stream = torch.cuda.current_stream()
-    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, undo_slots)
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, undo_slots,
+                        step_variant=step_variant)
     opt.load_state(W.initial_master(w, device="cuda"))
     opt.cast_params(stream=stream)
     trace = []
@@ -126,8 +136,9 @@ def test_speculative_flow_is_bitwise_the_check_first_flow(name):
     windowed = _run_device_only(w, 9, undo_slots=2, speculative=True)
     shuffled = _run_device_only(w, 9, undo_slots=3, speculative=True,
                                 bucket_order=[3, 0, 2, 1] if name == "tiny" else [4, 1, 0, 3, 2])
-    assert ref[0] == full[0] == windowed[0] == shuffled[0]
-    assert ref[1] == full[1] == windowed[1] == shuffled[1]
+    registers = _run_device_only(w, 9, undo_slots=B.SO_ALL, speculative=True, step_variant=1)
+    assert ref[0] == full[0] == windowed[0] == shuffled[0] == registers[0]
+    assert ref[1] == full[1] == windowed[1] == shuffled[1] == registers[1]
 
 
 def test_repeat_runs_are_bitwise_identical():
@@ -206,7 +217,7 @@ def test_nonfinite_flag_for_every_special_bf16_pattern_and_position():
     n, bucket = 5000, 1024
     specials = [0x7F80, 0xFF80, 0x7F81, 0x7FC0, 0xFFFF, 0x7FFF]
     finite_extremes = [0x7F7F, 0xFF7F, 0x0001, 0x8001, 0x0000, 0x8000]
-    hp = oracle.HParams()
+    hp = oracle.HParams(max_grad_norm=0.0)
     opt = BucketedAdamW([n], bucket, undo_slots=0)
     base = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
     for pos in (0, 1023, 1024, 4095, 4096, 4999):
