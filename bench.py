@@ -104,6 +104,21 @@ class ClockSampler:
         return {"sm_mhz": med, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def max_over_ranks(values, device):
+    """Element-wise maximum over all ranks of the default process group."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_value(world: int, params_per_replica: int, ms_per_step: float) -> float:
+    """Replicas only: every rank steps its own copy of the workload, so the
+    job's throughput is world x params over the slowest rank's step time."""
+    return world * params_per_replica / (ms_per_step * 1e-3)
+
+
 def _hparams(w, oracle_mod=None):
     from paper_2509_21271_b200.binding import so_hparams
     return so_hparams(w.lr, w.beta1, w.beta2, w.eps, w.weight_decay, w.max_grad_norm)
@@ -284,19 +299,16 @@ def main():
 
     # ---- max over ranks ----------------------------------------------------
     if dist is not None:
-        vals = torch.tensor([elapsed_ms, e2e["ms"] if e2e else 0.0], device="cuda",
-                            dtype=torch.float64)
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(vals[0])
+        elapsed_ms, e2e_ms = max_over_ranks([elapsed_ms, e2e["ms"] if e2e else 0.0], "cuda")
         if e2e:
-            e2e["ms"] = float(vals[1])
+            e2e["ms"] = e2e_ms
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
     ms_per_step = elapsed_ms / args.steps
-    value = world * N / (ms_per_step * 1e-3)
+    value = whole_job_value(world, N, ms_per_step)
     peak, peak_kind = _measured_peak()
     bpp = BYTES_PER_PARAM[w.grad_dtype]
     roofline = None
