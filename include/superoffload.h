@@ -58,7 +58,8 @@ enum {
     SO_ERR_UNDO_EXHAUSTED = -4,        /* no free slot for another speculative step  */
     SO_ERR_NOMEM = -5,                 /* host allocation failed                     */
     SO_ERR_UNSUPPORTED = -6,
-    SO_ERR_TIMEOUT = -7                /* a kernel's bounded wait on its own copies ran out */
+    SO_ERR_TIMEOUT = -7,               /* a kernel's bounded wait on its own copies ran out */
+    SO_ERR_TOO_LARGE = -8              /* input exceeds a fixed built-in capacity           */
 };
 
 enum { SO_GRAD_BF16 = 0, SO_GRAD_FP32 = 1 };
@@ -228,6 +229,41 @@ so_status so_cast_params(so_ctx *ctx, int32_t bucket, void *stream);
  */
 so_status so_iteration_host(so_ctx *ctx, const so_hparams *hp, const void *host_grad,
                             void *host_param_bf16, void *stream, so_step_result *out);
+
+/*
+ * so_grad_check_static -- the gradient check for callers that cannot allocate.
+ * (The paper has no counterpart: this is a packaging variant of so_grad_check,
+ * not a step of its method.)
+ *
+ * so_grad_check needs a scratch arena that somebody allocated with cudaMalloc
+ * or a framework allocator.  Some callers have neither: code running inside a
+ * memory pool that is already fully handed out, start-up or diagnostic paths
+ * where a device-synchronising allocation is not acceptable, plug-ins that are
+ * given raw pointers and nothing else.  This entry point needs no context and
+ * no scratch from the caller: its tile sums live in a fixed array inside the
+ * library image (SO_STATIC_CHECK_MAX_ELEMS / 1024 doubles = 512 KB of device
+ * memory on every GPU that uses the library, held until the process exits).
+ * It calls no cudaMalloc / cudaFree and nothing else that allocates.
+ *   grad          DEVICE, flat gradient of n_elems values in grad_dtype,
+ *                 16-byte aligned (input; not modified)
+ *   n_elems       0 .. SO_STATIC_CHECK_MAX_ELEMS; larger -> SO_ERR_TOO_LARGE
+ *   max_grad_norm clip threshold for the coefficient (<= 0: coefficient 1)
+ *   out_device    DEVICE, 8-byte aligned so_grad_stats written by the call
+ *                 (sumsq, norm, clip_coef, nonfinite); caller-owned output
+ * Enqueues two kernels on `stream` and returns; no synchronisation, no host
+ * copy.  Same summation order as so_grad_check over one bucket of n_elems.
+ * The first call on each device looks up the device address of the built-in
+ * array (cudaGetSymbolAddress, with that device current) and caches it; make
+ * that first call outside any stream capture.  All calls on a device share the
+ * one array: it keeps whatever the previous call left, which is harmless
+ * because each call overwrites every entry it later reads (nothing has to
+ * start at zero), but two calls whose kernels overlap on the GPU (different
+ * streams, or different threads/processes' streams of one process) race on it
+ * -- serialise them.
+ */
+#define SO_STATIC_CHECK_MAX_ELEMS (1 << 26)
+so_status so_grad_check_static(const void *grad, int64_t n_elems, int32_t grad_dtype,
+                               double max_grad_norm, void *stream, so_grad_stats *out_device);
 
 /* Slot of the state arenas that holds bucket b's committed master/m/v. */
 so_status so_bucket_slot(const so_ctx *ctx, int32_t bucket, int32_t *slot);

@@ -16,6 +16,8 @@ SO_OK = 0
 SO_ERR_INVALID_ARG, SO_ERR_STATE, SO_ERR_CUDA = -1, -2, -3
 SO_ERR_UNDO_EXHAUSTED, SO_ERR_NOMEM, SO_ERR_UNSUPPORTED = -4, -5, -6
 SO_ERR_TIMEOUT = -7
+SO_ERR_TOO_LARGE = -8
+SO_STATIC_CHECK_MAX_ELEMS = 1 << 26
 SO_GRAD_BF16, SO_GRAD_FP32 = 0, 1
 SO_DECISION_COMMIT, SO_DECISION_SKIP, SO_DECISION_CLIP_RESTEP = 0, 1, 2
 SO_ALL = -1
@@ -70,7 +72,7 @@ _lib = None
 
 EXPORTS = ["so_layout_init", "so_layout_get_info", "so_layout_tensor", "so_layout_bind",
            "so_grad_check", "so_adam_step_speculative", "so_validate_commit_or_rollback",
-           "so_cast_params", "so_iteration_host", "so_bucket_slot", "so_get_step", "so_set_step",
+           "so_cast_params", "so_iteration_host", "so_grad_check_static", "so_bucket_slot", "so_get_step", "so_set_step",
            "so_pending_buckets", "so_get_counters", "so_last_cuda_error", "so_strerror",
            "so_destroy", "so_debug_set_dry_run", "so_debug_set_bucket_stats",
            "so_debug_set_step_variant"]
@@ -98,6 +100,7 @@ def lib() -> C.CDLL:
         "so_validate_commit_or_rollback": [vp, P(so_hparams), vp, P(so_step_result)],
         "so_cast_params": [vp, i32, vp],
         "so_iteration_host": [vp, P(so_hparams), vp, vp, vp, P(so_step_result)],
+        "so_grad_check_static": [vp, i64, i32, dbl, vp, vp],
         "so_bucket_slot": [vp, i32, P(i32)],
         "so_get_step": [vp, P(i64)],
         "so_set_step": [vp, i64],
@@ -219,6 +222,14 @@ def so_iteration_host(ctx, hp, host_grad: int, host_param_bf16: int, stream=None
     _ok(ctx, lib().so_iteration_host(ctx, C.byref(h), host_grad, host_param_bf16 or None,
                                      _stream(stream), C.byref(out)), "so_iteration_host")
     return out
+
+
+def so_grad_check_static(grad: int, n_elems: int, grad_dtype: int, max_grad_norm: float,
+                         stream, out_device: int) -> None:
+    """Gradient check without any allocation: `grad` and `out_device` are raw
+    device addresses (a gradient buffer and a 32-byte so_grad_stats record)."""
+    _ok(None, lib().so_grad_check_static(grad, n_elems, grad_dtype, max_grad_norm,
+                                         _stream(stream), out_device), "so_grad_check_static")
 
 
 def so_bucket_slot(ctx, bucket: int) -> int:

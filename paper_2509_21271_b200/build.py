@@ -10,8 +10,9 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libsuperoffload.so")
-SOURCES = [os.path.join(CSRC, "superoffload.cu")]
-_DEPS = SOURCES + [os.path.join(CSRC, "so_kernels.cuh"), os.path.join(INCLUDE, "superoffload.h")]
+SOURCES = [os.path.join(CSRC, "superoffload.cu"), os.path.join(CSRC, "so_static_check.cu")]
+_DEPS = SOURCES + [os.path.join(CSRC, "so_kernels.cuh"), os.path.join(CSRC, "so_step_tma.cuh"),
+                   os.path.join(INCLUDE, "superoffload.h")]
 
 
 def _nvcc() -> str:

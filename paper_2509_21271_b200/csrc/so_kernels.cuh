@@ -352,7 +352,7 @@ __global__ void __launch_bounds__(kThreads) grad_check_kernel(const __grid_const
 // g^2 is formed in double, so it cannot overflow for a finite fp32/bf16 input,
 // and a sum of non-negative finite doubles this long cannot overflow either: a
 // tile sum is Inf or NaN exactly when the tile holds a NaN or an infinity.
-__global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(const double *partials,
+static __global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(const double *partials,
                                                                       BucketStats *stats,
                                                                       Geometry geo)
 {
@@ -391,7 +391,7 @@ __global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(const dou
 // ---------------------------------------------------------------------------
 // stand-alone cast: fp32 master (slot src) -> bf16 copy of the bucket
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads) cast_params_kernel(const __grid_constant__ CastArgs a)
+static __global__ void __launch_bounds__(kThreads) cast_params_kernel(const __grid_constant__ CastArgs a)
 {
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);

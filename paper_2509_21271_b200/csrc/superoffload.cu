@@ -825,6 +825,7 @@ const char *so_strerror(so_status s)
         case SO_ERR_NOMEM: return "host allocation failed";
         case SO_ERR_UNSUPPORTED: return "unsupported";
         case SO_ERR_TIMEOUT: return "a kernel gave up waiting for one of its own copies";
+        case SO_ERR_TOO_LARGE: return "input exceeds the fixed built-in capacity of this entry point";
         default: return "unknown status";
     }
 }
