@@ -272,3 +272,36 @@ def test_gpt2_small_clip_path_lockstep():
     rep, opt = run_lockstep(W.gpt2_small(clip=True), steps=3, guard_bands=False)
     assert rep.decisions == [R] * 3
     assert rep.max_ulp["p"] <= 2
+
+
+# ---------------------------------------------------------------------------
+# the host-fed, bucket-pipelined iteration
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("name,undo", [("tiny", B.SO_ALL), ("tiny_ragged", 2), ("tiny", 0)])
+def test_host_fed_iteration_is_bitwise_the_device_fed_one(name, undo):
+    """so_iteration_host (pinned gradients in, bf16 parameters out, copies
+    overlapped per bucket) must leave exactly the state, statistics and
+    decisions of the ordinary call sequence, and deliver the committed bf16
+    parameters to the host -- through commits, clip re-steps and a skip."""
+    w = W.by_name(name)
+    hp = hparams_of(w)
+    stream = torch.cuda.current_stream()
+    ref = _run_device_only(w, 8, undo_slots=undo, speculative=True)
+
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, undo)
+    opt.load_state(W.initial_master(w, device="cuda"))
+    opt.cast_params(stream=stream)
+    host_g = torch.empty(w.total, dtype=torch.bfloat16, pin_memory=True)
+    host_p = torch.empty(w.total, dtype=torch.bfloat16, pin_memory=True)
+    trace = []
+    for step in range(1, 9):
+        host_g.copy_(W.gradients(w, step, device="cuda"))     # same bits as the reference run
+        res = B.so_iteration_host(opt.ctx, hp, host_g.data_ptr(), host_p.data_ptr(), stream)
+        trace.append((res.decision, res.stats.sumsq, res.stats.norm, res.stats.clip_coef,
+                      res.stats.nonfinite, res.step_after))
+        dev_pb = opt.gather_param_bf16().cpu()
+        assert torch.equal(host_p.view(torch.int16), dev_pb.view(torch.int16)), step
+    assert trace == ref[0]
+    assert _state_bytes(opt) == ref[1]
+    assert S in [t[0] for t in trace]
