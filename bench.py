@@ -217,12 +217,20 @@ def main():
 
     hp = _hparams(w)
     stream = torch.cuda.current_stream()
-    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, args.undo_slots,
+    undo = args.undo_slots
+    if undo < 0:
+        # as many undo slots as fit next to the 16 B/param resident state
+        stride = (w.bucket_elems + 63) // 64 * 64
+        free_bytes, _ = torch.cuda.mem_get_info()
+        gsz_arena = 2 if w.grad_dtype == "bf16" else 4
+        resident = w.n_buckets * stride * (12 + gsz_arena + 2)
+        room = free_bytes - resident - (6 << 30)
+        undo = max(0, min(w.n_buckets, room // (12 * stride)))
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, undo,
                         step_variant=args.step_variant)
-    opt.load_state(W.initial_master(w, device="cuda"))
+    opt.load_state_stream(W.iter_initial_master(w, device="cuda"))
     opt.cast_params(stream=stream)
-    g = W.gradients(w, 1, device="cuda")
-    opt.load_grads(g)
+    opt.load_grads_stream(W.iter_gradients(w, 1, device="cuda"))
     torch.cuda.synchronize()
     N = w.total
     nb = opt.n_buckets
@@ -279,10 +287,11 @@ def main():
 
     # ---- end to end through the host-buffer entry point -------------------
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and N <= (1 << 31):
         gsz = 2 if w.grad_dtype == "bf16" else 4
         host_g = torch.empty(N, dtype=opt.grad_torch_dtype, pin_memory=True)
-        host_g.copy_(g)
+        for start, piece in W.iter_gradients(w, 1, device="cuda"):
+            host_g[start:start + piece.numel()].copy_(piece)
         host_p = torch.empty(N, dtype=torch.bfloat16, pin_memory=True)
         for _ in range(3):
             B.so_iteration_host(opt.ctx, hp, host_g.data_ptr(), host_p.data_ptr(), stream)

@@ -141,7 +141,8 @@ so_status so_layout_tensor(const so_ctx *ctx, int32_t i, int64_t *flat_offset,
  * are fp32, grad is bf16 or fp32 per grad_dtype, param_bf16 is bf16.  The
  * caller fills master/m/v slot b with bucket b's initial state (m = v = 0 for
  * a fresh optimizer) and normally calls so_cast_params(SO_ALL) once.  Scratch
- * needs no initialisation.  Records the current device.  No launch, no sync.
+ * needs no initialisation by the caller (bind zeroes its 528-byte control
+ * block with one synchronous cudaMemset).  Records the current device.
  */
 so_status so_layout_bind(so_ctx *ctx, void *master, void *m, void *v, void *grad,
                          void *param_bf16, void *scratch);
@@ -297,8 +298,9 @@ so_status so_debug_set_bucket_stats(so_ctx *ctx, int32_t bucket, double sumsq,
                                     int32_t nonfinite);
 
 /* Which implementation of the fused step runs: 0 (default) stages bulk copies
- * through shared memory, 1 keeps everything in registers.  Both produce the
- * same bits; the switch exists for measurements and for testing both. */
+ * through shared memory, 1 keeps everything in registers, 10 and 11 are the
+ * default with other pipeline shapes.  All produce the same bits; the switch
+ * exists for measurements and for testing them against each other. */
 so_status so_debug_set_step_variant(so_ctx *ctx, int32_t variant);
 
 #ifdef __cplusplus

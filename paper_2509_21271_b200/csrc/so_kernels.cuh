@@ -175,43 +175,38 @@ __device__ __forceinline__ double warp_fold(double x)
 // bias corrections into per-step scalars (one division and one square root per
 // element); it agrees with the textbook order to a few 1e-16 relative.
 
-// sqrt(x) for x >= 0 in double, to within an ulp: hardware reciprocal-square-
-// root seed (about 20 bits, from the upper word) and two coupled Newton steps
-// on g ~ sqrt(x), h ~ 1/(2 sqrt(x)), then one residual correction.  Straight-
-// line code: the library routine's range checks and slow path are not needed
-// here (x is a finite, non-negative, never subnormal second moment; x = 0 is
-// selected away at the end; a NaN/Inf input only occurs in a speculative step
-// that validation discards).
+// sqrt(x) for x >= 0 in double, to within about an ulp: hardware reciprocal-
+// square-root seed (about 20 bits, from the upper word) and two coupled Newton
+// steps on g ~ sqrt(x), h ~ 1/(2 sqrt(x)).  Straight-line code: the library
+// routine's range checks and slow path are not needed here (x is a finite,
+// non-negative, never subnormal second moment).  The seed is taken of
+// max(x, 1e-290): for every real input that changes nothing, and for x = 0 it
+// keeps the seed finite so that g = 0 * seed = 0 comes out exactly.  A NaN/Inf
+// input only occurs in a speculative step that validation discards.
 __device__ __forceinline__ double sqrt_nonneg(double x)
 {
     double y;
-    asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
+    const double xs = fmax(x, 1e-290);
+    asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(xs));
     double g = __dmul_rn(x, y);
     double h = __dmul_rn(0.5, y);
     double r = __fma_rn(-g, h, 0.5);
     g = __fma_rn(g, r, g);
     h = __fma_rn(h, r, h);
     r = __fma_rn(-g, h, 0.5);
-    g = __fma_rn(g, r, g);
-    h = __fma_rn(h, r, h);
-    const double d = __fma_rn(-g, g, x);
-    g = __fma_rn(d, h, g);
-    return x > 0.0 ? g : x;
+    return __fma_rn(g, r, g);
 }
 
-// a / b for finite b >= eps-ish > 0, to within an ulp or two: reciprocal seed
-// (about 20 bits), two Newton steps, one residual correction of the quotient.
-__device__ __forceinline__ double div_pos(double a, double b)
+// 1 / b for finite, normal b > 0, to within an ulp or two: reciprocal seed
+// (about 20 bits) and two Newton steps.
+__device__ __forceinline__ double rcp_pos(double b)
 {
     double y;
     asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(b));
     double e = __fma_rn(-b, y, 1.0);
     y = __fma_rn(y, e, y);
     e = __fma_rn(-b, y, 1.0);
-    y = __fma_rn(y, e, y);
-    const double q = __dmul_rn(a, y);
-    const double r = __fma_rn(-b, q, a);
-    return __fma_rn(r, y, q);
+    return __fma_rn(y, e, y);
 }
 
 template <bool kScaled>
@@ -225,7 +220,7 @@ __device__ __forceinline__ void adamw_element(float g, float &p, float &m, float
     const double m64 = __dadd_rn(__dmul_rn(k.beta1, (double)m), __dmul_rn(k.omb1, gs));
     const double v64 = __dadd_rn(__dmul_rn(k.beta2, (double)v), __dmul_rn(k.omb2, sq));
     const double denom = __fma_rn(sqrt_nonneg(v64), k.rsqrt_bc2, k.eps);
-    const double u = __dmul_rn(k.step_size, div_pos(m64, denom));
+    const double u = __dmul_rn(__dmul_rn(k.step_size, m64), rcp_pos(denom));
     const double p64 = __fma_rn((double)p, k.decay, -u);
     p = __double2float_rn(p64);
     m = __double2float_rn(m64);

@@ -1,10 +1,13 @@
-// Fused AdamW step with bulk-copy (TMA) staging through shared memory.
+// Fused AdamW step with bulk-copy (TMA) staging through shared memory and
+// dynamic tile scheduling.
 //
 // Same arithmetic, same tile/row/quad ownership and same summation order as
-// adamw_step_kernel; only the data movement differs.  The register version
-// keeps a warp's loads in flight only while that warp is not computing, which
-// leaves both DRAM and the issue slots half idle.  Here every warp runs a
-// private software pipeline over *chunks* of 256 elements:
+// adamw_step_kernel; only the data movement and the work distribution differ.
+//
+// Data movement.  The register version keeps a warp's loads in flight only
+// while that warp is not computing, which leaves both DRAM and the issue slots
+// half idle.  Here every warp runs a private software pipeline over *chunks*
+// (2 or 4 rows of a tile), consumed one row at a time:
 //
 //   global --cp.async.bulk--> shared (kStagesIn chunks ahead, completion on an
 //   mbarrier) --> registers --> fp64 AdamW --> shared --cp.async.bulk--> global
@@ -14,9 +17,20 @@
 // well.  Pipelines are private to a warp, so there is no block-wide
 // synchronisation and the deterministic per-tile reduction is unchanged.
 // Bulk copies need 16-byte aligned addresses and sizes: slots are 256-byte
-// aligned and chunk starts are multiples of 256 elements, so only a chunk
+// aligned and chunk starts are multiples of 128 elements, so only a chunk
 // whose valid length is not a multiple of 8 elements (the ragged end of a
 // bucket) takes the guarded register path instead.
+//
+// Work distribution.  Tiles are not dealt out statically: each warp claims its
+// next tile from a global counter (one atomicAdd per 1024 elements, issued one
+// tile ahead of need).  With a static round-robin the SMs drift apart and the
+// set of DRAM pages being touched spreads; claiming in order keeps every SM
+// working inside one compact, advancing window, which on B200 is worth about
+// 10 % of HBM throughput for this 4-in / 4-out stream pattern (measured with a
+// copy-only kernel: 5.9-6.3 TB/s static, 6.8-6.9 TB/s dynamic).  Which warp
+// processes a tile has no influence on any result: tile sums are per tile.
+// The counter lives in a small control block in scratch; the last warp to
+// finish puts it back to zero for the next launch.
 //
 // Every wait on an mbarrier is bounded: on expiry the kernel raises a status
 // word for the host, drains what it can with bounded waits, and returns.
@@ -27,6 +41,15 @@
 namespace so {
 
 constexpr uint32_t kSpinLimit = 1u << 20;              // bounded mbarrier polling
+constexpr int kCounterPairs = 64;                      // launches that may overlap in time
+
+// Control block in scratch (zeroed once at bind time): a status record and a
+// ring of {next tile, finished warps} counter pairs, one pair per launch.
+struct ControlBlock {
+    int32_t status;
+    int32_t pad[3];
+    uint32_t counters[kCounterPairs][2];
+};
 
 // Shape of the per-warp pipeline: rows (of 128 elements) per chunk, warps per
 // block (one block per SM), chunks in flight ahead of the arithmetic, and
@@ -42,6 +65,18 @@ struct PipeShape {
     static constexpr int kThreads = kWarps_ * 32;
 };
 
+// What a pipeline stage holds, written by the issuing lane and read by the
+// whole warp when the chunk is consumed.
+struct ChunkDesc {
+    uint32_t start;        // first element of the chunk within its bucket
+    uint32_t len;          // valid elements (0 marks the end of the warp's work)
+    uint32_t n;            // elements in the bucket
+    uint32_t tile_in_bucket;
+    int32_t bucket, src_slot, dst_slot;
+    uint32_t flags;        // kLastOfTile | kRagged
+};
+constexpr uint32_t kLastOfTile = 1u, kRagged = 2u;
+
 template <typename GradT, typename S>
 struct TmaLayout {
     static constexpr int kGradBytes = S::kChunkElems * (int)sizeof(GradT);
@@ -49,8 +84,9 @@ struct TmaLayout {
     static constexpr int kInStage = 3 * kF32Bytes + kGradBytes;            // p, m, v, g
     static constexpr int kOutStage = 3 * kF32Bytes + S::kChunkElems * 2;   // p, m, v, bf16
     static constexpr int kWarpBytes = S::kStagesIn * kInStage + S::kStagesOut * kOutStage;
-    static constexpr int kBarrierBytes = 128 * ((S::kWarps * S::kStagesIn * 8 + 127) / 128);
-    static constexpr int kSmemBytes = kBarrierBytes + S::kWarps * kWarpBytes;
+    // per warp and input stage: one mbarrier (8 B) and one descriptor (32 B)
+    static constexpr int kHeaderBytes = 128 * ((S::kWarps * S::kStagesIn * 40 + 127) / 128);
+    static constexpr int kSmemBytes = kHeaderBytes + S::kWarps * kWarpBytes;
 };
 
 // ---- PTX wrappers -----------------------------------------------------------
@@ -130,78 +166,11 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// ---- cursor over the chunks a warp owns -------------------------------------
-//
-// Tiles are dealt to warps round-robin (tile = warp, warp + n_warps, ...); a
-// tile holds up to 4 chunks.  The cursor walks the warp's chunks in order and
-// skips tiles that lie beyond the end of a partial last bucket.
-struct ChunkCursor {
-    uint32_t tile;       // index in the launch's tile space
-    uint32_t sub;        // chunk within the tile
-    uint32_t n;          // elements in the tile's bucket
-    uint32_t base;       // first element of the tile within the bucket
-    int32_t bucket, src_slot, dst_slot;
-    bool valid;
-};
-
-__device__ __forceinline__ void cursor_seek(ChunkCursor &c, const StepArgs &a, uint32_t n_warps)
-{
-    const uint32_t tps = a.geo.tiles_per_slot;
-    const uint32_t total = (uint32_t)a.n_entries * tps;
-    while (c.tile < total) {
-        const uint32_t j = c.tile / tps;
-        const uint32_t lt = c.tile - j * tps;
-        const BucketEntry e = a.e[j];
-        const uint32_t n = (e.bucket == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
-        if (lt * kTileElems < n) {
-            c.n = n;
-            c.base = lt * kTileElems;
-            c.bucket = e.bucket;
-            c.src_slot = e.src_slot;
-            c.dst_slot = e.dst_slot;
-            c.sub = 0;
-            c.valid = true;
-            return;
-        }
-        c.tile += n_warps;
-    }
-    c.valid = false;
-}
-
-template <typename S>
-__device__ __forceinline__ void cursor_next(ChunkCursor &c, const StepArgs &a, uint32_t n_warps)
-{
-    c.sub += 1;
-    if (c.sub < (uint32_t)S::kChunksPerTile && c.base + c.sub * S::kChunkElems < c.n) return;
-    c.tile += n_warps;
-    cursor_seek(c, a, n_warps);
-}
-
-template <typename S>
-__device__ __forceinline__ uint32_t chunk_start(const ChunkCursor &c)
-{
-    return c.base + c.sub * S::kChunkElems;
-}
-
-template <typename S>
-__device__ __forceinline__ uint32_t chunk_len(const ChunkCursor &c)
-{
-    const uint32_t left = c.n - chunk_start<S>(c);
-    return left < (uint32_t)S::kChunkElems ? left : (uint32_t)S::kChunkElems;
-}
-
-template <typename S>
-__device__ __forceinline__ bool chunk_is_last_of_tile(const ChunkCursor &c)
-{
-    return c.sub + 1 == (uint32_t)S::kChunksPerTile ||
-           c.base + (c.sub + 1) * S::kChunkElems >= c.n;
-}
-
 // ---- the kernel ---------------------------------------------------------------
 
 template <typename GradT, bool kSpec, typename S>
 __global__ void __launch_bounds__(S::kThreads, 1)
-adamw_step_tma_kernel(const __grid_constant__ StepArgs a, int32_t *status)
+adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, int pair)
 {
     using L = TmaLayout<GradT, S>;
     constexpr int kStagesIn = S::kStagesIn, kStagesOut = S::kStagesOut;
@@ -210,55 +179,108 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, int32_t *status)
 
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t wib = threadIdx.x >> 5;
-    const uint32_t warp = blockIdx.x * kTmaWarps + wib;
     const uint32_t n_warps = gridDim.x * kTmaWarps;
     const uint32_t tps = a.geo.tiles_per_slot;
+    const uint32_t total_tiles = (uint32_t)a.n_entries * tps;
 
     const uint32_t bars = smem_u32(smem) + wib * kStagesIn * 8;
-    unsigned char *wbase = smem + L::kBarrierBytes + wib * L::kWarpBytes;
+    ChunkDesc *descs = reinterpret_cast<ChunkDesc *>(smem + kTmaWarps * kStagesIn * 8) +
+                       wib * kStagesIn;
+    unsigned char *wbase = smem + L::kHeaderBytes + wib * L::kWarpBytes;
     unsigned char *out_base = wbase + kStagesIn * L::kInStage;
+    uint32_t *next_tile = &ctrl->counters[pair][0];
+    uint32_t *done_warps = &ctrl->counters[pair][1];
+
+    const uint64_t policy = l2_evict_first_policy();
+    const int64_t stride = a.geo.stride;
+
+    // ---- producer state: meaningful in lane 0 only ----
+    uint32_t cur_tile = 0, claimed = 0;        // tile being cut into chunks; tile claimed ahead
+    uint32_t cur_sub = 0, cur_n = 0, cur_base = 0, cur_lt = 0;
+    int32_t cur_bucket = 0, cur_src = 0, cur_dst = 0;
+    bool cur_valid = false;
+
+    // take the tile claimed earlier, claim the next one (its value is not
+    // needed until this tile is used up), skip tiles past a partial bucket's end
+    auto next_tile_for_lane0 = [&]() {
+        for (;;) {
+            cur_tile = claimed;
+            claimed = atomicAdd(next_tile, 1u);
+            if (cur_tile >= total_tiles) {
+                cur_valid = false;
+                return;
+            }
+            const uint32_t j = cur_tile / tps;
+            const uint32_t lt = cur_tile - j * tps;
+            const BucketEntry e = a.e[j];
+            const uint32_t n =
+                (e.bucket == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
+            if (lt * kTileElems < n) {
+                cur_n = n;
+                cur_lt = lt;
+                cur_base = lt * kTileElems;
+                cur_bucket = e.bucket;
+                cur_src = e.src_slot;
+                cur_dst = e.dst_slot;
+                cur_sub = 0;
+                cur_valid = true;
+                return;
+            }
+        }
+    };
+
+    // describe the next chunk in stage s and start its loads (lane 0 only)
+    auto produce = [&](int s) {
+        ChunkDesc d;
+        if (!cur_valid) {
+            d.start = d.len = d.n = d.tile_in_bucket = d.flags = 0;
+            d.bucket = d.src_slot = d.dst_slot = 0;
+            descs[s] = d;
+            return;
+        }
+        const uint32_t start = cur_base + cur_sub * S::kChunkElems;
+        const uint32_t left = cur_n - start;
+        const uint32_t len = left < (uint32_t)S::kChunkElems ? left : (uint32_t)S::kChunkElems;
+        const bool last = cur_sub + 1 == (uint32_t)S::kChunksPerTile ||
+                          start + S::kChunkElems >= cur_n;
+        const bool ragged = (len & 7u) != 0;
+        d.start = start;
+        d.len = len;
+        d.n = cur_n;
+        d.tile_in_bucket = cur_lt;
+        d.bucket = cur_bucket;
+        d.src_slot = cur_src;
+        d.dst_slot = cur_dst;
+        d.flags = (last ? kLastOfTile : 0u) | (ragged ? kRagged : 0u);
+        descs[s] = d;
+        if (!ragged) {
+            const int64_t src = (int64_t)cur_src * stride + start;
+            const uint32_t bar = bars + s * 8;
+            const uint32_t dst = smem_u32(wbase + s * L::kInStage);
+            const uint32_t fbytes = len * 4u, gbytes = len * (uint32_t)sizeof(GradT);
+            mbar_expect_tx(bar, 3u * fbytes + gbytes);
+            bulk_load(dst, a.master + src, fbytes, bar, policy);
+            bulk_load(dst + L::kF32Bytes, a.mom + src, fbytes, bar, policy);
+            bulk_load(dst + 2 * L::kF32Bytes, a.var + src, fbytes, bar, policy);
+            bulk_load(dst + 3 * L::kF32Bytes,
+                      static_cast<const GradT *>(a.grad) + (int64_t)cur_bucket * stride + start,
+                      gbytes, bar, policy);
+        }
+        if (last) next_tile_for_lane0();
+        else cur_sub += 1;
+    };
 
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < kStagesIn; ++s) mbar_init(bars + s * 8, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
+        claimed = atomicAdd(next_tile, 1u);
+        next_tile_for_lane0();
+#pragma unroll 1
+        for (int s = 0; s < kStagesIn; ++s) produce(s);
     }
     __syncwarp();
-
-    const uint64_t policy = l2_evict_first_policy();
-    const int64_t stride = a.geo.stride;
-
-    // issue the four bulk loads of the chunk under `c` into stage s (lane 0 only)
-    auto issue_load = [&](const ChunkCursor &c, int s) {
-        const uint32_t len = chunk_len<S>(c);
-        if ((len & 7u) != 0) return;                       // ragged chunk: register path
-        const uint32_t start = chunk_start<S>(c);
-        const int64_t src = (int64_t)c.src_slot * stride + start;
-        const uint32_t bar = bars + s * 8;
-        const uint32_t dst = smem_u32(wbase + s * L::kInStage);
-        const uint32_t fbytes = len * 4u, gbytes = len * (uint32_t)sizeof(GradT);
-        mbar_expect_tx(bar, 3u * fbytes + gbytes);
-        bulk_load(dst, a.master + src, fbytes, bar, policy);
-        bulk_load(dst + L::kF32Bytes, a.mom + src, fbytes, bar, policy);
-        bulk_load(dst + 2 * L::kF32Bytes, a.var + src, fbytes, bar, policy);
-        bulk_load(dst + 3 * L::kF32Bytes,
-                  static_cast<const GradT *>(a.grad) + (int64_t)c.bucket * stride + start, gbytes,
-                  bar, policy);
-    };
-
-    ChunkCursor ld;                    // next chunk to load
-    ld.tile = warp;
-    cursor_seek(ld, a, n_warps);
-    ChunkCursor cs = ld;               // next chunk to consume
-
-    // prologue: fill the pipeline
-#pragma unroll 1
-    for (int s = 0; s < kStagesIn; ++s) {
-        if (!ld.valid) break;
-        if (lane == 0) issue_load(ld, s);
-        cursor_next<S>(ld, a, n_warps);
-    }
 
     uint32_t phases = 0;               // parity bit per input stage
     int stage = 0, ostage = 0;
@@ -266,11 +288,13 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, int32_t *status)
     bool failed = false;
 
 #pragma unroll 1
-    while (cs.valid) {
-        const uint32_t len = chunk_len<S>(cs);
-        const uint32_t start = chunk_start<S>(cs);
-        const bool bulk = (len & 7u) == 0;
-        float gq[kChunkRows][4], pq[kChunkRows][4], mq[kChunkRows][4], vq[kChunkRows][4];
+    for (;;) {
+        const ChunkDesc d = descs[stage];
+        if (d.len == 0) break;
+        const uint32_t len = d.len, start = d.start;
+        const bool bulk = (d.flags & kRagged) == 0;
+        const int64_t dst = (int64_t)d.dst_slot * stride;
+        uint16_t *pb = a.param_bf16 + (int64_t)d.bucket * stride;
 
         if (bulk) {
             if (!mbar_wait_bounded(bars + stage * 8, (phases >> stage) & 1u)) {
@@ -278,85 +302,52 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, int32_t *status)
                 break;
             }
             phases ^= 1u << stage;
-            const unsigned char *in = wbase + stage * L::kInStage;
-#pragma unroll
-            for (int r = 0; r < kChunkRows; ++r) {
-                const uint32_t off = r * kRowElems + lane * 4;     // element within the chunk
-                if (off < len) {
-                    const float4 p4 = *reinterpret_cast<const float4 *>(in + off * 4);
-                    const float4 m4 = *reinterpret_cast<const float4 *>(in + L::kF32Bytes + off * 4);
-                    const float4 v4 =
-                        *reinterpret_cast<const float4 *>(in + 2 * L::kF32Bytes + off * 4);
-                    pq[r][0] = p4.x; pq[r][1] = p4.y; pq[r][2] = p4.z; pq[r][3] = p4.w;
-                    mq[r][0] = m4.x; mq[r][1] = m4.y; mq[r][2] = m4.z; mq[r][3] = m4.w;
-                    vq[r][0] = v4.x; vq[r][1] = v4.y; vq[r][2] = v4.z; vq[r][3] = v4.w;
-                    if (sizeof(GradT) == 2) {
-                        const uint2 g2 = *reinterpret_cast<const uint2 *>(in + 3 * L::kF32Bytes +
-                                                                          off * 2);
-                        gq[r][0] = __uint_as_float(g2.x << 16);
-                        gq[r][1] = __uint_as_float(g2.x & 0xFFFF0000u);
-                        gq[r][2] = __uint_as_float(g2.y << 16);
-                        gq[r][3] = __uint_as_float(g2.y & 0xFFFF0000u);
-                    } else {
-                        const float4 g4 = *reinterpret_cast<const float4 *>(
-                            in + 3 * L::kF32Bytes + off * 4);
-                        gq[r][0] = g4.x; gq[r][1] = g4.y; gq[r][2] = g4.z; gq[r][3] = g4.w;
-                    }
-                } else {
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) gq[r][q] = pq[r][q] = mq[r][q] = vq[r][q] = 0.0f;
-                }
-            }
-        } else {
-            const GradT *g = static_cast<const GradT *>(a.grad) + (int64_t)cs.bucket * stride;
-            const int64_t src = (int64_t)cs.src_slot * stride;
-#pragma unroll
-            for (int r = 0; r < kChunkRows; ++r) {
-                const uint32_t idx = start + r * kRowElems + lane * 4;
-                load_quad(g, idx, cs.n, gq[r]);
-                load_quad(a.master + src, idx, cs.n, pq[r]);
-                load_quad(a.mom + src, idx, cs.n, mq[r]);
-                load_quad(a.var + src, idx, cs.n, vq[r]);
-            }
-        }
-        // every lane has copied its part of the stage: refill it
-        __syncwarp();
-        if (ld.valid) {
-            if (lane == 0) issue_load(ld, stage);
-            cursor_next<S>(ld, a, n_warps);
-        }
-
-#pragma unroll
-        for (int r = 0; r < kChunkRows; ++r)
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-                adamw_element<!kSpec>(gq[r][q], pq[r][q], mq[r][q], vq[r][q], a.k, acc);
-
-        const int64_t dst = (int64_t)cs.dst_slot * stride;
-        uint16_t *pb = a.param_bf16 + (int64_t)cs.bucket * stride;
-        if (bulk) {
             // the output stage is free once the bulk stores issued from it
             // kStagesOut chunks ago have finished reading shared memory
             if (lane == 0) bulk_wait_read<kStagesOut - 1>();
             __syncwarp();
+            const unsigned char *in = wbase + stage * L::kInStage;
             unsigned char *out = out_base + ostage * L::kOutStage;
-#pragma unroll
+            // one row (4 elements per lane) at a time: keeps the register
+            // footprint small enough for 16 warps per SM
+#pragma unroll 1
             for (int r = 0; r < kChunkRows; ++r) {
-                const uint32_t off = r * kRowElems + lane * 4;
-                if (off < len) {
-                    *reinterpret_cast<float4 *>(out + off * 4) =
-                        make_float4(pq[r][0], pq[r][1], pq[r][2], pq[r][3]);
-                    *reinterpret_cast<float4 *>(out + L::kF32Bytes + off * 4) =
-                        make_float4(mq[r][0], mq[r][1], mq[r][2], mq[r][3]);
-                    *reinterpret_cast<float4 *>(out + 2 * L::kF32Bytes + off * 4) =
-                        make_float4(vq[r][0], vq[r][1], vq[r][2], vq[r][3]);
-                    *reinterpret_cast<uint2 *>(out + 3 * L::kF32Bytes + off * 2) =
-                        make_uint2(pack_bf16x2(pq[r][0], pq[r][1]), pack_bf16x2(pq[r][2], pq[r][3]));
+                const uint32_t off = r * kRowElems + lane * 4;     // element within the chunk
+                if (off >= len) break;
+                float gq[4], pq[4], mq[4], vq[4];
+                const float4 p4 = *reinterpret_cast<const float4 *>(in + off * 4);
+                const float4 m4 = *reinterpret_cast<const float4 *>(in + L::kF32Bytes + off * 4);
+                const float4 v4 = *reinterpret_cast<const float4 *>(in + 2 * L::kF32Bytes + off * 4);
+                pq[0] = p4.x; pq[1] = p4.y; pq[2] = p4.z; pq[3] = p4.w;
+                mq[0] = m4.x; mq[1] = m4.y; mq[2] = m4.z; mq[3] = m4.w;
+                vq[0] = v4.x; vq[1] = v4.y; vq[2] = v4.z; vq[3] = v4.w;
+                if (sizeof(GradT) == 2) {
+                    const uint2 g2 = *reinterpret_cast<const uint2 *>(in + 3 * L::kF32Bytes + off * 2);
+                    gq[0] = __uint_as_float(g2.x << 16);
+                    gq[1] = __uint_as_float(g2.x & 0xFFFF0000u);
+                    gq[2] = __uint_as_float(g2.y << 16);
+                    gq[3] = __uint_as_float(g2.y & 0xFFFF0000u);
+                } else {
+                    const float4 g4 = *reinterpret_cast<const float4 *>(in + 3 * L::kF32Bytes + off * 4);
+                    gq[0] = g4.x; gq[1] = g4.y; gq[2] = g4.z; gq[3] = g4.w;
                 }
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    adamw_element<!kSpec>(gq[q], pq[q], mq[q], vq[q], a.k, acc);
+                *reinterpret_cast<float4 *>(out + off * 4) = make_float4(pq[0], pq[1], pq[2], pq[3]);
+                *reinterpret_cast<float4 *>(out + L::kF32Bytes + off * 4) =
+                    make_float4(mq[0], mq[1], mq[2], mq[3]);
+                *reinterpret_cast<float4 *>(out + 2 * L::kF32Bytes + off * 4) =
+                    make_float4(vq[0], vq[1], vq[2], vq[3]);
+                *reinterpret_cast<uint2 *>(out + 3 * L::kF32Bytes + off * 2) =
+                    make_uint2(pack_bf16x2(pq[0], pq[1]), pack_bf16x2(pq[2], pq[3]));
             }
             fence_async_smem();        // generic writes -> visible to the async proxy
+            // every lane is done with the input stage and has filled its part
+            // of the output stage: refill the one, drain the other
             __syncwarp();
             if (lane == 0) {
+                produce(stage);
                 const uint32_t src_s = smem_u32(out);
                 const uint32_t fbytes = len * 4u;
                 bulk_store(a.master + dst + start, src_s, fbytes, policy);
@@ -367,27 +358,37 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, int32_t *status)
             }
             ostage = (ostage + 1 == kStagesOut) ? 0 : ostage + 1;
         } else {
-#pragma unroll
+            const GradT *g = static_cast<const GradT *>(a.grad) + (int64_t)d.bucket * stride;
+            const int64_t src = (int64_t)d.src_slot * stride;
+#pragma unroll 1
             for (int r = 0; r < kChunkRows; ++r) {
                 const uint32_t idx = start + r * kRowElems + lane * 4;
-                if (idx < cs.n) {
-                    store_quad(a.master + dst, idx, cs.n, pq[r]);
-                    store_quad(a.mom + dst, idx, cs.n, mq[r]);
-                    store_quad(a.var + dst, idx, cs.n, vq[r]);
-                    store_quad_bf16(pb, idx, cs.n, pq[r]);
+                float gq[4], pq[4], mq[4], vq[4];
+                load_quad(g, idx, d.n, gq);
+                load_quad(a.master + src, idx, d.n, pq);
+                load_quad(a.mom + src, idx, d.n, mq);
+                load_quad(a.var + src, idx, d.n, vq);
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    adamw_element<!kSpec>(gq[q], pq[q], mq[q], vq[q], a.k, acc);
+                if (idx < d.n) {
+                    store_quad(a.master + dst, idx, d.n, pq);
+                    store_quad(a.mom + dst, idx, d.n, mq);
+                    store_quad(a.var + dst, idx, d.n, vq);
+                    store_quad_bf16(pb, idx, d.n, pq);
                 }
             }
+            __syncwarp();
+            if (lane == 0) produce(stage);
         }
 
-        if (chunk_is_last_of_tile<S>(cs)) {
+        if (d.flags & kLastOfTile) {
             if (kSpec) {
                 const double tile_sum = warp_fold(acc);
-                if (lane == 0)
-                    a.partials[(int64_t)cs.bucket * tps + cs.base / kTileElems] = tile_sum;
+                if (lane == 0) a.partials[(int64_t)d.bucket * tps + d.tile_in_bucket] = tile_sum;
             }
             acc = 0.0;
         }
-        cursor_next<S>(cs, a, n_warps);
         stage = (stage + 1 == kStagesIn) ? 0 : stage + 1;
     }
 
@@ -395,10 +396,21 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, int32_t *status)
         // a copy never completed: tell the host, then give the copies that are
         // still in flight a bounded chance to land before this block's shared
         // memory is released
-        if (lane == 0) atomicExch(status, 1);
+        if (lane == 0) atomicExch(&ctrl->status, 1);
         for (int s = 0; s < kStagesIn; ++s) mbar_wait_bounded(bars + s * 8, (phases >> s) & 1u);
     }
-    if (lane == 0) bulk_wait_all();
+    if (lane == 0) {
+        bulk_wait_all();
+        // The last warp of the launch to get here re-arms the counters.  The
+        // fence orders this warp's tile claims (including the look-ahead claim
+        // whose value is never used) before its arrival, so no claim can land
+        // after the reset.
+        __threadfence();
+        if (atomicAdd(done_warps, 1u) == n_warps - 1) {
+            *next_tile = 0;
+            *done_warps = 0;
+        }
+    }
     __syncwarp();
 }
 

@@ -35,7 +35,8 @@ struct so_ctx {
     double *d_partials = nullptr;
     BucketStats *d_stats = nullptr;     // n_buckets results, then one record whose first
                                         // word is the device status (0 = fine)
-    int32_t *d_status = nullptr;
+    ControlBlock *d_ctrl = nullptr;     // status word + tile counters, right after d_stats
+    uint32_t launch_seq = 0;            // picks the counter pair of each pipeline launch
     int step_variant = 0;               // 0: bulk-copy pipeline, 1: register path
     BucketStats *h_stats = nullptr;
     bool h_stats_pinned = false;
@@ -147,66 +148,57 @@ so_status after_launch(so_ctx *c)
 
 // ---- launches --------------------------------------------------------------
 
-// Shapes of the bulk-copy pipeline (rows per chunk, warps per block, input
-// stages, output stages).  Variant 0 is the default.
-using ShapeDefault = PipeShape<2, 12, 3, 1>;
-using ShapeA = PipeShape<2, 8, 4, 2>;
-using ShapeB = PipeShape<1, 16, 4, 2>;
-using ShapeC = PipeShape<1, 24, 3, 2>;
-using ShapeD = PipeShape<1, 32, 3, 1>;
-using ShapeE = PipeShape<2, 16, 2, 1>;
+// Shapes of the bulk-copy pipeline: rows per chunk, warps per block (one block
+// per SM), input stages, output stages.  The defaults came out of a sweep on
+// B200: 512-element chunks halve the per-chunk bookkeeping, two input stages of
+// 7 KB per warp keep ~140 KB of loads in flight per SM, and ten warps are the
+// most that fit in shared memory (nine with fp32 gradients).  The alternates
+// stay selectable for measurements (so_debug_set_step_variant 10 / 11).
+using ShapeBf16 = PipeShape<4, 10, 2, 1>;
+using ShapeFp32 = PipeShape<4, 9, 2, 1>;
+using ShapeAlt16 = PipeShape<2, 16, 3, 1>;      // bf16 gradients only
+using ShapeAlt12 = PipeShape<2, 12, 3, 1>;
 
-template <typename S>
+template <typename GradT, typename S>
 void launch_tma(so_ctx *c, const StepArgs &a, int n, bool speculative, cudaStream_t stream)
 {
     int64_t blocks = ((int64_t)n * a.geo.tiles_per_slot + S::kWarps - 1) / S::kWarps;
     if (blocks > c->num_sms) blocks = c->num_sms;
     const unsigned grid = (unsigned)(blocks < 1 ? 1 : blocks);
-    if (c->grad_dtype == SO_GRAD_BF16) {
-        const size_t sm = TmaLayout<uint16_t, S>::kSmemBytes;
-        if (speculative)
-            adamw_step_tma_kernel<uint16_t, true, S><<<grid, S::kThreads, sm, stream>>>(a, c->d_status);
-        else
-            adamw_step_tma_kernel<uint16_t, false, S><<<grid, S::kThreads, sm, stream>>>(a, c->d_status);
-    } else {
-        const size_t sm = TmaLayout<float, S>::kSmemBytes;
-        if (speculative)
-            adamw_step_tma_kernel<float, true, S><<<grid, S::kThreads, sm, stream>>>(a, c->d_status);
-        else
-            adamw_step_tma_kernel<float, false, S><<<grid, S::kThreads, sm, stream>>>(a, c->d_status);
-    }
+    // launches that may overlap in time (other streams) must not share a tile counter
+    const int pair = (int)(c->launch_seq++ % kCounterPairs);
+    const size_t sm = TmaLayout<GradT, S>::kSmemBytes;
+    if (speculative)
+        adamw_step_tma_kernel<GradT, true, S><<<grid, S::kThreads, sm, stream>>>(a, c->d_ctrl, pair);
+    else
+        adamw_step_tma_kernel<GradT, false, S><<<grid, S::kThreads, sm, stream>>>(a, c->d_ctrl, pair);
 }
 
 void launch_tma_variant(so_ctx *c, const StepArgs &a, int n, bool speculative, cudaStream_t stream)
 {
-    switch (c->step_variant) {
-        case 10: launch_tma<ShapeA>(c, a, n, speculative, stream); break;
-        case 11: launch_tma<ShapeB>(c, a, n, speculative, stream); break;
-        case 12: launch_tma<ShapeC>(c, a, n, speculative, stream); break;
-        case 13: launch_tma<ShapeD>(c, a, n, speculative, stream); break;
-        case 14: launch_tma<ShapeE>(c, a, n, speculative, stream); break;
-        default: launch_tma<ShapeDefault>(c, a, n, speculative, stream); break;
+    const bool bf16 = c->grad_dtype == SO_GRAD_BF16;
+    if (c->step_variant == 10 && bf16) {
+        launch_tma<uint16_t, ShapeAlt16>(c, a, n, speculative, stream);
+    } else if (c->step_variant == 11) {
+        if (bf16) launch_tma<uint16_t, ShapeAlt12>(c, a, n, speculative, stream);
+        else launch_tma<float, ShapeAlt12>(c, a, n, speculative, stream);
+    } else {
+        if (bf16) launch_tma<uint16_t, ShapeBf16>(c, a, n, speculative, stream);
+        else launch_tma<float, ShapeFp32>(c, a, n, speculative, stream);
     }
 }
 
 // The bulk-copy kernels stage through more than 48 KB of shared memory.
-template <typename S>
+template <typename GradT, typename S>
 cudaError_t allow_smem()
 {
+    static_assert(TmaLayout<GradT, S>::kSmemBytes <= 227 * 1024, "pipeline does not fit");
     const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-    cudaError_t e = cudaFuncSetAttribute(adamw_step_tma_kernel<uint16_t, true, S>, attr,
-                                         TmaLayout<uint16_t, S>::kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(adamw_step_tma_kernel<GradT, true, S>, attr,
+                                         TmaLayout<GradT, S>::kSmemBytes);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(adamw_step_tma_kernel<uint16_t, false, S>, attr,
-                                 TmaLayout<uint16_t, S>::kSmemBytes);
-    if constexpr (TmaLayout<float, S>::kSmemBytes <= 227 * 1024) {
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(adamw_step_tma_kernel<float, true, S>, attr,
-                                     TmaLayout<float, S>::kSmemBytes);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(adamw_step_tma_kernel<float, false, S>, attr,
-                                     TmaLayout<float, S>::kSmemBytes);
-    }
+        e = cudaFuncSetAttribute(adamw_step_tma_kernel<GradT, false, S>, attr,
+                                 TmaLayout<GradT, S>::kSmemBytes);
     return e;
 }
 
@@ -334,9 +326,12 @@ so_status finalize_check(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
             if (e != cudaSuccess) return cuda_fail(c, e);
             e = cudaStreamSynchronize(stream);
             if (e != cudaSuccess) return cuda_fail(c, e);
-            if (c->h_stats[c->n_buckets].nonfinite != 0 || c->h_stats[c->n_buckets].pad != 0) {
-                // a kernel gave up waiting for one of its own copies
-                cudaMemsetAsync(c->d_status, 0, sizeof(BucketStats), stream);
+            int32_t device_status = 0;
+            std::memcpy(&device_status, &c->h_stats[c->n_buckets], sizeof(device_status));
+            if (device_status != 0) {
+                // a kernel gave up waiting for one of its own copies; its tile
+                // counters may be left mid-way, so re-arm the whole control block
+                cudaMemsetAsync(c->d_ctrl, 0, sizeof(ControlBlock), stream);
                 return SO_ERR_TIMEOUT;
             }
         } else {
@@ -454,7 +449,7 @@ so_status so_layout_get_info(const so_ctx *c, so_layout_info *info)
                        (c->grad_dtype == SO_GRAD_BF16 ? 2u : 4u);
     info->bytes_param_bf16 = (uint64_t)c->n_buckets * (uint64_t)c->stride * 2u;
     const uint64_t partial_bytes = (uint64_t)c->n_buckets * (uint64_t)c->tiles_per_slot * 8u;
-    const uint64_t stats_bytes = (uint64_t)(c->n_buckets + 1) * sizeof(BucketStats);
+    const uint64_t stats_bytes = (uint64_t)c->n_buckets * sizeof(BucketStats) + sizeof(ControlBlock);
     info->bytes_scratch = (partial_bytes + 255u) / 256u * 256u + stats_bytes + 256u;
     return SO_OK;
 }
@@ -501,12 +496,11 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_cast, cast_params_kernel,
                                                           kThreads, 0);
         if (e != cudaSuccess) return cuda_fail(c, e);
-        e = allow_smem<ShapeDefault>();
-        if (e == cudaSuccess) e = allow_smem<ShapeA>();
-        if (e == cudaSuccess) e = allow_smem<ShapeB>();
-        if (e == cudaSuccess) e = allow_smem<ShapeC>();
-        if (e == cudaSuccess) e = allow_smem<ShapeD>();
-        if (e == cudaSuccess) e = allow_smem<ShapeE>();
+        e = allow_smem<uint16_t, ShapeBf16>();
+        if (e == cudaSuccess) e = allow_smem<float, ShapeFp32>();
+        if (e == cudaSuccess) e = allow_smem<uint16_t, ShapeAlt16>();
+        if (e == cudaSuccess) e = allow_smem<uint16_t, ShapeAlt12>();
+        if (e == cudaSuccess) e = allow_smem<float, ShapeAlt12>();
         if (e != cudaSuccess) return cuda_fail(c, e);
     } else {
         c->num_sms = 148;
@@ -532,10 +526,10 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
     const uint64_t partial_bytes = (uint64_t)c->n_buckets * (uint64_t)c->tiles_per_slot * 8u;
     c->d_stats = reinterpret_cast<BucketStats *>(static_cast<char *>(scratch) +
                                                  (partial_bytes + 255u) / 256u * 256u);
-    c->d_status = reinterpret_cast<int32_t *>(c->d_stats + c->n_buckets);
+    c->d_ctrl = reinterpret_cast<ControlBlock *>(c->d_stats + c->n_buckets);
     if (!c->dry_run) {
-        // the status record is the only part of scratch that must start at zero
-        const cudaError_t e = cudaMemset(c->d_status, 0, sizeof(BucketStats));
+        // the control block is the only part of scratch that must start at zero
+        const cudaError_t e = cudaMemset(c->d_ctrl, 0, sizeof(ControlBlock));
         if (e != cudaSuccess) return cuda_fail(c, e);
     }
     c->bound = true;
@@ -853,7 +847,7 @@ so_status so_debug_set_dry_run(so_ctx *c, int32_t on)
 
 so_status so_debug_set_step_variant(so_ctx *c, int32_t variant)
 {
-    if (!c || variant < 0 || variant > 14) return SO_ERR_INVALID_ARG;
+    if (!c || (variant != 0 && variant != 1 && variant != 10 && variant != 11)) return SO_ERR_INVALID_ARG;
     if (c->phase != kIdle) return SO_ERR_STATE;
     c->step_variant = variant;
     return SO_OK;

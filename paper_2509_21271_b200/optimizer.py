@@ -116,6 +116,30 @@ class BucketedAdamW:
             lo, hi = self.bucket_range(b)
             self._slot_view(self.grad, b, hi - lo).copy_(g[lo:hi], non_blocking=non_blocking)
 
+    def _scatter(self, arena: torch.Tensor, start: int, piece: torch.Tensor) -> None:
+        """Copy a piece of the flat space starting at `start` into bucket slots."""
+        Bk = self.info.bucket_elems
+        pos, end = start, start + piece.numel()
+        while pos < end:
+            b = pos // Bk
+            hi = min(end, (b + 1) * Bk)
+            slot = b if arena is self.grad or arena is self.param_bf16 \
+                else B.so_bucket_slot(self.ctx, b)
+            off = slot * self.info.slot_stride_elems + (pos - b * Bk)
+            arena[off:off + hi - pos].copy_(piece[pos - start:hi - start])
+            pos = hi
+
+    def load_state_stream(self, pieces) -> None:
+        """Master weights from an iterator of (start, fp32 piece); m and v are
+        left as they are (zero after construction)."""
+        for start, piece in pieces:
+            self._scatter(self.master, start, piece)
+
+    def load_grads_stream(self, pieces) -> None:
+        """Gradients from an iterator of (start, piece in the gradient dtype)."""
+        for start, piece in pieces:
+            self._scatter(self.grad, start, piece)
+
     def gather_state(self):
         """Flat (p, m, v) of the committed state, in parameter order."""
         N = self.info.total_elems

@@ -176,13 +176,23 @@ def _gen(device, seed: int) -> torch.Generator:
     return g
 
 
-def initial_master(w: Workload, device="cpu", chunk: int = 1 << 26) -> torch.Tensor:
-    """Flat fp32 master weights ~ N(0, sigma_p), seeded by the workload."""
-    out = torch.empty(w.total, dtype=torch.float32, device=device)
+def iter_initial_master(w: Workload, device="cpu", chunk: int = 1 << 26):
+    """Yields (start, fp32 tensor) pieces of the flat master weights in order.
+    The pieces are drawn from one generator, so the values do not depend on
+    who consumes them (a flat tensor or the slot arenas directly)."""
     gen = _gen(device, w.seed * 1_000_003 + 999_983)
     for s in range(0, w.total, chunk):
         e = min(s + chunk, w.total)
-        out[s:e].normal_(0.0, w.sigma_p, generator=gen)
+        z = torch.empty(e - s, dtype=torch.float32, device=device)
+        z.normal_(0.0, w.sigma_p, generator=gen)
+        yield s, z
+
+
+def initial_master(w: Workload, device="cpu", chunk: int = 1 << 26) -> torch.Tensor:
+    """Flat fp32 master weights ~ N(0, sigma_p), seeded by the workload."""
+    out = torch.empty(w.total, dtype=torch.float32, device=device)
+    for s, z in iter_initial_master(w, device, chunk):
+        out[s:s + z.numel()] = z
     return out
 
 
@@ -200,19 +210,19 @@ def faults_for_step(w: Workload, step: int) -> List[Fault]:
     return out
 
 
-def gradients(w: Workload, step: int, device="cpu", chunk: int = 1 << 26) -> torch.Tensor:
-    """Flat gradient of iteration ``step`` (1-based): bf16 or fp32 tensor.
+def iter_gradients(w: Workload, step: int, device="cpu", chunk: int = 1 << 26):
+    """Yields (start, tensor) pieces of the flat gradient of iteration ``step``
+    (1-based) in order, in the workload's gradient dtype.
 
     Drawn in fp32 ~ N(0, sigma_g); when the workload fixes a target global
     norm the draw is rescaled by ``target / ||draw||`` (double precision
     scalar) before the bf16 rounding; faults are written last.
     """
     dtype = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
-    out = torch.empty(w.total, dtype=dtype, device=device)
     gen = _gen(device, w.seed * 1_000_003 + step)
     scale = None
     if w.target_norm is not None:
-        # first pass: norm of the fp32 draw; second pass re-draws the same bits
+        # first pass: norm of the fp32 draw; the second pass re-draws the same bits
         acc = 0.0
         state = gen.get_state()
         for s in range(0, w.total, chunk):
@@ -222,15 +232,26 @@ def gradients(w: Workload, step: int, device="cpu", chunk: int = 1 << 26) -> tor
             acc += float(z.double().pow(2).sum().item())
         gen.set_state(state)
         scale = w.target_norm(step) / (acc ** 0.5)
+    faults = faults_for_step(w, step)
     for s in range(0, w.total, chunk):
         e = min(s + chunk, w.total)
         z = torch.empty(e - s, dtype=torch.float32, device=device)
         z.normal_(0.0, w.sigma_g, generator=gen)
         if scale is not None:
             z = (z.double() * scale).float()
-        out[s:e] = z.to(dtype)
-    for f in faults_for_step(w, step):
-        out[f.flat_index] = _fault_value(f.kind)
+        z = z.to(dtype)
+        for f in faults:
+            if s <= f.flat_index < e:
+                z[f.flat_index - s] = _fault_value(f.kind)
+        yield s, z
+
+
+def gradients(w: Workload, step: int, device="cpu", chunk: int = 1 << 26) -> torch.Tensor:
+    """Flat gradient of iteration ``step`` (1-based): bf16 or fp32 tensor."""
+    dtype = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
+    out = torch.empty(w.total, dtype=dtype, device=device)
+    for s, z in iter_gradients(w, step, device, chunk):
+        out[s:s + z.numel()] = z
     return out
 
 
