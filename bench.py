@@ -260,8 +260,11 @@ def main():
     # ---- device-resident timing ------------------------------------------
     for _ in range(args.warmup):
         one_step()
-    kernel_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                     for _ in range(args.steps)]
+    # the fused step kernel is timed on every 4th step of the timed region (an
+    # event pair costs a few microseconds of an iteration that lasts ~0.5 ms)
+    sampled = set(range(0, args.steps, 4))
+    kernel_events = {k: (torch.cuda.Event(enable_timing=True),
+                         torch.cuda.Event(enable_timing=True)) for k in sampled}
     launches0 = opt.counters().kernel_launches
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -272,7 +275,7 @@ def main():
     decisions = set()
     t_start.record(stream)
     for k in range(args.steps):
-        decisions.add(one_step(kernel_events[k]).decision)
+        decisions.add(one_step(kernel_events.get(k)).decision)
     t_end.record(stream)
     barrier()
     elapsed_ms = t_start.elapsed_time(t_end)
@@ -282,7 +285,7 @@ def main():
     spec_params = sum(opt.bucket_range(b)[1] - opt.bucket_range(b)[0] for b in range(spec_buckets))
     kernel_ms = None
     if not args.per_bucket:
-        times = [a.elapsed_time(b) for a, b in kernel_events]
+        times = [a.elapsed_time(b) for a, b in kernel_events.values()]
         kernel_ms = sum(times) / len(times)
 
     # ---- end to end through the host-buffer entry point -------------------
@@ -323,13 +326,13 @@ def main():
     roofline = None
     if kernel_ms:
         achieved = bpp * spec_params / (kernel_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": "adamw_step_kernel (fused speculative step+cast)",
+        roofline = {"bound": "hbm", "kernel": "adamw_step_tma_kernel (fused speculative AdamW step + bf16 cast + tile sums)",
                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}",
                     "unit": "GB/s", "frac": achieved / peak,
                     "traffic": (NCU_TRAFFIC_BYTES_PER_PARAM * spec_params
                                 if NCU_TRAFFIC_BYTES_PER_PARAM else None),
                     "bytes_per_param": bpp, "params_per_launch": spec_params,
-                    "kernel_ms": kernel_ms}
+                    "kernel_ms": kernel_ms, "launches_timed": len(kernel_events)}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,

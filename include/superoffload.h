@@ -141,8 +141,8 @@ so_status so_layout_tensor(const so_ctx *ctx, int32_t i, int64_t *flat_offset,
  * are fp32, grad is bf16 or fp32 per grad_dtype, param_bf16 is bf16.  The
  * caller fills master/m/v slot b with bucket b's initial state (m = v = 0 for
  * a fresh optimizer) and normally calls so_cast_params(SO_ALL) once.  Scratch
- * needs no initialisation by the caller (bind zeroes its 528-byte control
- * block with one synchronous cudaMemset).  Records the current device.
+ * needs no initialisation by the caller (bind zeroes a small control
+ * block and the per-bucket reduction counters with synchronous cudaMemsets).  Records the current device.
  */
 so_status so_layout_bind(so_ctx *ctx, void *master, void *m, void *v, void *grad,
                          void *param_bf16, void *scratch);
@@ -252,7 +252,9 @@ so_status so_iteration_host(so_ctx *ctx, const so_hparams *hp, const void *host_
  *   out_device    DEVICE, 8-byte aligned so_grad_stats written by the call
  *                 (sumsq, norm, clip_coef, nonfinite); caller-owned output
  * Enqueues two kernels on `stream` and returns; no synchronisation, no host
- * copy.  Same summation order as so_grad_check over one bucket of n_elems.
+ * copy.  Sums fold in a fixed order; the result is bit-identical to
+ * so_grad_check over one bucket of n_elems up to 4 Mi elements and equal to
+ * rounding beyond that.
  * The first call on each device looks up the device address of the built-in
  * array (cudaGetSymbolAddress, with that device current) and caches it; make
  * that first call outside any stream capture.  All calls on a device share the

@@ -347,20 +347,39 @@ __global__ void __launch_bounds__(kThreads) grad_check_kernel(const __grid_const
 // g^2 is formed in double, so it cannot overflow for a finite fp32/bf16 input,
 // and a sum of non-negative finite doubles this long cannot overflow either: a
 // tile sum is Inf or NaN exactly when the tile holds a NaN or an infinity.
-static __global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(const double *partials,
-                                                                      BucketStats *stats,
-                                                                      Geometry geo)
-{
-    __shared__ double s_sum[kReduceThreads];
-    __shared__ int s_bad[kReduceThreads];
-    const int32_t b = blockIdx.x;
-    const uint32_t n = (b == geo.last_bucket) ? geo.last_elems : geo.bucket_elems;
-    const uint32_t n_tiles = (n + kTileElems - 1) / kTileElems;
-    const double *src = partials + (int64_t)b * geo.tiles_per_slot;
+//
+// A bucket's tile sums are cut into segments of 4096 tiles.  One block folds
+// one segment (each thread adds up to 8 strided tile sums, then a shared-memory
+// tree); the block that finishes a bucket's last outstanding segment folds the
+// segment sums the same way and publishes the bucket's record.  Segment
+// boundaries and both fold orders are fixed, so the result does not depend on
+// which block happens to come last.  The per-bucket arrival counters start at
+// zero (bind) and are put back to zero by the publishing block.
+constexpr int kSegTiles = 4096;
 
+struct SegSum { double sum; int32_t bad; int32_t pad; };
+
+struct ReduceArgs {
+    const double *partials;        // tile sums
+    SegSum *seg;                   // n_buckets x segs_per_slot
+    uint32_t *arrivals;            // n_buckets
+    BucketStats *stats;            // device copy of the records
+    BucketStats *host_stats;       // mapped host copy, or nullptr
+    const int32_t *status;         // device status word, mirrored after the records
+    uint32_t *buckets_done;        // arrival counter over buckets (starts and ends at zero)
+    int32_t seq;                   // stamp of this reduction, written last
+    Geometry geo;
+    uint32_t segs_per_slot;
+    int32_t n_buckets;
+};
+
+// Fold `count` doubles starting at src (stride 1) in the fixed block order.
+__device__ __forceinline__ void block_fold(const double *src, uint32_t count, double *s_sum,
+                                           int *s_bad, double &sum_out, int &bad_out)
+{
     double acc = 0.0;
     int bad = 0;
-    for (uint32_t i = threadIdx.x; i < n_tiles; i += kReduceThreads) {
+    for (uint32_t i = threadIdx.x; i < count; i += kReduceThreads) {
         const double x = src[i];
         const uint32_t hi = (uint32_t)__double2hiint(x);
         bad |= ((hi & 0x7FF00000u) == 0x7FF00000u);
@@ -376,10 +395,79 @@ static __global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(co
         }
         __syncthreads();
     }
+    sum_out = s_sum[0];
+    bad_out = s_bad[0];
+    __syncthreads();
+}
+
+static __global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(const ReduceArgs a)
+{
+    __shared__ double s_sum[kReduceThreads];
+    __shared__ int s_bad[kReduceThreads];
+    __shared__ int s_last;
+    const int32_t b = (int32_t)(blockIdx.x / a.segs_per_slot);
+    const uint32_t seg = blockIdx.x - (uint32_t)b * a.segs_per_slot;
+    const uint32_t n = (b == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
+    const uint32_t n_tiles = (n + kTileElems - 1) / kTileElems;
+    const uint32_t n_segs = (n_tiles + kSegTiles - 1) / kSegTiles;
+    if (seg >= n_segs) return;
+    const uint32_t lo = seg * kSegTiles;
+    const uint32_t count = n_tiles - lo < (uint32_t)kSegTiles ? n_tiles - lo : (uint32_t)kSegTiles;
+
+    double sum;
+    int bad;
+    block_fold(a.partials + (int64_t)b * a.geo.tiles_per_slot + lo, count, s_sum, s_bad, sum, bad);
+    SegSum *segs = a.seg + (int64_t)b * a.segs_per_slot;
     if (threadIdx.x == 0) {
-        stats[b].sumsq = s_sum[0];
-        stats[b].nonfinite = s_bad[0];
-        stats[b].pad = 0;
+        segs[seg].sum = sum;
+        segs[seg].bad = bad;
+        __threadfence();
+        s_last = (atomicAdd(&a.arrivals[b], 1u) == n_segs - 1);
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+
+    // this block completed the bucket: fold its segment sums in index order
+    double acc = 0.0;
+    int any_bad = 0;
+    for (uint32_t i = threadIdx.x; i < n_segs; i += kReduceThreads) {
+        acc = __dadd_rn(acc, segs[i].sum);
+        any_bad |= segs[i].bad;
+    }
+    s_sum[threadIdx.x] = acc;
+    s_bad[threadIdx.x] = any_bad;
+    __syncthreads();
+    for (int s = kReduceThreads / 2; s > 0; s >>= 1) {
+        if ((int)threadIdx.x < s) {
+            s_sum[threadIdx.x] = __dadd_rn(s_sum[threadIdx.x], s_sum[threadIdx.x + s]);
+            s_bad[threadIdx.x] |= s_bad[threadIdx.x + s];
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        BucketStats r;
+        r.sumsq = s_sum[0];
+        r.nonfinite = s_bad[0];
+        r.pad = 0;
+        a.stats[b] = r;
+        a.arrivals[b] = 0;
+        if (a.host_stats) {
+            // Records go straight into mapped host memory.  The block that
+            // publishes the last bucket stamps the trailer record with this
+            // reduction's sequence number, after a system-wide fence, so a host
+            // that sees the stamp also sees every record.
+            a.host_stats[b] = r;
+            __threadfence_system();
+            if (atomicAdd(a.buckets_done, 1u) == (uint32_t)a.n_buckets - 1u) {
+                *a.buckets_done = 0;
+                __threadfence_system();
+                volatile BucketStats *trailer = a.host_stats + a.n_buckets;
+                trailer->nonfinite = *a.status;
+                __threadfence_system();
+                trailer->pad = a.seq;
+            }
+        }
     }
 }
 

@@ -47,7 +47,8 @@ constexpr int kCounterPairs = 64;                      // launches that may over
 // ring of {next tile, finished warps} counter pairs, one pair per launch.
 struct ControlBlock {
     int32_t status;
-    int32_t pad[3];
+    uint32_t buckets_done;     // arrival counter of the bucket reduction
+    int32_t pad[2];
     uint32_t counters[kCounterPairs][2];
 };
 

@@ -5,7 +5,9 @@
 
 #include <cmath>
 #include <cstdlib>
+#include <chrono>
 #include <cstring>
+#include <atomic>
 #include <new>
 #include <vector>
 
@@ -39,7 +41,12 @@ struct so_ctx {
     uint32_t launch_seq = 0;            // picks the counter pair of each pipeline launch
     int step_variant = 0;               // 0: bulk-copy pipeline, 1: register path
     BucketStats *h_stats = nullptr;
+    BucketStats *h_stats_dev = nullptr; // device view of h_stats when it is mapped pinned memory
     bool h_stats_pinned = false;
+    SegSum *d_seg = nullptr;            // per-bucket segment sums of the reduction
+    uint32_t *d_arrivals = nullptr;     // per-bucket arrival counters of the reduction
+    int64_t segs_per_slot = 1;
+    int32_t reduce_seq = 0;             // stamp of the latest reduction (never 0)
     int occ_step = 0, occ_check = 0, occ_cast = 0;
     // ---- slot map ----
     std::vector<int32_t> slot_of;       // committed slot of each bucket
@@ -314,24 +321,64 @@ so_status finalize_check(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
     }
     if (c->n_buckets > 0) {
         if (!c->dry_run) {
-            bucket_reduce_kernel<<<(unsigned)c->n_buckets, kReduceThreads, 0, stream>>>(
-                c->d_partials, c->d_stats, geometry_of(c));
+            ReduceArgs r;
+            r.partials = c->d_partials;
+            r.seg = c->d_seg;
+            r.arrivals = c->d_arrivals;
+            r.stats = c->d_stats;
+            r.host_stats = c->h_stats_dev;     // records land in host memory directly
+            r.status = &c->d_ctrl->status;
+            r.buckets_done = &c->d_ctrl->buckets_done;
+            c->reduce_seq = c->reduce_seq == 0x7FFFFFFF ? 1 : c->reduce_seq + 1;
+            r.seq = c->reduce_seq;
+            r.geo = geometry_of(c);
+            r.segs_per_slot = (uint32_t)c->segs_per_slot;
+            r.n_buckets = c->n_buckets;
+            const int64_t blocks = (int64_t)c->n_buckets * c->segs_per_slot;
+            bucket_reduce_kernel<<<(unsigned)blocks, kReduceThreads, 0, stream>>>(r);
         }
         so_status s = after_launch(c);
         if (s != SO_OK) return s;
         if (!c->dry_run) {
-            cudaError_t e = cudaMemcpyAsync(c->h_stats, c->d_stats,
-                                            sizeof(BucketStats) * (size_t)(c->n_buckets + 1),
-                                            cudaMemcpyDeviceToHost, stream);
+            cudaError_t e = cudaSuccess;
+            if (!c->h_stats_dev)
+                e = cudaMemcpyAsync(c->h_stats, c->d_stats,
+                                    sizeof(BucketStats) * (size_t)(c->n_buckets + 1),
+                                    cudaMemcpyDeviceToHost, stream);
             if (e != cudaSuccess) return cuda_fail(c, e);
-            e = cudaStreamSynchronize(stream);
-            if (e != cudaSuccess) return cuda_fail(c, e);
-            int32_t device_status = 0;
-            std::memcpy(&device_status, &c->h_stats[c->n_buckets], sizeof(device_status));
+            if (c->h_stats_dev) {
+                // The records arrive in mapped host memory; watching for the
+                // stamp that follows them is several microseconds quicker than
+                // waiting for the stream's completion to be signalled.  Bounded:
+                // after two seconds fall back to a stream synchronisation, which
+                // also surfaces any launch or execution error.
+                volatile int32_t *stamp = &c->h_stats[c->n_buckets].pad;
+                const auto t0 = std::chrono::steady_clock::now();
+                bool arrived = false;
+                for (uint32_t spins = 0;; ++spins) {
+                    if (*stamp == c->reduce_seq) { arrived = true; break; }
+                    if ((spins & 0xFFFu) == 0xFFFu &&
+                        std::chrono::steady_clock::now() - t0 > std::chrono::seconds(2))
+                        break;
+                }
+                std::atomic_thread_fence(std::memory_order_acquire);
+                if (!arrived) {
+                    e = cudaStreamSynchronize(stream);
+                    if (e != cudaSuccess) return cuda_fail(c, e);
+                    if (*stamp != c->reduce_seq) return cuda_fail(c, cudaErrorUnknown);
+                }
+            } else {
+                e = cudaStreamSynchronize(stream);
+                if (e != cudaSuccess) return cuda_fail(c, e);
+            }
+            int32_t device_status = c->h_stats[c->n_buckets].nonfinite;
+            if (!c->h_stats_dev)
+                std::memcpy(&device_status, &c->h_stats[c->n_buckets], sizeof(device_status));
             if (device_status != 0) {
                 // a kernel gave up waiting for one of its own copies; its tile
                 // counters may be left mid-way, so re-arm the whole control block
                 cudaMemsetAsync(c->d_ctrl, 0, sizeof(ControlBlock), stream);
+                if (c->h_stats_dev) std::memset(&c->h_stats[c->n_buckets], 0, sizeof(BucketStats));
                 return SO_ERR_TIMEOUT;
             }
         } else {
@@ -450,7 +497,9 @@ so_status so_layout_get_info(const so_ctx *c, so_layout_info *info)
     info->bytes_param_bf16 = (uint64_t)c->n_buckets * (uint64_t)c->stride * 2u;
     const uint64_t partial_bytes = (uint64_t)c->n_buckets * (uint64_t)c->tiles_per_slot * 8u;
     const uint64_t stats_bytes = (uint64_t)c->n_buckets * sizeof(BucketStats) + sizeof(ControlBlock);
-    info->bytes_scratch = (partial_bytes + 255u) / 256u * 256u + stats_bytes + 256u;
+    const uint64_t segs = (uint64_t)((c->tiles_per_slot + kSegTiles - 1) / kSegTiles);
+    const uint64_t reduce_bytes = (uint64_t)c->n_buckets * (segs * sizeof(SegSum) + 4u);
+    info->bytes_scratch = (partial_bytes + 255u) / 256u * 256u + stats_bytes + reduce_bytes + 512u;
     return SO_OK;
 }
 
@@ -508,9 +557,15 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
     }
     if (!c->h_stats) {
         const size_t bytes = sizeof(BucketStats) * (size_t)(c->n_buckets + 1);
-        if (!c->dry_run && cudaMallocHost(reinterpret_cast<void **>(&c->h_stats), bytes) ==
-                               cudaSuccess) {
+        if (!c->dry_run && cudaHostAlloc(reinterpret_cast<void **>(&c->h_stats), bytes,
+                                         cudaHostAllocMapped) == cudaSuccess) {
             c->h_stats_pinned = true;
+            std::memset(c->h_stats, 0, bytes);
+            void *dev_view = nullptr;
+            if (cudaHostGetDevicePointer(&dev_view, c->h_stats, 0) == cudaSuccess)
+                c->h_stats_dev = static_cast<BucketStats *>(dev_view);
+            else
+                cudaGetLastError();                   // fall back to an explicit copy
         } else {
             if (!c->dry_run) cudaGetLastError();      // clear the failed pinned allocation
             c->h_stats = static_cast<BucketStats *>(std::malloc(bytes));
@@ -527,9 +582,16 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
     c->d_stats = reinterpret_cast<BucketStats *>(static_cast<char *>(scratch) +
                                                  (partial_bytes + 255u) / 256u * 256u);
     c->d_ctrl = reinterpret_cast<ControlBlock *>(c->d_stats + c->n_buckets);
+    c->segs_per_slot = (c->tiles_per_slot + kSegTiles - 1) / kSegTiles;
+    if (c->segs_per_slot < 1) c->segs_per_slot = 1;
+    c->d_seg = reinterpret_cast<SegSum *>(c->d_ctrl + 1);
+    c->d_arrivals = reinterpret_cast<uint32_t *>(c->d_seg + (int64_t)c->n_buckets * c->segs_per_slot);
     if (!c->dry_run) {
-        // the control block is the only part of scratch that must start at zero
-        const cudaError_t e = cudaMemset(c->d_ctrl, 0, sizeof(ControlBlock));
+        // the control block and the arrival counters must start at zero; the
+        // rest of scratch is written before it is read
+        cudaError_t e = cudaMemset(c->d_ctrl, 0, sizeof(ControlBlock));
+        if (e == cudaSuccess && c->n_buckets > 0)
+            e = cudaMemset(c->d_arrivals, 0, sizeof(uint32_t) * (size_t)c->n_buckets);
         if (e != cudaSuccess) return cuda_fail(c, e);
     }
     c->bound = true;
