@@ -452,22 +452,33 @@ static __global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(co
         r.pad = 0;
         a.stats[b] = r;
         a.arrivals[b] = 0;
+        s_last = 0;
         if (a.host_stats) {
-            // Records go straight into mapped host memory.  The block that
-            // publishes the last bucket stamps the trailer record with this
-            // reduction's sequence number, after a system-wide fence, so a host
-            // that sees the stamp also sees every record.
-            a.host_stats[b] = r;
-            __threadfence_system();
-            if (atomicAdd(a.buckets_done, 1u) == (uint32_t)a.n_buckets - 1u) {
-                *a.buckets_done = 0;
-                __threadfence_system();
-                volatile BucketStats *trailer = a.host_stats + a.n_buckets;
-                trailer->nonfinite = *a.status;
-                __threadfence_system();
-                trailer->pad = a.seq;
-            }
+            __threadfence();
+            s_last = (atomicAdd(a.buckets_done, 1u) == (uint32_t)a.n_buckets - 1u);
         }
+    }
+    __syncthreads();
+    if (!s_last) return;
+
+    // This block published the last bucket.  It alone writes to the mapped
+    // host copy: all records, one system-wide fence, then the stamp -- a host
+    // that sees the stamp therefore sees every record, and the kernel pays for
+    // two trips to host memory instead of one per bucket.
+    __threadfence();
+    for (int32_t i = threadIdx.x; i < a.n_buckets; i += kReduceThreads) {
+        // records of other blocks: read them from L2, not from a stale L1 line
+        const int4 rec = __ldcg(reinterpret_cast<const int4 *>(a.stats + i));
+        *reinterpret_cast<int4 *>(a.host_stats + i) = rec;
+    }
+    __threadfence_system();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        *a.buckets_done = 0;
+        volatile BucketStats *trailer = a.host_stats + a.n_buckets;
+        trailer->nonfinite = *a.status;
+        __threadfence_system();
+        trailer->pad = a.seq;
     }
 }
 
