@@ -141,3 +141,93 @@ def run_lockstep(w: W.Workload, steps: int, undo_slots: int = B.SO_ALL,
     if guard_bands:
         assert opt.guard_bands_intact(), "a kernel wrote outside its arena"
     return rep, opt
+
+
+# ---------------------------------------------------------------------------
+# sampled parity for workloads too large to replay in full on the host
+# ---------------------------------------------------------------------------
+
+def _bucket_grads_numpy(opt: BucketedAdamW, b: int) -> np.ndarray:
+    lo, hi = opt.bucket_range(b)
+    g = opt._slot_view(opt.grad, b, hi - lo)
+    return grads_to_numpy(g)
+
+
+def _bucket_state_numpy(opt: BucketedAdamW, b: int):
+    p, m, v, pb = opt.gather_bucket(b)
+    return [p.cpu().numpy(), m.cpu().numpy(), v.cpu().numpy()], bf16_to_numpy(pb)
+
+
+def run_sampled(w: W.Workload, steps: int, pick_buckets, undo_slots: int = B.SO_ALL,
+                expect_decisions=None):
+    """Parity on a large workload: norm, coefficient, flag and decision are
+    checked on every step against the oracle streamed over all gradients
+    (bucket by bucket, bucket order); element results are checked in lock-step
+    on the buckets `pick_buckets(step)` names, from the device's own pre-step
+    state, with the device's coefficient on a clip re-step."""
+    hp = hparams_of(w)
+    stream = torch.cuda.current_stream()
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, undo_slots)
+    opt.load_state_stream(W.iter_initial_master(w, device="cuda"))
+    opt.cast_params(stream=stream)
+    torch.cuda.synchronize()
+    rep = Report()
+    t = 0
+    for step in range(1, steps + 1):
+        opt.load_grads_stream(W.iter_gradients(w, step, device="cuda"))
+        buckets = sorted(set(pick_buckets(step)))
+        pre = {b: _bucket_state_numpy(opt, b) for b in buckets}
+        for b in buckets:                 # step boundary invariant: bf16 copy == RNE(master)
+            assert np.array_equal(pre[b][1], oracle.bf16_rne(pre[b][0][0]))
+        res = opt.iteration(hp, stream=stream)
+        torch.cuda.synchronize()
+
+        total, flag = 0.0, 0
+        for b in range(opt.n_buckets):
+            gb = _bucket_grads_numpy(opt, b)
+            s, f = oracle.grad_check_range(gb, 0, gb.size)
+            total += s
+            flag |= f
+        norm = float(np.sqrt(np.float64(total)))
+        own_coef = oracle.clip_coef(norm, hp.max_grad_norm)
+        own_decision = oracle.decision(flag, own_coef)
+        assert res.decision == own_decision, (step, res.decision, own_decision)
+        orc_res = oracle.IterationResult(own_decision, total, norm, own_coef, flag, 0)
+        check_stats(res.stats, orc_res, hp.max_grad_norm, rep)
+        rep.decisions.append(res.decision)
+
+        for b in buckets:
+            (p, m, v), pb = pre[b]
+            gb = _bucket_grads_numpy(opt, b)
+            if res.decision != B.SO_DECISION_SKIP:
+                scale = res.stats.clip_coef if res.decision == B.SO_DECISION_CLIP_RESTEP else 1.0
+                oracle.adamw_step_range(p, m, v, gb, 0, p.size, scale, t + 1, hp)
+                pb = oracle.bf16_rne(p)
+            dev, pb_dev = _bucket_state_numpy(opt, b)
+            compare_state(dev, (p, m, v), rep)
+            assert_bf16_consistent(pb_dev, dev[0], pb, p, rep)
+            if res.decision == B.SO_DECISION_SKIP:
+                for a_, b_ in zip(dev, (p, m, v)):
+                    assert a_.tobytes() == b_.tobytes()
+        if res.decision != B.SO_DECISION_SKIP:
+            t += 1
+        assert res.step_after == t == opt.step_count
+    if expect_decisions is not None:
+        assert rep.decisions == expect_decisions, rep.decisions
+    return rep, opt
+
+
+def write_report(name: str, rep: Report, extra: dict | None = None) -> None:
+    """Leave the parity maxima where a results table can pick them up."""
+    import json
+    import os
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out_dir = os.path.join(root, "gpurun_out")
+    if not os.path.isdir(out_dir):
+        return
+    rec = {"workload": name, "decisions": rep.decisions, "max_ulp": rep.max_ulp,
+           "n_diff": rep.n_diff, "n_elems_compared": rep.n_elems,
+           "max_norm_rel": rep.max_norm_rel, "bf16_mismatch": rep.bf16_mismatch}
+    rec.update(extra or {})
+    with open(os.path.join(out_dir, f"parity_{name}.json"), "w") as fh:
+        json.dump(rec, fh)

@@ -1,0 +1,111 @@
+"""GPU parity at the full sizes of the paper-shaped workloads (the launch
+configurations bench.py times), on sampled buckets: norm, coefficient, flags
+and decisions on every step; element results in lock-step on named buckets."""
+from __future__ import annotations
+
+import pytest
+import torch
+
+from gpu_harness import run_lockstep, run_sampled, write_report
+from paper_2509_21271_b200 import binding as B
+from paper_2509_21271_b200 import build as so_build
+from paper_2509_21271_b200 import workloads as W
+
+import os
+
+pytestmark = [pytest.mark.gpu,
+              pytest.mark.skipif(os.environ.get("SO_SKIP_FULL_SIZE") == "1",
+                                 reason="full-size workloads skipped on request")]
+
+C, S, R = B.SO_DECISION_COMMIT, B.SO_DECISION_SKIP, B.SO_DECISION_CLIP_RESTEP
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    so_build.build_library()
+    torch.cuda.set_device(0)
+
+
+@pytest.fixture(autouse=True)
+def _release_device_memory():
+    """These workloads take most of the GPU: drop whatever the previous test
+    left in torch's caching allocator before sizing the next one."""
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    yield
+    gc.collect()
+    torch.cuda.empty_cache()
+
+
+def _undo_that_fits(w: W.Workload) -> int:
+    stride = (w.bucket_elems + 63) // 64 * 64
+    free_bytes, _ = torch.cuda.mem_get_info()
+    gsz = 2 if w.grad_dtype == "bf16" else 4
+    resident = w.n_buckets * stride * (12 + gsz + 2)
+    room = free_bytes - resident - (8 << 30)
+    assert room > 0, "workload does not fit on this GPU"
+    return int(max(0, min(w.n_buckets, room // (12 * stride))))
+
+
+def test_tiny_and_gpt2_reports():
+    """Config 1 and 2b in full, leaving their parity maxima for the results table."""
+    rep, _ = run_lockstep(W.tiny(), steps=10)
+    write_report("tiny", rep)
+    rep, _ = run_lockstep(W.gpt2_small(clip=False), steps=2, guard_bands=False)
+    write_report("gpt2_small", rep)
+
+
+def test_llama_1b_alternating_clip_and_nan():
+    """1.24 B parameters in 100 M-element buckets; the global norm alternates
+    0.5 / 3.0 (clip active on even steps) and a NaN lands every 4th step here
+    (every 50th in the long-running recipe), where the skip must win over the clip."""
+    w = W.llama_1b()
+    w.nan_every = 4
+    torch.manual_seed(0)
+    nb = w.n_buckets
+    picks = {1: [0, nb - 1], 2: [5, nb - 1], 3: [12], 4: [3], 5: [7], 6: [nb - 1]}
+    rep, opt = run_sampled(w, steps=6, pick_buckets=lambda s: picks[s],
+                           expect_decisions=[C, R, C, S, C, R])
+    assert opt.step_count == 5
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+    write_report("llama_1b", rep)
+    opt.close()
+    del opt
+
+
+def test_llama_8b_windowed_undo():
+    """8.03 B parameters (128.5 GB resident) in 200 M-element buckets: only part
+    of the buckets can be stepped speculatively, the rest are scanned and
+    stepped in place inside validation; every step commits."""
+    w = W.llama_8b()
+    undo = _undo_that_fits(w)
+    assert 0 < undo < w.n_buckets
+    nb = w.n_buckets
+    picks = {1: [0, undo - 1, undo, nb - 1], 2: [1, undo + 1, nb - 1]}
+    rep, opt = run_sampled(w, steps=2, pick_buckets=lambda s: picks[s], undo_slots=undo,
+                           expect_decisions=[C, C])
+    c = opt.counters()
+    assert c.elems_checked == 2 * sum(opt.bucket_range(b)[1] - opt.bucket_range(b)[0]
+                                      for b in range(undo, nb))
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+    write_report("llama_8b", rep, {"undo_slots": undo})
+    opt.close()
+    del opt
+
+
+@pytest.mark.parametrize("grad_dtype", ["bf16", "fp32"])
+@pytest.mark.parametrize("bucket_mi", [1, 16, 64, 256, 512])
+def test_sweep_one_bucket_per_combination(bucket_mi, grad_dtype):
+    """The bucket-size sweep on a 4 Gi-element flat buffer: one seeded bucket
+    per (bucket size, gradient dtype) pair, first step."""
+    w = W.sweep(bucket_mi, grad_dtype)
+    undo = _undo_that_fits(w)
+    nb = w.n_buckets
+    pick = [(7 * bucket_mi + 3) % min(nb, max(undo, 1))]
+    rep, opt = run_sampled(w, steps=1, pick_buckets=lambda s: pick, undo_slots=undo,
+                           expect_decisions=[C])
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+    write_report(w.name, rep, {"undo_slots": undo})
+    opt.close()
+    del opt
