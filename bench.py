@@ -34,8 +34,10 @@ UNIT = "params/s"
 BYTES_PER_PARAM = {"bf16": 28, "fp32": 30}      # algorithmic HBM bytes of the fused step
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per parameter of the fused step
-# kernel, from the ncu capture summarised under profiles/ (None until measured)
-NCU_TRAFFIC_BYTES_PER_PARAM = None
+# kernel (gpt2_small capture: 1.742 GB read + 1.688 GB written per launch of
+# 124 439 808 parameters; profiles/adamw_step_tma_kernel_gpt2_small.md), scaled
+# to the launch by the parameters it processes (traffic is proportional)
+NCU_TRAFFIC_BYTES_PER_PARAM = 27.57
 
 
 def _measured_peak():
