@@ -18,8 +18,8 @@
  *     so_destroy frees only that.  Device pointers must be 256-byte aligned.
  *   - `stream` arguments are cudaStream_t values passed as void* (NULL = the
  *     legacy default stream).  Calls that launch work enqueue it and return;
- *     only calls that fill a host struct from device results synchronise that
- *     stream (stated per function).
+ *     only calls that fill a host struct from device results wait for the
+ *     device (stated per function).
  *   - The device that is current when so_layout_bind is called must be current
  *     for every later call on that context.  A context is not thread-safe;
  *     separate contexts are independent.
@@ -156,7 +156,9 @@ so_status so_layout_bind(so_ctx *ctx, void *master, void *m, void *v, void *grad
  *   bucket == SO_ALL : scan every bucket not yet covered this iteration, reduce
  *                 per bucket and over buckets, and fill `out` (host, may be
  *                 NULL) with sumsq, norm, clip coefficient for
- *                 hp->max_grad_norm, and the flag.  Synchronises `stream`.
+ *                 hp->max_grad_norm, and the flag.  Blocks until the reduction's
+ *                 results have reached the host (everything enqueued on
+ *                 `stream` before this call has completed by then).
  * The reduction order is fixed (independent of grid size and of whether the
  * scan ran inside the fused step), so results repeat bit for bit.
  */
@@ -188,7 +190,7 @@ so_status so_adam_step_speculative(so_ctx *ctx, const so_hparams *hp, int32_t bu
  * validation, either keep the speculative update, skip the iteration when a
  * NaN/Inf was found, or revert it and re-execute with clipped gradients).
  * Completes the gradient check if so_grad_check(SO_ALL) has not run
- * (synchronises `stream`), then
+ * (blocks until its results have reached the host), then
  *   nonfinite          -> SKIP: speculative slots are dropped, the bf16 copy of
  *                         those buckets is re-derived from the untouched master,
  *                         the step count does not advance;

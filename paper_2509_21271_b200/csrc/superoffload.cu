@@ -306,8 +306,8 @@ so_status launch_casts(so_ctx *c, const std::vector<BucketEntry> &entries, cudaS
 }
 
 // Finish the gradient check: scan what is still uncovered, fold per bucket on
-// the device, bring the per-bucket results to the host, fold over buckets in
-// index order, derive norm and clip coefficient.  Synchronises the stream.
+// the device, wait for the per-bucket records to reach the host, fold over
+// buckets in index order, derive norm and clip coefficient.
 so_status finalize_check(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
 {
     std::vector<int32_t> todo;
