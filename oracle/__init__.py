@@ -22,7 +22,7 @@ _SRC = os.path.join(_HERE, "so_oracle.c")
 _LIB = os.path.join(_HERE, "liboracle.so")
 
 DECISION_COMMIT, DECISION_SKIP, DECISION_CLIP_RESTEP = 0, 1, 2
-GRAD_BF16, GRAD_FP32 = 0, 1
+GRAD_BF16, GRAD_FP32, GRAD_FP16 = 0, 1, 2
 
 
 def build(force: bool = False) -> str:
@@ -51,27 +51,31 @@ def _load():
     pd, pi, pi64 = c.POINTER(c.c_double), c.POINTER(c.c_int), c.POINTER(c.c_int64)
     lib.orc_widen_bf16.restype = None
     lib.orc_widen_bf16.argtypes = [vp, vp, i64]
+    lib.orc_widen_fp16.restype = None
+    lib.orc_widen_fp16.argtypes = [vp, vp, i64]
+    lib.orc_loss_scale_update.restype = None
+    lib.orc_loss_scale_update.argtypes = [pd, pi64, c.c_int, dbl, dbl, i64]
     lib.orc_bf16_rne.restype = c.c_uint16
     lib.orc_bf16_rne.argtypes = [c.c_float]
     lib.orc_cast_params.restype = None
     lib.orc_cast_params.argtypes = [vp, vp, i64]
     lib.orc_grad_check_range.restype = c.c_int
-    lib.orc_grad_check_range.argtypes = [vp, c.c_int, i64, i64, pd]
+    lib.orc_grad_check_range.argtypes = [vp, c.c_int, i64, i64, dbl, pd]
     lib.orc_global_grad_check.restype = c.c_int
-    lib.orc_global_grad_check.argtypes = [vp, c.c_int, i64, i64, pd, pd]
+    lib.orc_global_grad_check.argtypes = [vp, c.c_int, i64, i64, dbl, pd, pd]
     lib.orc_clip_coef.restype = dbl
     lib.orc_clip_coef.argtypes = [dbl, dbl]
     lib.orc_decision.restype = c.c_int
     lib.orc_decision.argtypes = [c.c_int, dbl]
     lib.orc_adamw_step_range.restype = None
-    lib.orc_adamw_step_range.argtypes = [vp, vp, vp, vp, c.c_int, i64, i64, dbl, i64,
+    lib.orc_adamw_step_range.argtypes = [vp, vp, vp, vp, c.c_int, i64, i64, dbl, dbl, i64,
                                          dbl, dbl, dbl, dbl, dbl]
     lib.orc_iteration_ste.restype = c.c_int
     lib.orc_iteration_ste.argtypes = [vp, vp, vp, vp, vp, c.c_int, i64, i64, pi64,
-                                      dbl, dbl, dbl, dbl, dbl, dbl, pd, pd, pd, pi]
+                                      dbl, dbl, dbl, dbl, dbl, dbl, dbl, pd, pd, pd, pi]
     lib.orc_iteration_stv.restype = c.c_int
     lib.orc_iteration_stv.argtypes = [vp, vp, vp, vp, vp, c.c_int, i64, i64, pi64,
-                                      dbl, dbl, dbl, dbl, dbl, dbl, dbl, pd, pd, pd, pi]
+                                      dbl, dbl, dbl, dbl, dbl, dbl, dbl, dbl, pd, pd, pd, pi]
     lib.orc_layout_offsets.restype = i64
     lib.orc_layout_offsets.argtypes = [pi64, i32, pi64]
     lib.orc_num_buckets.restype = i64
@@ -118,7 +122,9 @@ def _grad_dtype(g: np.ndarray) -> int:
         return GRAD_BF16
     if g.dtype == np.float32:
         return GRAD_FP32
-    raise TypeError("gradients must be uint16 (bf16 bit patterns) or float32")
+    if g.dtype == np.float16:
+        return GRAD_FP16
+    raise TypeError("gradients must be uint16 (bf16 bit patterns), float16 or float32")
 
 
 def bf16_rne(x: np.ndarray) -> np.ndarray:
@@ -137,19 +143,37 @@ def bf16_to_f32(b: np.ndarray) -> np.ndarray:
     return out
 
 
-def grad_check_range(g: np.ndarray, begin: int, end: int):
-    """(sum of squares in index order, non-finite flag) of g[begin:end]."""
+def fp16_to_f32(h: np.ndarray) -> np.ndarray:
+    """IEEE binary16 bit patterns (uint16) -> fp32, exact."""
+    h = _check(np.ascontiguousarray(h), np.uint16)
+    out = np.empty(h.shape, dtype=np.float32)
+    _load().orc_widen_fp16(_ptr(h), _ptr(out), h.size)
+    return out
+
+
+def grad_check_range(g: np.ndarray, begin: int, end: int, unscale: float = 1.0):
+    """(sum of squares in index order, non-finite flag) of unscale * g[begin:end]."""
     s = ctypes.c_double()
-    flag = _load().orc_grad_check_range(_ptr(g), _grad_dtype(g), begin, end, ctypes.byref(s))
+    flag = _load().orc_grad_check_range(_ptr(g), _grad_dtype(g), begin, end, unscale,
+                                        ctypes.byref(s))
     return s.value, int(flag)
 
 
-def global_grad_check(g: np.ndarray, bucket_elems: int):
-    """(sumsq, norm, nonfinite) over all of g, bucket partials in bucket order."""
+def global_grad_check(g: np.ndarray, bucket_elems: int, unscale: float = 1.0):
+    """(sumsq, norm, nonfinite) over all of unscale * g, bucket partials in bucket order."""
     s, nrm = ctypes.c_double(), ctypes.c_double()
-    flag = _load().orc_global_grad_check(_ptr(g), _grad_dtype(g), g.size, bucket_elems,
+    flag = _load().orc_global_grad_check(_ptr(g), _grad_dtype(g), g.size, bucket_elems, unscale,
                                          ctypes.byref(s), ctypes.byref(nrm))
     return s.value, nrm.value, int(flag)
+
+
+def loss_scale_update(scale: float, good_steps: int, nonfinite: int, growth: float = 2.0,
+                      backoff: float = 0.5, interval: int = 2000):
+    """One step of the dynamic loss-scale schedule: returns (scale, good_steps)."""
+    s, gcount = ctypes.c_double(scale), ctypes.c_int64(good_steps)
+    _load().orc_loss_scale_update(ctypes.byref(s), ctypes.byref(gcount), int(nonfinite),
+                                  growth, backoff, interval)
+    return s.value, gcount.value
 
 
 def clip_coef(norm: float, max_norm: float) -> float:
@@ -160,16 +184,17 @@ def decision(nonfinite: int, coef: float) -> int:
     return _load().orc_decision(int(nonfinite), coef)
 
 
-def adamw_step_range(p, m, v, g, begin, end, scale, tt, hp: HParams) -> None:
+def adamw_step_range(p, m, v, g, begin, end, scale, tt, hp: HParams,
+                     unscale: float = 1.0) -> None:
     """In-place AdamW step of elements [begin, end) with step index ``tt``."""
     for a in (p, m, v):
         _check(a, np.float32)
     _load().orc_adamw_step_range(_ptr(p), _ptr(m), _ptr(v), _ptr(g), _grad_dtype(g),
-                                 begin, end, scale, tt, hp.lr, hp.beta1, hp.beta2,
+                                 begin, end, unscale, scale, tt, hp.lr, hp.beta1, hp.beta2,
                                  hp.eps, hp.weight_decay)
 
 
-def _iteration(fn_name, p, m, v, pb, g, bucket_elems, t, hp, forced_coef=None):
+def _iteration(fn_name, p, m, v, pb, g, bucket_elems, t, hp, forced_coef=None, unscale=1.0):
     for a in (p, m, v):
         _check(a, np.float32)
     _check(pb, np.uint16)
@@ -179,7 +204,7 @@ def _iteration(fn_name, p, m, v, pb, g, bucket_elems, t, hp, forced_coef=None):
     flag = ctypes.c_int()
     args = [_ptr(p), _ptr(m), _ptr(v), _ptr(pb), _ptr(g), _grad_dtype(g), p.size,
             bucket_elems, ctypes.byref(tt), hp.lr, hp.beta1, hp.beta2, hp.eps,
-            hp.weight_decay, hp.max_grad_norm]
+            hp.weight_decay, hp.max_grad_norm, float(unscale)]
     if fn_name == "orc_iteration_stv":
         args.append(0.0 if forced_coef is None else float(forced_coef))
     args += [ctypes.byref(s), ctypes.byref(nrm), ctypes.byref(coef), ctypes.byref(flag)]
@@ -189,15 +214,17 @@ def _iteration(fn_name, p, m, v, pb, g, bucket_elems, t, hp, forced_coef=None):
     return IterationResult(d, s.value, nrm.value, coef.value, flag.value, tt.value)
 
 
-def iteration_ste(p, m, v, pb, g, bucket_elems: int, t: int, hp: HParams) -> IterationResult:
+def iteration_ste(p, m, v, pb, g, bucket_elems: int, t: int, hp: HParams,
+                  unscale: float = 1.0) -> IterationResult:
     """Check every gradient, then step (or skip): the plain definition."""
-    return _iteration("orc_iteration_ste", p, m, v, pb, g, bucket_elems, t, hp)
+    return _iteration("orc_iteration_ste", p, m, v, pb, g, bucket_elems, t, hp, None, unscale)
 
 
 def iteration_stv(p, m, v, pb, g, bucket_elems: int, t: int, hp: HParams,
-                  forced_coef: float | None = None) -> IterationResult:
+                  forced_coef: float | None = None, unscale: float = 1.0) -> IterationResult:
     """Speculate every bucket, validate, then commit / restore / re-step."""
-    return _iteration("orc_iteration_stv", p, m, v, pb, g, bucket_elems, t, hp, forced_coef)
+    return _iteration("orc_iteration_stv", p, m, v, pb, g, bucket_elems, t, hp, forced_coef,
+                      unscale)
 
 
 def layout_offsets(numel):

@@ -12,7 +12,9 @@
  *     -ffp-contract=off so that no multiply-add is fused;
  *   - state is stored as fp32 (master weight p, first moment m, second moment
  *     v) and rounded to nearest-even after every step, denormals kept;
- *   - gradients arrive as bf16 bit patterns (uint16_t) or as fp32;
+ *   - gradients arrive as bf16 bit patterns (uint16_t), as fp32, or as IEEE
+ *     binary16 bit patterns (the paper's own FP16 path), the latter normally
+ *     multiplied by a loss scale that `unscale` = 1/scale takes out again;
  *   - a "bucket" is the contiguous flat range [b*B, min((b+1)*B, N)).
  *
  * What follows which passage of the paper
@@ -36,7 +38,7 @@
 #include <string.h>
 
 enum { ORC_DECISION_COMMIT = 0, ORC_DECISION_SKIP = 1, ORC_DECISION_CLIP_RESTEP = 2 };
-enum { ORC_GRAD_BF16 = 0, ORC_GRAD_FP32 = 1 };
+enum { ORC_GRAD_BF16 = 0, ORC_GRAD_FP32 = 1, ORC_GRAD_FP16 = 2 };
 
 /* ---- bit views ---------------------------------------------------------- */
 
@@ -49,6 +51,29 @@ float orc_bf16_to_f32(uint16_t b) { return bits_f32((uint32_t)b << 16); }
 void orc_widen_bf16(const uint16_t *b, float *out, int64_t n)
 {
     for (int64_t i = 0; i < n; ++i) out[i] = orc_bf16_to_f32(b[i]);
+}
+
+/*
+ * IEEE binary16 -> fp32 (exact): 1 sign, 5 exponent (bias 15), 10 mantissa
+ * bits; exponent 0 is zero or a subnormal (mantissa * 2^-24), exponent 31 is
+ * infinity (mantissa 0) or NaN.  This is the gradient format of the paper's
+ * mixed-precision runs (Section 4.5).
+ */
+float orc_fp16_to_f32(uint16_t h)
+{
+    const int sign = (h >> 15) & 1;
+    const int exponent = (h >> 10) & 0x1F;
+    const int mantissa = h & 0x3FF;
+    double v;
+    if (exponent == 0) v = ldexp((double)mantissa, -24);
+    else if (exponent == 31) v = mantissa ? NAN : INFINITY;
+    else v = ldexp(1.0 + (double)mantissa / 1024.0, exponent - 15);
+    return (float)(sign ? -v : v);
+}
+
+void orc_widen_fp16(const uint16_t *h, float *out, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = orc_fp16_to_f32(h[i]);
 }
 
 /*
@@ -84,19 +109,23 @@ static double grad_at(const void *g, int grad_dtype, int64_t i)
 {
     if (grad_dtype == ORC_GRAD_BF16)
         return (double)orc_bf16_to_f32(((const uint16_t *)g)[i]);
+    if (grad_dtype == ORC_GRAD_FP16)
+        return (double)orc_fp16_to_f32(((const uint16_t *)g)[i]);
     return (double)((const float *)g)[i];
 }
 
 /* Sum of squares of one range in index order, and whether any element is
- * NaN or +-Inf.  The square is taken in double, so it cannot overflow for a
- * finite fp32/bf16 input. */
+ * NaN or +-Inf.  Each stored gradient is first multiplied by `unscale` (1 when
+ * no loss scaling is in use, 1/loss_scale otherwise), so the norm is that of
+ * the true gradient.  The square is taken in double, so it cannot overflow for
+ * a finite fp32/bf16/fp16 input. */
 int orc_grad_check_range(const void *g, int grad_dtype, int64_t begin, int64_t end,
-                         double *sumsq_out)
+                         double unscale, double *sumsq_out)
 {
     double s = 0.0;
     int nonfinite = 0;
     for (int64_t i = begin; i < end; ++i) {
-        double x = grad_at(g, grad_dtype, i);
+        double x = grad_at(g, grad_dtype, i) * unscale;
         if (!isfinite(x)) nonfinite = 1;
         s += x * x;
     }
@@ -107,14 +136,14 @@ int orc_grad_check_range(const void *g, int grad_dtype, int64_t begin, int64_t e
 /* Per-bucket partials in index order, then the sum over buckets in bucket
  * order; norm = sqrt(sum). */
 int orc_global_grad_check(const void *g, int grad_dtype, int64_t n, int64_t bucket_elems,
-                          double *sumsq_out, double *norm_out)
+                          double unscale, double *sumsq_out, double *norm_out)
 {
     double total = 0.0;
     int nonfinite = 0;
     for (int64_t b0 = 0; b0 < n; b0 += bucket_elems) {
         int64_t b1 = b0 + bucket_elems < n ? b0 + bucket_elems : n;
         double s;
-        if (orc_grad_check_range(g, grad_dtype, b0, b1, &s)) nonfinite = 1;
+        if (orc_grad_check_range(g, grad_dtype, b0, b1, unscale, &s)) nonfinite = 1;
         total += s;
     }
     *sumsq_out = total;
@@ -147,7 +176,7 @@ int orc_decision(int nonfinite, double coef)
  * One AdamW step over the flat range [begin, end) with step index tt (1-based)
  * and gradient scale `scale` (1 for an unclipped step, the clip coefficient
  * otherwise).  Kingma & Ba, Algorithm 1, with decoupled decay:
- *     g~   = scale * g
+ *     g~   = scale * (unscale * g_stored)
  *     m    = beta1*m + (1-beta1)*g~
  *     v    = beta2*v + (1-beta2)*g~^2
  *     mhat = m / (1 - beta1^tt),   vhat = v / (1 - beta2^tt)
@@ -155,13 +184,13 @@ int orc_decision(int nonfinite, double coef)
  * all in double; p, m, v are then rounded to fp32.
  */
 void orc_adamw_step_range(float *p, float *m, float *v, const void *g, int grad_dtype,
-                          int64_t begin, int64_t end, double scale, int64_t tt,
+                          int64_t begin, int64_t end, double unscale, double scale, int64_t tt,
                           double lr, double beta1, double beta2, double eps, double wd)
 {
     const double bc1 = 1.0 - pow(beta1, (double)tt);
     const double bc2 = 1.0 - pow(beta2, (double)tt);
     for (int64_t i = begin; i < end; ++i) {
-        double gs = grad_at(g, grad_dtype, i) * scale;
+        double gs = (grad_at(g, grad_dtype, i) * unscale) * scale;
         double m64 = beta1 * (double)m[i] + (1.0 - beta1) * gs;
         double v64 = beta2 * (double)v[i] + (1.0 - beta2) * (gs * gs);
         double mhat = m64 / bc1;
@@ -185,15 +214,15 @@ void orc_adamw_step_range(float *p, float *m, float *v, const void *g, int grad_
 int orc_iteration_ste(float *p, float *m, float *v, uint16_t *pb, const void *g,
                       int grad_dtype, int64_t n, int64_t bucket_elems, int64_t *t,
                       double lr, double beta1, double beta2, double eps, double wd,
-                      double max_norm, double *sumsq_out, double *norm_out,
+                      double max_norm, double unscale, double *sumsq_out, double *norm_out,
                       double *coef_out, int *nonfinite_out)
 {
     double sumsq, norm;
-    int nonfinite = orc_global_grad_check(g, grad_dtype, n, bucket_elems, &sumsq, &norm);
+    int nonfinite = orc_global_grad_check(g, grad_dtype, n, bucket_elems, unscale, &sumsq, &norm);
     double coef = orc_clip_coef(norm, max_norm);
     int decision = orc_decision(nonfinite, coef);
     if (decision != ORC_DECISION_SKIP) {
-        orc_adamw_step_range(p, m, v, g, grad_dtype, 0, n, coef, *t + 1,
+        orc_adamw_step_range(p, m, v, g, grad_dtype, 0, n, unscale, coef, *t + 1,
                              lr, beta1, beta2, eps, wd);
         orc_cast_params(p, pb, n);
         *t += 1;
@@ -217,7 +246,7 @@ int orc_iteration_ste(float *p, float *m, float *v, uint16_t *pb, const void *g,
 int orc_iteration_stv(float *p, float *m, float *v, uint16_t *pb, const void *g,
                       int grad_dtype, int64_t n, int64_t bucket_elems, int64_t *t,
                       double lr, double beta1, double beta2, double eps, double wd,
-                      double max_norm, double forced_coef, double *sumsq_out,
+                      double max_norm, double unscale, double forced_coef, double *sumsq_out,
                       double *norm_out, double *coef_out, int *nonfinite_out)
 {
     size_t fbytes = (size_t)n * sizeof(float);
@@ -231,14 +260,14 @@ int orc_iteration_stv(float *p, float *m, float *v, uint16_t *pb, const void *g,
     /* speculation: bucket by bucket, scale 1 */
     for (int64_t b0 = 0; b0 < n; b0 += bucket_elems) {
         int64_t b1 = b0 + bucket_elems < n ? b0 + bucket_elems : n;
-        orc_adamw_step_range(p, m, v, g, grad_dtype, b0, b1, 1.0, *t + 1,
+        orc_adamw_step_range(p, m, v, g, grad_dtype, b0, b1, unscale, 1.0, *t + 1,
                              lr, beta1, beta2, eps, wd);
         orc_cast_params(p + b0, pb + b0, b1 - b0);
     }
 
     /* validation */
     double sumsq, norm;
-    int nonfinite = orc_global_grad_check(g, grad_dtype, n, bucket_elems, &sumsq, &norm);
+    int nonfinite = orc_global_grad_check(g, grad_dtype, n, bucket_elems, unscale, &sumsq, &norm);
     double coef = orc_clip_coef(norm, max_norm);
     if (forced_coef > 0.0) coef = forced_coef;
     int decision = orc_decision(nonfinite, coef);
@@ -249,7 +278,7 @@ int orc_iteration_stv(float *p, float *m, float *v, uint16_t *pb, const void *g,
         memcpy(p, p0, fbytes); memcpy(m, m0, fbytes); memcpy(v, v0, fbytes);
         memcpy(pb, pb0, (size_t)n * 2);
         if (decision == ORC_DECISION_CLIP_RESTEP) {
-            orc_adamw_step_range(p, m, v, g, grad_dtype, 0, n, coef, *t + 1,
+            orc_adamw_step_range(p, m, v, g, grad_dtype, 0, n, unscale, coef, *t + 1,
                                  lr, beta1, beta2, eps, wd);
             orc_cast_params(p, pb, n);
             *t += 1;
@@ -258,6 +287,32 @@ int orc_iteration_stv(float *p, float *m, float *v, uint16_t *pb, const void *g,
     free(p0); free(m0); free(v0); free(pb0);
     *sumsq_out = sumsq; *norm_out = norm; *coef_out = coef; *nonfinite_out = nonfinite;
     return decision;
+}
+
+/* ---- dynamic loss scaling (the paper's FP16 runs; Section 4.4's NaN/Inf check
+ *      is this scaler's overflow test) ------------------------------------- */
+
+/*
+ * The loss-scale schedule of mixed-precision training (Micikevicius et al.,
+ * which the paper cites for its NaN/Inf check): after an iteration that found
+ * a non-finite gradient (and was therefore skipped) the scale is multiplied by
+ * `backoff` (< 1); after `interval` consecutive clean iterations it is
+ * multiplied by `growth` (> 1).  interval <= 0 keeps the scale fixed.
+ */
+void orc_loss_scale_update(double *scale, int64_t *good_steps, int nonfinite,
+                           double growth, double backoff, int64_t interval)
+{
+    if (interval <= 0) return;
+    if (nonfinite) {
+        *scale *= backoff;
+        *good_steps = 0;
+    } else {
+        *good_steps += 1;
+        if (*good_steps == interval) {
+            *scale *= growth;
+            *good_steps = 0;
+        }
+    }
 }
 
 /* ---- layout (Section 4.3: flat model states cut into fixed-size buckets) - */

@@ -454,3 +454,83 @@ def test_resident_bytes_follow_the_papers_accounting():
                 parts[line[0]] = int(line[1])
     assert sum(v for k, v in parts.items() if k != "total") == parts["total"] == 16
     assert oracle.resident_bytes(1_000_000) == parts["total"] * 1_000_000
+
+
+# ---------------------------------------------------------------------------
+# fp16 gradients and loss scaling (the paper's own precision path)
+# ---------------------------------------------------------------------------
+
+def test_fp16_widening_for_all_patterns_against_numpy():
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    got = oracle.fp16_to_f32(bits)
+    ref = bits.view(np.float16).astype(np.float32)
+    nan = np.isnan(ref)
+    assert nan.sum() == 2 * 1023
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got.view(np.uint32)[~nan], ref.view(np.uint32)[~nan])
+    # hand-checked anchors: 1.0, smallest subnormal, largest finite, -2.0, +inf
+    anchors = {0x3C00: 1.0, 0x0001: 2.0 ** -24, 0x7BFF: 65504.0, 0xC000: -2.0, 0x7C00: np.inf}
+    for pat, val in anchors.items():
+        assert got[pat] == np.float32(val), hex(pat)
+
+
+@pytest.mark.parametrize("unscale", [2.0 ** -16, 1.0 / 3000.0])
+@pytest.mark.parametrize("scale", [1.0, 0.25])
+def test_first_step_with_fp16_gradients_and_unscale_matches_exact_rationals(unscale, scale):
+    """Stored gradient g_s = S*g: the step must see g = unscale*g_s, then the
+    clip scale; closed form of the first Adam step in exact rationals."""
+    rng = np.random.default_rng(21)
+    n = 400
+    hp = HParams()
+    p0 = rng.normal(0, 0.02, n).astype(np.float32)
+    g = (rng.normal(0, 1e-2, n) / unscale).astype(np.float16)
+    assert np.isfinite(g).all()
+    p, m, v = p0.copy(), np.zeros(n, np.float32), np.zeros(n, np.float32)
+    oracle.adamw_step_range(p, m, v, g, 0, n, scale, 1, hp, unscale=unscale)
+    lr, b1, b2, eps, wd = map(_fr, (hp.lr, hp.beta1, hp.beta2, hp.eps, hp.weight_decay))
+    for i in range(n):
+        gs = _fr(g[i]) * _fr(unscale) * _fr(scale)
+        exp_m = f32_from_fraction((1 - b1) * gs)
+        exp_v = f32_from_fraction((1 - b2) * gs * gs)
+        exp_p = f32_from_fraction(_fr(p0[i]) * (1 - lr * wd) - lr * gs / (abs(gs) + eps))
+        assert ulp_distance(np.array([m[i]]), np.array([exp_m]))[0] <= 1
+        assert ulp_distance(np.array([v[i]]), np.array([exp_v]))[0] <= 1
+        assert ulp_distance(np.array([p[i]]), np.array([exp_p]))[0] <= 1
+
+
+def test_power_of_two_unscale_scales_the_norm_exactly():
+    rng = np.random.default_rng(22)
+    g = (rng.normal(0, 1.0, 20000) * 500).astype(np.float16)
+    s1, n1, f1 = oracle.global_grad_check(g, 4096)
+    s2, n2, f2 = oracle.global_grad_check(g, 4096, unscale=2.0 ** -12)
+    assert f1 == f2 == 0
+    assert s2 == s1 * 2.0 ** -24 and n2 == n1 * 2.0 ** -12
+    # an fp16 overflow in the stored gradient is a non-finite gradient
+    g[77] = np.float16(np.inf)
+    assert oracle.global_grad_check(g, 4096, unscale=2.0 ** -12)[2] == 1
+    # whole iteration: unscale folded into the step equals stepping on pre-divided fp32 gradients
+    g[77] = np.float16(3.0)
+    hp = HParams(max_grad_norm=0.0)
+    n = g.size
+    p0 = rng.normal(0, 0.02, n).astype(np.float32)
+    a = [p0.copy(), np.zeros(n, np.float32), np.zeros(n, np.float32), oracle.bf16_rne(p0)]
+    b = [x.copy() for x in a]
+    oracle.iteration_ste(*a, g, 4096, 0, hp, unscale=2.0 ** -12)
+    g32 = (g.astype(np.float32) * np.float32(2.0 ** -12))          # exact: power of two
+    oracle.iteration_ste(*b, g32, 4096, 0, hp)
+    for x, y in zip(a, b):
+        assert x.tobytes() == y.tobytes()
+
+
+def test_loss_scale_schedule():
+    """Back off on overflow, grow after `interval` clean steps, counter resets."""
+    scale, good = 65536.0, 0
+    seen = []
+    for bad in [0, 0, 0, 0, 1, 0, 0, 1, 1, 0, 0, 0]:
+        scale, good = oracle.loss_scale_update(scale, good, bad, 2.0, 0.5, 3)
+        seen.append(scale)
+    assert seen == [65536, 65536, 131072, 131072, 65536, 65536, 65536, 32768, 16384,
+                    16384, 16384, 32768]
+    # a static scale never moves
+    assert oracle.loss_scale_update(1024.0, 0, 1, 2.0, 0.5, 0) == (1024.0, 0)
+    assert oracle.loss_scale_update(1024.0, 0, 0, 2.0, 0.5, 0) == (1024.0, 0)
