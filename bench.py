@@ -31,7 +31,7 @@ if ROOT not in sys.path:
 
 METRIC = "optimizer_params_per_sec"
 UNIT = "params/s"
-BYTES_PER_PARAM = {"bf16": 28, "fp32": 30}      # algorithmic HBM bytes of the fused step
+BYTES_PER_PARAM = {"bf16": 28, "fp16": 28, "fp32": 30}      # algorithmic HBM bytes of the fused step
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per parameter of the fused step
 # kernel (gpt2_small capture: 1.742 GB read + 1.688 GB written per launch of
@@ -224,7 +224,7 @@ def main():
         # as many undo slots as fit next to the 16 B/param resident state
         stride = (w.bucket_elems + 63) // 64 * 64
         free_bytes, _ = torch.cuda.mem_get_info()
-        gsz_arena = 2 if w.grad_dtype == "bf16" else 4
+        gsz_arena = 4 if w.grad_dtype == "fp32" else 2
         resident = w.n_buckets * stride * (12 + gsz_arena + 2)
         room = free_bytes - resident - (6 << 30)
         undo = max(0, min(w.n_buckets, room // (12 * stride)))
@@ -232,7 +232,9 @@ def main():
                         step_variant=args.step_variant)
     opt.load_state_stream(W.iter_initial_master(w, device="cuda"))
     opt.cast_params(stream=stream)
-    opt.load_grads_stream(W.iter_gradients(w, 1, device="cuda"))
+    if w.grad_dtype == "fp16":
+        B.so_loss_scale_config(opt.ctx, w.loss_scale, w.ls_growth, w.ls_backoff, w.ls_interval)
+    opt.load_grads_stream(W.iter_gradients(w, 1, device="cuda", loss_scale=w.loss_scale))
     torch.cuda.synchronize()
     N = w.total
     nb = opt.n_buckets
@@ -293,9 +295,9 @@ def main():
     # ---- end to end through the host-buffer entry point -------------------
     e2e = None
     if not args.no_e2e and N <= (1 << 31):
-        gsz = 2 if w.grad_dtype == "bf16" else 4
+        gsz = 4 if w.grad_dtype == "fp32" else 2
         host_g = torch.empty(N, dtype=opt.grad_torch_dtype, pin_memory=True)
-        for start, piece in W.iter_gradients(w, 1, device="cuda"):
+        for start, piece in W.iter_gradients(w, 1, device="cuda", loss_scale=w.loss_scale):
             host_g[start:start + piece.numel()].copy_(piece)
         host_p = torch.empty(N, dtype=torch.bfloat16, pin_memory=True)
         for _ in range(3):

@@ -62,7 +62,7 @@ enum {
     SO_ERR_TOO_LARGE = -8              /* input exceeds a fixed built-in capacity           */
 };
 
-enum { SO_GRAD_BF16 = 0, SO_GRAD_FP32 = 1 };
+enum { SO_GRAD_BF16 = 0, SO_GRAD_FP32 = 1, SO_GRAD_FP16 = 2 };
 enum { SO_DECISION_COMMIT = 0, SO_DECISION_SKIP = 1, SO_DECISION_CLIP_RESTEP = 2 };
 #define SO_ALL (-1)
 
@@ -102,6 +102,7 @@ typedef struct {
     int32_t buckets_speculated;        /* buckets that had been stepped speculatively*/
     int64_t step_after;                /* committed step count after this call       */
     so_grad_stats stats;
+    double loss_scale;                 /* loss scale in effect for the next iteration */
 } so_step_result;
 
 typedef struct {
@@ -117,7 +118,7 @@ typedef struct {
  *   out          receives a new context (caller frees it with so_destroy)
  *   n_tensors    number of tensors (>= 0); numel[i] >= 0 elements each (host)
  *   bucket_elems B, 1 <= B <= 2^30
- *   grad_dtype   SO_GRAD_BF16 or SO_GRAD_FP32 (dtype of the gradient arena)
+ *   grad_dtype   SO_GRAD_BF16, SO_GRAD_FP32 or SO_GRAD_FP16 (dtype of the gradient arena)
  *   undo_slots   how many buckets may be stepped speculatively per iteration:
  *                0..n_buckets, or SO_ALL for n_buckets
  *   info         optional (host): filled with the sizes to allocate
@@ -138,7 +139,7 @@ so_status so_layout_tensor(const so_ctx *ctx, int32_t i, int64_t *flat_offset,
 /*
  * so_layout_bind -- hand the caller-owned DEVICE arenas to the context.
  * Sizes as reported by so_layout_init; pointers 256-byte aligned; master, m, v
- * are fp32, grad is bf16 or fp32 per grad_dtype, param_bf16 is bf16.  The
+ * are fp32, grad is bf16, fp16 or fp32 per grad_dtype, param_bf16 is bf16.  The
  * caller fills master/m/v slot b with bucket b's initial state (m = v = 0 for
  * a fresh optimizer) and normally calls so_cast_params(SO_ALL) once.  Scratch
  * needs no initialisation by the caller (bind zeroes a small control
@@ -269,6 +270,25 @@ so_status so_iteration_host(so_ctx *ctx, const so_hparams *hp, const void *host_
 #define SO_STATIC_CHECK_MAX_ELEMS (1 << 26)
 so_status so_grad_check_static(const void *grad, int64_t n_elems, int32_t grad_dtype,
                                double max_grad_norm, void *stream, so_grad_stats *out_device);
+
+/*
+ * so_loss_scale_config -- loss scaling for fp16 gradients (the paper trains in
+ * FP16 mixed precision, Section 4.5; the NaN/Inf check of Section 4.4 is the
+ * overflow test of this scheme).  The gradient arena then holds
+ * loss_scale * gradient; the check and the step multiply every stored value by
+ * 1 / loss_scale first, so norm, clipping and the update see the true gradient.
+ * interval > 0 enables the dynamic schedule: after an iteration that was
+ * skipped for a non-finite gradient the scale is multiplied by `backoff`
+ * (0 < backoff <= 1), after `interval` consecutive kept iterations by `growth`
+ * (>= 1); interval = 0 keeps the scale fixed.  The scale used by an iteration
+ * is the one in effect when the iteration starts; so_step_result.loss_scale
+ * tells the producer of the next gradients which scale to apply.
+ * Only for SO_GRAD_FP16 contexts (SO_ERR_UNSUPPORTED otherwise), only between
+ * iterations.  Host-only.
+ */
+so_status so_loss_scale_config(so_ctx *ctx, double init_scale, double growth, double backoff,
+                               int64_t interval);
+so_status so_get_loss_scale(const so_ctx *ctx, double *scale);
 
 /* Slot of the state arenas that holds bucket b's committed master/m/v. */
 so_status so_bucket_slot(const so_ctx *ctx, int32_t bucket, int32_t *slot);

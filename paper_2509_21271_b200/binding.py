@@ -18,7 +18,7 @@ SO_ERR_UNDO_EXHAUSTED, SO_ERR_NOMEM, SO_ERR_UNSUPPORTED = -4, -5, -6
 SO_ERR_TIMEOUT = -7
 SO_ERR_TOO_LARGE = -8
 SO_STATIC_CHECK_MAX_ELEMS = 1 << 26
-SO_GRAD_BF16, SO_GRAD_FP32 = 0, 1
+SO_GRAD_BF16, SO_GRAD_FP32, SO_GRAD_FP16 = 0, 1, 2
 SO_DECISION_COMMIT, SO_DECISION_SKIP, SO_DECISION_CLIP_RESTEP = 0, 1, 2
 SO_ALL = -1
 DECISION_NAMES = {0: "COMMIT", 1: "SKIP", 2: "CLIP_RESTEP"}
@@ -49,7 +49,8 @@ class so_grad_stats(C.Structure):
 
 class so_step_result(C.Structure):
     _fields_ = [("decision", C.c_int32), ("buckets_speculated", C.c_int32),
-                ("step_after", C.c_int64), ("stats", so_grad_stats)]
+                ("step_after", C.c_int64), ("stats", so_grad_stats),
+                ("loss_scale", C.c_double)]
 
 
 class so_counters(C.Structure):
@@ -72,7 +73,8 @@ _lib = None
 
 EXPORTS = ["so_layout_init", "so_layout_get_info", "so_layout_tensor", "so_layout_bind",
            "so_grad_check", "so_adam_step_speculative", "so_validate_commit_or_rollback",
-           "so_cast_params", "so_iteration_host", "so_grad_check_static", "so_bucket_slot", "so_get_step", "so_set_step",
+           "so_cast_params", "so_iteration_host", "so_grad_check_static", "so_loss_scale_config",
+           "so_get_loss_scale", "so_bucket_slot", "so_get_step", "so_set_step",
            "so_pending_buckets", "so_get_counters", "so_last_cuda_error", "so_strerror",
            "so_destroy", "so_debug_set_dry_run", "so_debug_set_bucket_stats",
            "so_debug_set_step_variant"]
@@ -101,6 +103,8 @@ def lib() -> C.CDLL:
         "so_cast_params": [vp, i32, vp],
         "so_iteration_host": [vp, P(so_hparams), vp, vp, vp, P(so_step_result)],
         "so_grad_check_static": [vp, i64, i32, dbl, vp, vp],
+        "so_loss_scale_config": [vp, dbl, dbl, dbl, i64],
+        "so_get_loss_scale": [vp, P(dbl)],
         "so_bucket_slot": [vp, i32, P(i32)],
         "so_get_step": [vp, P(i64)],
         "so_set_step": [vp, i64],
@@ -230,6 +234,18 @@ def so_grad_check_static(grad: int, n_elems: int, grad_dtype: int, max_grad_norm
     device addresses (a gradient buffer and a 32-byte so_grad_stats record)."""
     _ok(None, lib().so_grad_check_static(grad, n_elems, grad_dtype, max_grad_norm,
                                          _stream(stream), out_device), "so_grad_check_static")
+
+
+def so_loss_scale_config(ctx, init_scale: float, growth: float = 2.0, backoff: float = 0.5,
+                         interval: int = 0) -> None:
+    _ok(ctx, lib().so_loss_scale_config(ctx, init_scale, growth, backoff, interval),
+        "so_loss_scale_config")
+
+
+def so_get_loss_scale(ctx) -> float:
+    s = C.c_double()
+    _ok(ctx, lib().so_get_loss_scale(ctx, C.byref(s)), "so_get_loss_scale")
+    return s.value
 
 
 def so_bucket_slot(ctx, bucket: int) -> int:

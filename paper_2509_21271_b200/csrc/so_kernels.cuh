@@ -21,6 +21,7 @@
 // the stand-alone check kernel.
 #pragma once
 
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -43,6 +44,14 @@ struct Geometry {
 };
 
 // Per-step constants, all derived on the host in double precision.
+// Gradient element types: uint16_t carries bf16 bit patterns, half_t IEEE
+// binary16 bit patterns (the only type that is used with a loss scale), float
+// plain fp32.
+struct half_t { uint16_t bits; };
+
+template <typename GradT> struct grad_traits { static constexpr bool kUnscale = false; };
+template <> struct grad_traits<half_t> { static constexpr bool kUnscale = true; };
+
 struct AdamScalars {
     double beta1, omb1;                   // beta1, 1 - beta1
     double beta2, omb2;
@@ -51,6 +60,7 @@ struct AdamScalars {
     double decay;                         // 1 - lr * wd
     double eps;
     double scale;                         // gradient scale (clip coefficient)
+    double unscale;                       // 1 / loss scale (fp16 gradients), else 1
 };
 
 struct BucketEntry { int32_t bucket, src_slot, dst_slot; };
@@ -69,6 +79,7 @@ struct StepArgs {
 struct CheckArgs {
     const void *grad;
     double *partials;
+    double unscale;                       // 1 / loss scale (fp16 gradients), else 1
     Geometry geo;
     int32_t n_entries;
     int32_t bucket[kMaxBatch];
@@ -113,6 +124,41 @@ __device__ __forceinline__ void load_quad(const uint16_t *base, uint32_t idx, ui
 #pragma unroll
         for (int j = 0; j < 4; ++j)
             x[j] = (idx + j < n) ? bf16_bits_to_float(__ldcs(base + idx + j)) : 0.0f;
+    }
+}
+
+// two packed 16-bit gradients -> two floats (element at the lower address first)
+template <typename GradT>
+__device__ __forceinline__ void unpack2(uint32_t w, float &lo, float &hi);
+
+template <>
+__device__ __forceinline__ void unpack2<uint16_t>(uint32_t w, float &lo, float &hi)
+{
+    lo = __uint_as_float(w << 16);
+    hi = __uint_as_float(w & 0xFFFF0000u);
+}
+
+template <>
+__device__ __forceinline__ void unpack2<half_t>(uint32_t w, float &lo, float &hi)
+{
+    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w));
+    lo = f.x;
+    hi = f.y;
+}
+
+__device__ __forceinline__ void load_quad(const half_t *base, uint32_t idx, uint32_t n, float (&x)[4])
+{
+    if (idx + 4 <= n) {
+        const uint2 q = __ldcs(reinterpret_cast<const uint2 *>(base + idx));
+        unpack2<half_t>(q.x, x[0], x[1]);
+        unpack2<half_t>(q.y, x[2], x[3]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            x[j] = (idx + j < n)
+                       ? __half2float(__ushort_as_half(
+                             __ldcs(reinterpret_cast<const uint16_t *>(base) + idx + j)))
+                       : 0.0f;
     }
 }
 
@@ -209,11 +255,11 @@ __device__ __forceinline__ double rcp_pos(double b)
     return __fma_rn(y, e, y);
 }
 
-template <bool kScaled>
+template <bool kScaled, bool kUnscale>
 __device__ __forceinline__ void adamw_element(float g, float &p, float &m, float &v,
                                               const AdamScalars &k, double &sumsq)
 {
-    const double gd = (double)g;
+    const double gd = kUnscale ? __dmul_rn((double)g, k.unscale) : (double)g;
     const double gs = kScaled ? __dmul_rn(gd, k.scale) : gd;
     const double sq = __dmul_rn(gs, gs);
     if (!kScaled) sumsq = __dadd_rn(sumsq, sq);
@@ -278,7 +324,8 @@ __global__ void __launch_bounds__(kThreads, 2) adamw_step_kernel(const __grid_co
             for (int u = 0; u < kRowsInFlight; ++u) {
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
-                    adamw_element<!kSpec>(gq[u][q], pq[u][q], mq[u][q], vq[u][q], a.k, acc);
+                    adamw_element<!kSpec, grad_traits<GradT>::kUnscale>(gq[u][q], pq[u][q], mq[u][q],
+                                                                         vq[u][q], a.k, acc);
                 const uint32_t idx = base + (r0 + u) * kRowElems + lane * 4;
                 if (idx < n) {
                     store_quad(p_out, idx, n, pq[u]);
@@ -331,7 +378,9 @@ __global__ void __launch_bounds__(kThreads) grad_check_kernel(const __grid_const
         for (int r = 0; r < kRowsPerTile; ++r) {
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                const double gd = (double)gq[r][q];
+                const double gd = grad_traits<GradT>::kUnscale
+                                      ? __dmul_rn((double)gq[r][q], a.unscale)
+                                      : (double)gq[r][q];
                 acc = __dadd_rn(acc, __dmul_rn(gd, gd));
             }
         }

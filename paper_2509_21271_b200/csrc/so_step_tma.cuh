@@ -322,19 +322,18 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                 pq[0] = p4.x; pq[1] = p4.y; pq[2] = p4.z; pq[3] = p4.w;
                 mq[0] = m4.x; mq[1] = m4.y; mq[2] = m4.z; mq[3] = m4.w;
                 vq[0] = v4.x; vq[1] = v4.y; vq[2] = v4.z; vq[3] = v4.w;
-                if (sizeof(GradT) == 2) {
+                if constexpr (sizeof(GradT) == 2) {
                     const uint2 g2 = *reinterpret_cast<const uint2 *>(in + 3 * L::kF32Bytes + off * 2);
-                    gq[0] = __uint_as_float(g2.x << 16);
-                    gq[1] = __uint_as_float(g2.x & 0xFFFF0000u);
-                    gq[2] = __uint_as_float(g2.y << 16);
-                    gq[3] = __uint_as_float(g2.y & 0xFFFF0000u);
+                    unpack2<GradT>(g2.x, gq[0], gq[1]);
+                    unpack2<GradT>(g2.y, gq[2], gq[3]);
                 } else {
                     const float4 g4 = *reinterpret_cast<const float4 *>(in + 3 * L::kF32Bytes + off * 4);
                     gq[0] = g4.x; gq[1] = g4.y; gq[2] = g4.z; gq[3] = g4.w;
                 }
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
-                    adamw_element<!kSpec>(gq[q], pq[q], mq[q], vq[q], a.k, acc);
+                    adamw_element<!kSpec, grad_traits<GradT>::kUnscale>(gq[q], pq[q], mq[q], vq[q],
+                                                                         a.k, acc);
                 *reinterpret_cast<float4 *>(out + off * 4) = make_float4(pq[0], pq[1], pq[2], pq[3]);
                 *reinterpret_cast<float4 *>(out + L::kF32Bytes + off * 4) =
                     make_float4(mq[0], mq[1], mq[2], mq[3]);
@@ -371,7 +370,8 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                 load_quad(a.var + src, idx, d.n, vq);
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
-                    adamw_element<!kSpec>(gq[q], pq[q], mq[q], vq[q], a.k, acc);
+                    adamw_element<!kSpec, grad_traits<GradT>::kUnscale>(gq[q], pq[q], mq[q], vq[q],
+                                                                         a.k, acc);
                 if (idx < d.n) {
                     store_quad(a.master + dst, idx, d.n, pq);
                     store_quad(a.mom + dst, idx, d.n, mq);

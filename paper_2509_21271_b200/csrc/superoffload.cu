@@ -60,6 +60,12 @@ struct so_ctx {
     so_hparams hp_iter{};
     so_grad_stats stats{};
     int64_t t = 0;
+    // ---- loss scaling (fp16 gradients) ----
+    double loss_scale = 1.0;            // stored gradient = loss_scale * gradient
+    double ls_growth = 2.0, ls_backoff = 0.5;
+    int64_t ls_interval = 0;            // clean iterations before growth; 0 = static scale
+    int64_t ls_good_steps = 0;
+    double iter_unscale = 1.0;          // 1 / loss_scale, fixed for the iteration in flight
     // ---- bookkeeping ----
     so_counters counters{};
     int32_t last_cuda_error = 0;
@@ -110,7 +116,7 @@ bool hparams_equal(const so_hparams &a, const so_hparams &b)
     return std::memcmp(&a, &b, sizeof(so_hparams)) == 0;
 }
 
-AdamScalars scalars_for(const so_hparams &hp, int64_t step_index, double scale)
+AdamScalars scalars_for(const so_hparams &hp, int64_t step_index, double scale, double unscale)
 {
     const double bc1 = 1.0 - std::pow(hp.beta1, (double)step_index);
     const double bc2 = 1.0 - std::pow(hp.beta2, (double)step_index);
@@ -124,6 +130,7 @@ AdamScalars scalars_for(const so_hparams &hp, int64_t step_index, double scale)
     k.decay = 1.0 - hp.lr * hp.weight_decay;
     k.eps = hp.eps;
     k.scale = scale;
+    k.unscale = unscale;
     return k;
 }
 
@@ -183,14 +190,15 @@ void launch_tma(so_ctx *c, const StepArgs &a, int n, bool speculative, cudaStrea
 
 void launch_tma_variant(so_ctx *c, const StepArgs &a, int n, bool speculative, cudaStream_t stream)
 {
-    const bool bf16 = c->grad_dtype == SO_GRAD_BF16;
-    if (c->step_variant == 10 && bf16) {
+    const int dt = c->grad_dtype;
+    if (c->step_variant == 10 && dt == SO_GRAD_BF16) {
         launch_tma<uint16_t, ShapeAlt16>(c, a, n, speculative, stream);
-    } else if (c->step_variant == 11) {
-        if (bf16) launch_tma<uint16_t, ShapeAlt12>(c, a, n, speculative, stream);
+    } else if (c->step_variant == 11 && dt != SO_GRAD_FP16) {
+        if (dt == SO_GRAD_BF16) launch_tma<uint16_t, ShapeAlt12>(c, a, n, speculative, stream);
         else launch_tma<float, ShapeAlt12>(c, a, n, speculative, stream);
     } else {
-        if (bf16) launch_tma<uint16_t, ShapeBf16>(c, a, n, speculative, stream);
+        if (dt == SO_GRAD_BF16) launch_tma<uint16_t, ShapeBf16>(c, a, n, speculative, stream);
+        else if (dt == SO_GRAD_FP16) launch_tma<half_t, ShapeBf16>(c, a, n, speculative, stream);
         else launch_tma<float, ShapeFp32>(c, a, n, speculative, stream);
     }
 }
@@ -225,7 +233,7 @@ so_status launch_steps(so_ctx *c, const std::vector<BucketEntry> &entries, const
         a.param_bf16 = c->param_bf16;
         a.partials = c->d_partials;
         a.geo = geo;
-        a.k = scalars_for(hp, c->t + 1, scale);
+        a.k = scalars_for(hp, c->t + 1, scale, c->iter_unscale);
         a.n_entries = n;
         for (int i = 0; i < n; ++i) {
             a.e[i] = entries[first + i];
@@ -233,16 +241,17 @@ so_status launch_steps(so_ctx *c, const std::vector<BucketEntry> &entries, const
         }
         for (int i = n; i < kMaxBatch; ++i) a.e[i] = BucketEntry{0, 0, 0};
         if (!c->dry_run) {
-            const bool bf16 = c->grad_dtype == SO_GRAD_BF16;
+            const int dt = c->grad_dtype;
+            const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_step);
             if (c->step_variant != 1) {
                 launch_tma_variant(c, a, n, speculative, stream);
             } else if (speculative) {
-                const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_step);
-                if (bf16) adamw_step_kernel<uint16_t, true, 4><<<grid, kThreads, 0, stream>>>(a);
+                if (dt == SO_GRAD_BF16) adamw_step_kernel<uint16_t, true, 4><<<grid, kThreads, 0, stream>>>(a);
+                else if (dt == SO_GRAD_FP16) adamw_step_kernel<half_t, true, 4><<<grid, kThreads, 0, stream>>>(a);
                 else adamw_step_kernel<float, true, 4><<<grid, kThreads, 0, stream>>>(a);
             } else {
-                const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_step);
-                if (bf16) adamw_step_kernel<uint16_t, false, 4><<<grid, kThreads, 0, stream>>>(a);
+                if (dt == SO_GRAD_BF16) adamw_step_kernel<uint16_t, false, 4><<<grid, kThreads, 0, stream>>>(a);
+                else if (dt == SO_GRAD_FP16) adamw_step_kernel<half_t, false, 4><<<grid, kThreads, 0, stream>>>(a);
                 else adamw_step_kernel<float, false, 4><<<grid, kThreads, 0, stream>>>(a);
             }
         }
@@ -260,6 +269,7 @@ so_status launch_checks(so_ctx *c, const std::vector<int32_t> &buckets, cudaStre
         CheckArgs a;
         a.grad = c->grad;
         a.partials = c->d_partials;
+        a.unscale = c->iter_unscale;
         a.geo = geo;
         a.n_entries = n;
         for (int i = 0; i < n; ++i) {
@@ -271,6 +281,8 @@ so_status launch_checks(so_ctx *c, const std::vector<int32_t> &buckets, cudaStre
             const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_check);
             if (c->grad_dtype == SO_GRAD_BF16)
                 grad_check_kernel<uint16_t><<<grid, kThreads, 0, stream>>>(a);
+            else if (c->grad_dtype == SO_GRAD_FP16)
+                grad_check_kernel<half_t><<<grid, kThreads, 0, stream>>>(a);
             else
                 grad_check_kernel<float><<<grid, kThreads, 0, stream>>>(a);
         }
@@ -402,6 +414,7 @@ so_status finalize_check(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
 
 void end_iteration(so_ctx *c)
 {
+    c->iter_unscale = 1.0 / c->loss_scale;
     std::fill(c->cover.begin(), c->cover.end(), (uint8_t)kNone);
     std::fill(c->spec_slot.begin(), c->spec_slot.end(), -1);
     c->n_covered = 0;
@@ -431,7 +444,8 @@ so_status so_layout_init(so_ctx **out, int32_t n_tensors, const int64_t *numel,
 {
     if (!out || n_tensors < 0 || (n_tensors > 0 && !numel)) return SO_ERR_INVALID_ARG;
     if (bucket_elems < 1 || bucket_elems > ((int64_t)1 << 30)) return SO_ERR_INVALID_ARG;
-    if (grad_dtype != SO_GRAD_BF16 && grad_dtype != SO_GRAD_FP32) return SO_ERR_INVALID_ARG;
+    if (grad_dtype != SO_GRAD_BF16 && grad_dtype != SO_GRAD_FP32 && grad_dtype != SO_GRAD_FP16)
+        return SO_ERR_INVALID_ARG;
     int64_t total = 0;
     for (int32_t i = 0; i < n_tensors; ++i) {
         if (numel[i] < 0 || numel[i] > ((int64_t)1 << 46)) return SO_ERR_INVALID_ARG;
@@ -493,7 +507,7 @@ so_status so_layout_get_info(const so_ctx *c, so_layout_info *info)
     const uint64_t state = (uint64_t)c->n_slots * (uint64_t)c->stride * 4u;
     info->bytes_master = info->bytes_m = info->bytes_v = state;
     info->bytes_grad = (uint64_t)c->n_buckets * (uint64_t)c->stride *
-                       (c->grad_dtype == SO_GRAD_BF16 ? 2u : 4u);
+                       (c->grad_dtype == SO_GRAD_FP32 ? 4u : 2u);
     info->bytes_param_bf16 = (uint64_t)c->n_buckets * (uint64_t)c->stride * 2u;
     const uint64_t partial_bytes = (uint64_t)c->n_buckets * (uint64_t)c->tiles_per_slot * 8u;
     const uint64_t stats_bytes = (uint64_t)c->n_buckets * sizeof(BucketStats) + sizeof(ControlBlock);
@@ -531,21 +545,30 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
         if (e != cudaSuccess) return cuda_fail(c, e);
         e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, c->device);
         if (e != cudaSuccess) return cuda_fail(c, e);
-        const bool bf16 = c->grad_dtype == SO_GRAD_BF16;
-        e = bf16 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                       &c->occ_step, adamw_step_kernel<uint16_t, true, 4>, kThreads, 0)
-                 : cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                       &c->occ_step, adamw_step_kernel<float, true, 4>, kThreads, 0);
+        const int dt = c->grad_dtype;
+        e = dt == SO_GRAD_BF16
+                ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                      &c->occ_step, adamw_step_kernel<uint16_t, true, 4>, kThreads, 0)
+            : dt == SO_GRAD_FP16
+                ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                      &c->occ_step, adamw_step_kernel<half_t, true, 4>, kThreads, 0)
+                : cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                      &c->occ_step, adamw_step_kernel<float, true, 4>, kThreads, 0);
         if (e != cudaSuccess) return cuda_fail(c, e);
-        e = bf16 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                       &c->occ_check, grad_check_kernel<uint16_t>, kThreads, 0)
-                 : cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                       &c->occ_check, grad_check_kernel<float>, kThreads, 0);
+        e = dt == SO_GRAD_BF16
+                ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                      &c->occ_check, grad_check_kernel<uint16_t>, kThreads, 0)
+            : dt == SO_GRAD_FP16
+                ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                      &c->occ_check, grad_check_kernel<half_t>, kThreads, 0)
+                : cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+                      &c->occ_check, grad_check_kernel<float>, kThreads, 0);
         if (e != cudaSuccess) return cuda_fail(c, e);
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_cast, cast_params_kernel,
                                                           kThreads, 0);
         if (e != cudaSuccess) return cuda_fail(c, e);
         e = allow_smem<uint16_t, ShapeBf16>();
+        if (e == cudaSuccess) e = allow_smem<half_t, ShapeBf16>();
         if (e == cudaSuccess) e = allow_smem<float, ShapeFp32>();
         if (e == cudaSuccess) e = allow_smem<uint16_t, ShapeAlt16>();
         if (e == cudaSuccess) e = allow_smem<uint16_t, ShapeAlt12>();
@@ -720,11 +743,23 @@ so_status so_validate_commit_or_rollback(so_ctx *c, const so_hparams *hp, void *
         c->t += 1;
         if (clip) c->counters.clip_resteps += 1; else c->counters.commits += 1;
     }
+    // dynamic loss scaling: back off after an overflow, grow after a run of
+    // clean iterations (takes effect from the next iteration on)
+    if (c->ls_interval > 0) {
+        if (decision == SO_DECISION_SKIP) {
+            c->loss_scale *= c->ls_backoff;
+            c->ls_good_steps = 0;
+        } else if (++c->ls_good_steps == c->ls_interval) {
+            c->loss_scale *= c->ls_growth;
+            c->ls_good_steps = 0;
+        }
+    }
     if (out) {
         out->decision = decision;
         out->buckets_speculated = n_spec;
         out->step_after = c->t;
         out->stats = c->stats;
+        out->loss_scale = c->loss_scale;
     }
     end_iteration(c);
     return SO_OK;
@@ -767,7 +802,7 @@ so_status so_iteration_host(so_ctx *c, const so_hparams *hp, const void *host_gr
         if (e != cudaSuccess) return cuda_fail(c, e);
         c->events.push_back(ev);
     }
-    const size_t gsz = c->grad_dtype == SO_GRAD_BF16 ? 2 : 4;
+    const size_t gsz = c->grad_dtype == SO_GRAD_FP32 ? 4 : 2;
     const char *hg = static_cast<const char *>(host_grad);
     char *hp_out = static_cast<char *>(host_param_bf16);
     char *dgrad = static_cast<char *>(c->grad);
@@ -829,6 +864,32 @@ so_status so_iteration_host(so_ctx *c, const so_hparams *hp, const void *host_gr
     e = cudaStreamSynchronize(main);
     if (e != cudaSuccess) return cuda_fail(c, e);
     if (out) *out = res;
+    return SO_OK;
+}
+
+so_status so_loss_scale_config(so_ctx *c, double init_scale, double growth, double backoff,
+                               int64_t interval)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (c->phase != kIdle) return SO_ERR_STATE;
+    if (c->grad_dtype != SO_GRAD_FP16) return SO_ERR_UNSUPPORTED;
+    if (!(init_scale > 0.0) || !std::isfinite(init_scale) || interval < 0) return SO_ERR_INVALID_ARG;
+    if (interval > 0 && (!(growth >= 1.0) || !std::isfinite(growth) || !(backoff > 0.0) ||
+                         !(backoff <= 1.0)))
+        return SO_ERR_INVALID_ARG;
+    c->loss_scale = init_scale;
+    c->ls_growth = growth;
+    c->ls_backoff = backoff;
+    c->ls_interval = interval;
+    c->ls_good_steps = 0;
+    c->iter_unscale = 1.0 / init_scale;
+    return SO_OK;
+}
+
+so_status so_get_loss_scale(const so_ctx *c, double *scale)
+{
+    if (!c || !scale) return SO_ERR_INVALID_ARG;
+    *scale = c->loss_scale;
     return SO_OK;
 }
 

@@ -27,11 +27,12 @@ class BucketedAdamW:
                  undo_slots: int = B.SO_ALL, device: str = "cuda", guard_bands: bool = False,
                  step_variant: int = 0):
         self.device = torch.device(device)
-        gd = B.SO_GRAD_BF16 if grad_dtype == "bf16" else B.SO_GRAD_FP32
+        gd = {"bf16": B.SO_GRAD_BF16, "fp32": B.SO_GRAD_FP32, "fp16": B.SO_GRAD_FP16}[grad_dtype]
         self.ctx, self.info = B.so_layout_init(list(numel), bucket_elems, gd, undo_slots)
         if step_variant:
             B.so_debug_set_step_variant(self.ctx, step_variant)
-        self.grad_torch_dtype = torch.bfloat16 if gd == B.SO_GRAD_BF16 else torch.float32
+        self.grad_torch_dtype = {B.SO_GRAD_BF16: torch.bfloat16, B.SO_GRAD_FP32: torch.float32,
+                                 B.SO_GRAD_FP16: torch.float16}[gd]
         self.guard_bands = guard_bands
         i = self.info
         self._raw = {}

@@ -45,7 +45,13 @@ class Workload:
     beta2: float = 0.999
     eps: float = 1e-8
     weight_decay: float = 0.01
-    grad_dtype: str = "bf16"         # "bf16" | "fp32"
+    grad_dtype: str = "bf16"         # "bf16" | "fp32" | "fp16"
+    # fp16 gradients are stored multiplied by a loss scale (initial value and
+    # dynamic schedule: growth / backoff factors, clean iterations before growth)
+    loss_scale: float = 1.0
+    ls_growth: float = 2.0
+    ls_backoff: float = 0.5
+    ls_interval: int = 0
     faults: Tuple[Fault, ...] = ()
     # optional: target global gradient norm per step (gradients are rescaled)
     target_norm: Optional[Callable[[int], float]] = None
@@ -117,6 +123,20 @@ def tiny() -> Workload:
                     notes="clip=1.0 < norm ~ 10.24: CLIP_RESTEP every step, SKIP on step 7")
 
 
+def tiny_fp16() -> Workload:
+    """The tiny case with fp16 gradients under dynamic loss scaling: the
+    initial scale overflows fp16, so the first iterations are skipped while the
+    scale backs off; afterwards it grows every 3 clean iterations until it
+    overflows again."""
+    w = tiny()
+    w.name = "tiny_fp16"
+    w.grad_dtype = "fp16"
+    w.faults = ()
+    w.loss_scale = 2.0 ** 23
+    w.ls_interval = 3
+    return w
+
+
 def tiny_ragged() -> Workload:
     """The tiny case cut into odd-sized tensors and an odd bucket size."""
     sizes = [1, 7, 262_143, 5, 100_003, 333_331, 64, 2, 352_020]
@@ -151,11 +171,12 @@ def llama_8b() -> Workload:
 def sweep(bucket_mi: int, grad_dtype: str = "bf16", total: int = 4 << 30) -> Workload:
     return Workload(name=f"sweep_{bucket_mi}Mi_{grad_dtype}", numel=[total],
                     bucket_elems=bucket_mi * MI, sigma_g=1e-3, steps=10, max_grad_norm=0.0,
-                    grad_dtype=grad_dtype)
+                    grad_dtype=grad_dtype, loss_scale=4096.0 if grad_dtype == "fp16" else 1.0)
 
 
 def by_name(name: str) -> Workload:
-    table = {"tiny": tiny, "tiny_ragged": tiny_ragged, "gpt2_small": gpt2_small,
+    table = {"tiny": tiny, "tiny_ragged": tiny_ragged, "tiny_fp16": tiny_fp16,
+             "gpt2_small": gpt2_small,
              "gpt2_small_clip": lambda: gpt2_small(clip=True),
              "llama_1b": llama_1b, "llama_8b": llama_8b}
     if name in table:
@@ -210,15 +231,21 @@ def faults_for_step(w: Workload, step: int) -> List[Fault]:
     return out
 
 
-def iter_gradients(w: Workload, step: int, device="cpu", chunk: int = 1 << 26):
+_TORCH_DTYPE = {"bf16": torch.bfloat16, "fp32": torch.float32, "fp16": torch.float16}
+
+
+def iter_gradients(w: Workload, step: int, device="cpu", chunk: int = 1 << 26,
+                   loss_scale: float = 1.0):
     """Yields (start, tensor) pieces of the flat gradient of iteration ``step``
     (1-based) in order, in the workload's gradient dtype.
 
     Drawn in fp32 ~ N(0, sigma_g); when the workload fixes a target global
     norm the draw is rescaled by ``target / ||draw||`` (double precision
-    scalar) before the bf16 rounding; faults are written last.
+    scalar) before the rounding to the gradient dtype; ``loss_scale`` (fp16
+    training) multiplies the value that gets stored, so large scales overflow
+    to infinity exactly as a scaled backward pass would; faults are written last.
     """
-    dtype = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
+    dtype = _TORCH_DTYPE[w.grad_dtype]
     gen = _gen(device, w.seed * 1_000_003 + step)
     scale = None
     if w.target_norm is not None:
@@ -239,6 +266,8 @@ def iter_gradients(w: Workload, step: int, device="cpu", chunk: int = 1 << 26):
         z.normal_(0.0, w.sigma_g, generator=gen)
         if scale is not None:
             z = (z.double() * scale).float()
+        if loss_scale != 1.0:
+            z = z * loss_scale
         z = z.to(dtype)
         for f in faults:
             if s <= f.flat_index < e:
@@ -246,11 +275,11 @@ def iter_gradients(w: Workload, step: int, device="cpu", chunk: int = 1 << 26):
         yield s, z
 
 
-def gradients(w: Workload, step: int, device="cpu", chunk: int = 1 << 26) -> torch.Tensor:
-    """Flat gradient of iteration ``step`` (1-based): bf16 or fp32 tensor."""
-    dtype = torch.bfloat16 if w.grad_dtype == "bf16" else torch.float32
-    out = torch.empty(w.total, dtype=dtype, device=device)
-    for s, z in iter_gradients(w, step, device, chunk):
+def gradients(w: Workload, step: int, device="cpu", chunk: int = 1 << 26,
+              loss_scale: float = 1.0) -> torch.Tensor:
+    """Flat gradient of iteration ``step`` (1-based) in the workload's dtype."""
+    out = torch.empty(w.total, dtype=_TORCH_DTYPE[w.grad_dtype], device=device)
+    for s, z in iter_gradients(w, step, device, chunk, loss_scale):
         out[s:s + z.numel()] = z
     return out
 

@@ -33,7 +33,7 @@ def grads_to_numpy(g: torch.Tensor) -> np.ndarray:
     """Device/host gradient tensor -> what the oracle takes (bits or fp32)."""
     if g.dtype == torch.bfloat16:
         return g.view(torch.int16).cpu().numpy().view(np.uint16)
-    return g.cpu().numpy()
+    return g.cpu().numpy()                      # float32, or float16 (fp16 gradients)
 
 
 def bf16_to_numpy(t: torch.Tensor) -> np.ndarray:
@@ -48,6 +48,7 @@ class Report:
     n_elems: int = 0
     max_norm_rel: float = 0.0
     bf16_mismatch: int = 0
+    loss_scales: list = field(default_factory=list)
 
 
 def assert_bf16_consistent(pb_dev: np.ndarray, p_dev: np.ndarray, pb_orc: np.ndarray,
@@ -109,8 +110,12 @@ def run_lockstep(w: W.Workload, steps: int, undo_slots: int = B.SO_ALL,
     assert np.array_equal(pb, oracle.bf16_rne(p)), "initial cast differs from the oracle"
     rep = Report()
     t = 0
+    loss_scale, good_steps = w.loss_scale, 0
+    if w.grad_dtype == "fp16":
+        B.so_loss_scale_config(opt.ctx, w.loss_scale, w.ls_growth, w.ls_backoff, w.ls_interval)
+    rep.loss_scales = []
     for step in range(1, steps + 1):
-        g = W.gradients(w, step, device="cuda")
+        g = W.gradients(w, step, device="cuda", loss_scale=loss_scale)
         opt.load_grads(g)
         g_host = grads_to_numpy(g)
         res = opt.iteration(hp, stream=stream, speculative=speculative)
@@ -119,7 +124,12 @@ def run_lockstep(w: W.Workload, steps: int, undo_slots: int = B.SO_ALL,
         # oracle replay from the device's pre-step state
         forced = res.stats.clip_coef if res.decision == B.SO_DECISION_CLIP_RESTEP else None
         orc_res = oracle.iteration_stv(p, m, v, pb, g_host, w.bucket_elems, t, hp,
-                                       forced_coef=forced)
+                                       forced_coef=forced, unscale=1.0 / loss_scale)
+        # the loss-scale schedule must follow the oracle's, exactly
+        loss_scale, good_steps = oracle.loss_scale_update(
+            loss_scale, good_steps, orc_res.nonfinite, w.ls_growth, w.ls_backoff, w.ls_interval)
+        assert res.loss_scale == loss_scale == B.so_get_loss_scale(opt.ctx), step
+        rep.loss_scales.append(loss_scale)
         own_coef = oracle.clip_coef(orc_res.norm, hp.max_grad_norm)
         own_decision = oracle.decision(orc_res.nonfinite, own_coef)
         assert res.decision == own_decision == orc_res.decision, (step, res.decision, own_decision)

@@ -41,7 +41,7 @@ def _release_device_memory():
 def _undo_that_fits(w: W.Workload) -> int:
     stride = (w.bucket_elems + 63) // 64 * 64
     free_bytes, _ = torch.cuda.mem_get_info()
-    gsz = 2 if w.grad_dtype == "bf16" else 4
+    gsz = 4 if w.grad_dtype == "fp32" else 2
     resident = w.n_buckets * stride * (12 + gsz + 2)
     room = free_bytes - resident - (8 << 30)
     assert room > 0, "workload does not fit on this GPU"

@@ -305,3 +305,32 @@ def test_host_fed_iteration_is_bitwise_the_device_fed_one(name, undo):
     assert trace == ref[0]
     assert _state_bytes(opt) == ref[1]
     assert S in [t[0] for t in trace]
+
+
+# ---------------------------------------------------------------------------
+# fp16 gradients under dynamic loss scaling (the paper's own precision path)
+# ---------------------------------------------------------------------------
+
+def test_fp16_gradients_with_dynamic_loss_scale_lockstep():
+    """Stored gradients are loss_scale * g in fp16.  The initial scale 2^23
+    overflows (SKIP, scale halves) until the scaled gradients fit; then every
+    step clips (norm ~ 10 > 1) and the scale doubles every 3 kept steps until
+    it overflows again.  State, decisions and the scale schedule must follow
+    the oracle."""
+    rep, opt = run_lockstep(W.tiny_fp16(), steps=16)
+    assert rep.decisions[0] == S and R in rep.decisions
+    first_kept = rep.decisions.index(R)
+    assert all(d == S for d in rep.decisions[:first_kept]) and first_kept >= 2
+    assert S in rep.decisions[first_kept:]              # grew back into an overflow
+    assert rep.loss_scales[first_kept - 1] == 2.0 ** (23 - first_kept)
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+    assert opt.step_count == rep.decisions.count(R)
+
+
+def test_fp16_static_scale_register_variant_and_check_first_flow():
+    w = W.tiny_fp16()
+    w.loss_scale, w.ls_interval = 2.0 ** 12, 0
+    a, _ = run_lockstep(w, steps=4, step_variant=1)
+    b, _ = run_lockstep(w, steps=4, undo_slots=0, speculative=False)
+    assert a.decisions == b.decisions == [R] * 4
+    assert a.loss_scales == b.loss_scales == [2.0 ** 12] * 4

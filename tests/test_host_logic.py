@@ -270,3 +270,37 @@ def test_strerror_is_defined_for_every_status():
     for s in range(-6, 1):
         assert B.strerror(s) and B.strerror(s) != "unknown status"
     assert B.strerror(-99) == "unknown status"
+
+
+def test_loss_scale_schedule_follows_the_oracle():
+    ctx, _ = _dry_ctx([1000], 256, gd=B.SO_GRAD_FP16)
+    hp = HP(max_grad_norm=0.0)
+    B.so_loss_scale_config(ctx, 65536.0, 2.0, 0.5, 3)
+    scale, good = 65536.0, 0
+    for bad in [0, 0, 0, 0, 1, 0, 0, 1, 1, 0, 0, 0]:
+        for b in range(4):
+            B.so_debug_set_bucket_stats(ctx, b, 1e-4, 1 if (bad and b == 2) else 0)
+        B.so_adam_step_speculative(ctx, hp, B.SO_ALL)
+        r = B.so_validate_commit_or_rollback(ctx, hp)
+        scale, good = oracle.loss_scale_update(scale, good, bad, 2.0, 0.5, 3)
+        assert r.loss_scale == scale == B.so_get_loss_scale(ctx)
+        assert r.decision == (B.SO_DECISION_SKIP if bad else B.SO_DECISION_COMMIT)
+    assert B.so_get_step(ctx) == 9
+    B.so_destroy(ctx)
+
+
+def test_loss_scale_is_only_for_fp16_contexts_and_validates_its_arguments():
+    ctx, _ = _dry_ctx([1000], 256)
+    assert _status(B.so_loss_scale_config, ctx, 1024.0) == B.SO_ERR_UNSUPPORTED
+    B.so_destroy(ctx)
+    ctx, info = _dry_ctx([1000], 256, gd=B.SO_GRAD_FP16)
+    assert info.bytes_grad == 4 * 256 * 2
+    bad = B.SO_ERR_INVALID_ARG
+    assert _status(B.so_loss_scale_config, ctx, 0.0) == bad
+    assert _status(B.so_loss_scale_config, ctx, 1024.0, 0.5, 0.5, 10) == bad     # growth < 1
+    assert _status(B.so_loss_scale_config, ctx, 1024.0, 2.0, 1.5, 10) == bad     # backoff > 1
+    assert _status(B.so_loss_scale_config, ctx, 1024.0, 2.0, 0.5, -1) == bad
+    B.so_loss_scale_config(ctx, 1024.0)                                          # static scale
+    B.so_adam_step_speculative(ctx, HP(), 0)
+    assert _status(B.so_loss_scale_config, ctx, 2048.0) == B.SO_ERR_STATE        # mid-iteration
+    B.so_destroy(ctx)
