@@ -209,6 +209,21 @@ so_status so_validate_commit_or_rollback(so_ctx *ctx, const so_hparams *hp, void
                                          so_step_result *out);
 
 /*
+ * so_validate_begin / so_validate_poll -- validation off the critical path
+ * (Section 4.4: validation runs while the GPU executes the next forward pass,
+ * and the result is consulted after it).  so_validate_begin scans whatever is
+ * still uncovered and launches the reduction; its records make their own way
+ * to the host and the call returns at once.  The caller then enqueues other
+ * work (the next forward pass) and later calls
+ * so_validate_commit_or_rollback, which by then finds the verdict waiting;
+ * so_validate_poll tells without blocking whether it has arrived (*ready = 1).
+ * Between so_validate_begin and so_validate_commit_or_rollback no bucket may be
+ * stepped or scanned (SO_ERR_STATE).
+ */
+so_status so_validate_begin(so_ctx *ctx, const so_hparams *hp, void *stream);
+so_status so_validate_poll(so_ctx *ctx, int32_t *ready);
+
+/*
  * so_cast_params -- fp32 master -> bf16 parameter copy, round to nearest even
  * (Section 4.5: the cast runs on the GPU).  bucket >= 0 or SO_ALL.  Only
  * between iterations (SO_ERR_STATE while buckets are covered).  Enqueues only.
@@ -289,6 +304,21 @@ so_status so_grad_check_static(const void *grad, int64_t n_elems, int32_t grad_d
 so_status so_loss_scale_config(so_ctx *ctx, double init_scale, double growth, double backoff,
                                int64_t interval);
 so_status so_get_loss_scale(const so_ctx *ctx, double *scale);
+
+/*
+ * so_state_export / so_state_import -- checkpoint and resume.  Copy the
+ * committed fp32 state (master weights, first and second moments) between the
+ * slot arenas and flat arrays of N floats in parameter order; each of master,
+ * m, v may be NULL to skip it, and may point to device or host memory (pinned
+ * for truly asynchronous copies).  One cudaMemcpyAsync per bucket and array on
+ * `stream`; no synchronisation.  Together with so_get_step / so_set_step (and,
+ * for fp16, the loss scale) this is the whole optimizer state.  After an
+ * import call so_cast_params(SO_ALL) to re-derive the bf16 copy.  Only between
+ * iterations.
+ */
+so_status so_state_export(so_ctx *ctx, void *master, void *m, void *v, void *stream);
+so_status so_state_import(so_ctx *ctx, const void *master, const void *m, const void *v,
+                          void *stream);
 
 /* Slot of the state arenas that holds bucket b's committed master/m/v. */
 so_status so_bucket_slot(const so_ctx *ctx, int32_t bucket, int32_t *slot);

@@ -73,8 +73,8 @@ _lib = None
 
 EXPORTS = ["so_layout_init", "so_layout_get_info", "so_layout_tensor", "so_layout_bind",
            "so_grad_check", "so_adam_step_speculative", "so_validate_commit_or_rollback",
-           "so_cast_params", "so_iteration_host", "so_grad_check_static", "so_loss_scale_config",
-           "so_get_loss_scale", "so_bucket_slot", "so_get_step", "so_set_step",
+           "so_validate_begin", "so_validate_poll", "so_cast_params", "so_iteration_host", "so_grad_check_static", "so_loss_scale_config",
+           "so_get_loss_scale", "so_state_export", "so_state_import", "so_bucket_slot", "so_get_step", "so_set_step",
            "so_pending_buckets", "so_get_counters", "so_last_cuda_error", "so_strerror",
            "so_destroy", "so_debug_set_dry_run", "so_debug_set_bucket_stats",
            "so_debug_set_step_variant"]
@@ -100,11 +100,15 @@ def lib() -> C.CDLL:
         "so_grad_check": [vp, P(so_hparams), i32, vp, P(so_grad_stats)],
         "so_adam_step_speculative": [vp, P(so_hparams), i32, vp],
         "so_validate_commit_or_rollback": [vp, P(so_hparams), vp, P(so_step_result)],
+        "so_validate_begin": [vp, P(so_hparams), vp],
+        "so_validate_poll": [vp, P(i32)],
         "so_cast_params": [vp, i32, vp],
         "so_iteration_host": [vp, P(so_hparams), vp, vp, vp, P(so_step_result)],
         "so_grad_check_static": [vp, i64, i32, dbl, vp, vp],
         "so_loss_scale_config": [vp, dbl, dbl, dbl, i64],
         "so_get_loss_scale": [vp, P(dbl)],
+        "so_state_export": [vp, vp, vp, vp, vp],
+        "so_state_import": [vp, vp, vp, vp, vp],
         "so_bucket_slot": [vp, i32, P(i32)],
         "so_get_step": [vp, P(i64)],
         "so_set_step": [vp, i64],
@@ -215,6 +219,17 @@ def so_validate_commit_or_rollback(ctx, hp, stream=None) -> so_step_result:
     return out
 
 
+def so_validate_begin(ctx, hp, stream=None) -> None:
+    h = _hp(hp)
+    _ok(ctx, lib().so_validate_begin(ctx, C.byref(h), _stream(stream)), "so_validate_begin")
+
+
+def so_validate_poll(ctx) -> bool:
+    ready = C.c_int32()
+    _ok(ctx, lib().so_validate_poll(ctx, C.byref(ready)), "so_validate_poll")
+    return bool(ready.value)
+
+
 def so_cast_params(ctx, bucket: int = SO_ALL, stream=None) -> None:
     _ok(ctx, lib().so_cast_params(ctx, bucket, _stream(stream)), "so_cast_params")
 
@@ -246,6 +261,18 @@ def so_get_loss_scale(ctx) -> float:
     s = C.c_double()
     _ok(ctx, lib().so_get_loss_scale(ctx, C.byref(s)), "so_get_loss_scale")
     return s.value
+
+
+def so_state_export(ctx, master: int, m: int, v: int, stream=None) -> None:
+    """Flat fp32 arrays (device or host addresses, 0 to skip) <- committed state."""
+    _ok(ctx, lib().so_state_export(ctx, master or None, m or None, v or None, _stream(stream)),
+        "so_state_export")
+
+
+def so_state_import(ctx, master: int, m: int, v: int, stream=None) -> None:
+    """Committed state <- flat fp32 arrays (device or host addresses, 0 to skip)."""
+    _ok(ctx, lib().so_state_import(ctx, master or None, m or None, v or None, _stream(stream)),
+        "so_state_import")
 
 
 def so_bucket_slot(ctx, bucket: int) -> int:

@@ -18,7 +18,7 @@ using namespace so;
 
 namespace {
 
-enum Phase { kIdle = 0, kOpen = 1, kChecked = 2 };
+enum Phase { kIdle = 0, kOpen = 1, kReducing = 2, kChecked = 3 };
 enum Cover : uint8_t { kNone = 0, kCheckedOnly = 1, kSpeculated = 2 };
 
 }  // namespace
@@ -47,6 +47,8 @@ struct so_ctx {
     uint32_t *d_arrivals = nullptr;     // per-bucket arrival counters of the reduction
     int64_t segs_per_slot = 1;
     int32_t reduce_seq = 0;             // stamp of the latest reduction (never 0)
+    cudaStream_t reduce_stream = nullptr;   // stream the reduction in flight was launched on
+    cudaEvent_t reduce_done = nullptr;  // completion of the copy-back when h_stats is not mapped
     int occ_step = 0, occ_check = 0, occ_cast = 0;
     // ---- slot map ----
     std::vector<int32_t> slot_of;       // committed slot of each bucket
@@ -317,10 +319,10 @@ so_status launch_casts(so_ctx *c, const std::vector<BucketEntry> &entries, cudaS
     return SO_OK;
 }
 
-// Finish the gradient check: scan what is still uncovered, fold per bucket on
-// the device, wait for the per-bucket records to reach the host, fold over
-// buckets in index order, derive norm and clip coefficient.
-so_status finalize_check(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
+// First half of finishing the gradient check: scan what is still uncovered and
+// launch the per-bucket reduction, whose records travel to the host on their
+// own.  Nothing here waits.
+so_status begin_check(so_ctx *c, cudaStream_t stream)
 {
     std::vector<int32_t> todo;
     for (int32_t b = 0; b < c->n_buckets; ++b)
@@ -331,6 +333,7 @@ so_status finalize_check(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
         for (int32_t b : todo) c->cover[b] = kCheckedOnly;
         c->n_covered = c->n_buckets;
     }
+    c->reduce_stream = stream;
     if (c->n_buckets > 0) {
         if (!c->dry_run) {
             ReduceArgs r;
@@ -349,38 +352,62 @@ so_status finalize_check(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
             const int64_t blocks = (int64_t)c->n_buckets * c->segs_per_slot;
             bucket_reduce_kernel<<<(unsigned)blocks, kReduceThreads, 0, stream>>>(r);
         }
-        so_status s = after_launch(c);
+        const so_status s = after_launch(c);
         if (s != SO_OK) return s;
+        if (!c->dry_run && !c->h_stats_dev) {
+            cudaError_t e = cudaMemcpyAsync(c->h_stats, c->d_stats,
+                                            sizeof(BucketStats) * (size_t)(c->n_buckets + 1),
+                                            cudaMemcpyDeviceToHost, stream);
+            if (e == cudaSuccess && !c->reduce_done)
+                e = cudaEventCreateWithFlags(&c->reduce_done, cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventRecord(c->reduce_done, stream);
+            if (e != cudaSuccess) return cuda_fail(c, e);
+        }
+    }
+    c->phase = kReducing;
+    return SO_OK;
+}
+
+// Have the records of the reduction in flight reached the host?  Never blocks.
+bool check_arrived(so_ctx *c)
+{
+    if (c->dry_run || c->n_buckets == 0) return true;
+    if (c->h_stats_dev) {
+        const volatile int32_t *stamp = &c->h_stats[c->n_buckets].pad;
+        return *stamp == c->reduce_seq;
+    }
+    return cudaEventQuery(c->reduce_done) == cudaSuccess;
+}
+
+// Second half: wait for the per-bucket records to reach the host, fold over
+// buckets in index order, derive norm and clip coefficient.
+so_status finish_check(so_ctx *c, const so_hparams &hp)
+{
+    if (c->n_buckets > 0) {
         if (!c->dry_run) {
             cudaError_t e = cudaSuccess;
-            if (!c->h_stats_dev)
-                e = cudaMemcpyAsync(c->h_stats, c->d_stats,
-                                    sizeof(BucketStats) * (size_t)(c->n_buckets + 1),
-                                    cudaMemcpyDeviceToHost, stream);
-            if (e != cudaSuccess) return cuda_fail(c, e);
             if (c->h_stats_dev) {
                 // The records arrive in mapped host memory; watching for the
                 // stamp that follows them is several microseconds quicker than
                 // waiting for the stream's completion to be signalled.  Bounded:
                 // after two seconds fall back to a stream synchronisation, which
                 // also surfaces any launch or execution error.
-                volatile int32_t *stamp = &c->h_stats[c->n_buckets].pad;
                 const auto t0 = std::chrono::steady_clock::now();
                 bool arrived = false;
                 for (uint32_t spins = 0;; ++spins) {
-                    if (*stamp == c->reduce_seq) { arrived = true; break; }
+                    if (check_arrived(c)) { arrived = true; break; }
                     if ((spins & 0xFFFu) == 0xFFFu &&
                         std::chrono::steady_clock::now() - t0 > std::chrono::seconds(2))
                         break;
                 }
                 std::atomic_thread_fence(std::memory_order_acquire);
                 if (!arrived) {
-                    e = cudaStreamSynchronize(stream);
+                    e = cudaStreamSynchronize(c->reduce_stream);
                     if (e != cudaSuccess) return cuda_fail(c, e);
-                    if (*stamp != c->reduce_seq) return cuda_fail(c, cudaErrorUnknown);
+                    if (!check_arrived(c)) return cuda_fail(c, cudaErrorUnknown);
                 }
             } else {
-                e = cudaStreamSynchronize(stream);
+                e = cudaStreamSynchronize(c->reduce_stream);
                 if (e != cudaSuccess) return cuda_fail(c, e);
             }
             int32_t device_status = c->h_stats[c->n_buckets].nonfinite;
@@ -389,7 +416,7 @@ so_status finalize_check(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
             if (device_status != 0) {
                 // a kernel gave up waiting for one of its own copies; its tile
                 // counters may be left mid-way, so re-arm the whole control block
-                cudaMemsetAsync(c->d_ctrl, 0, sizeof(ControlBlock), stream);
+                cudaMemsetAsync(c->d_ctrl, 0, sizeof(ControlBlock), c->reduce_stream);
                 if (c->h_stats_dev) std::memset(&c->h_stats[c->n_buckets], 0, sizeof(BucketStats));
                 return SO_ERR_TIMEOUT;
             }
@@ -410,6 +437,15 @@ so_status finalize_check(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
     c->stats.reserved = 0;
     c->phase = kChecked;
     return SO_OK;
+}
+
+so_status finalize_check(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
+{
+    if (c->phase != kReducing) {
+        const so_status s = begin_check(c, stream);
+        if (s != SO_OK) return s;
+    }
+    return finish_check(c, hp);
 }
 
 void end_iteration(so_ctx *c)
@@ -627,6 +663,7 @@ so_status so_grad_check(so_ctx *c, const so_hparams *hp, int32_t bucket, void *s
     if (!c) return SO_ERR_INVALID_ARG;
     if (!c->bound) return SO_ERR_STATE;
     if (c->phase == kChecked) return SO_ERR_STATE;
+    if (c->phase == kReducing && bucket != SO_ALL) return SO_ERR_STATE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (bucket == SO_ALL) {
         so_status s = note_hparams(c, hp);
@@ -651,7 +688,7 @@ so_status so_adam_step_speculative(so_ctx *c, const so_hparams *hp, int32_t buck
 {
     if (!c) return SO_ERR_INVALID_ARG;
     if (!c->bound) return SO_ERR_STATE;
-    if (c->phase == kChecked) return SO_ERR_STATE;
+    if (c->phase == kChecked || c->phase == kReducing) return SO_ERR_STATE;
     so_status s = note_hparams(c, hp);
     if (s != SO_OK) return s;
     if (bucket != SO_ALL && (bucket < 0 || bucket >= c->n_buckets)) return SO_ERR_INVALID_ARG;
@@ -762,6 +799,28 @@ so_status so_validate_commit_or_rollback(so_ctx *c, const so_hparams *hp, void *
         out->loss_scale = c->loss_scale;
     }
     end_iteration(c);
+    return SO_OK;
+}
+
+so_status so_validate_begin(so_ctx *c, const so_hparams *hp, void *stream)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (!c->bound) return SO_ERR_STATE;
+    if (c->phase == kChecked || c->phase == kReducing) return SO_ERR_STATE;
+    so_status s = note_hparams(c, hp);
+    if (s != SO_OK) return s;
+    s = begin_check(c, static_cast<cudaStream_t>(stream));
+    if (s != SO_OK) return s;
+    if (!c->have_hp) { c->hp_iter = *hp; c->have_hp = true; }
+    return SO_OK;
+}
+
+so_status so_validate_poll(so_ctx *c, int32_t *ready)
+{
+    if (!c || !ready) return SO_ERR_INVALID_ARG;
+    if (c->phase == kChecked) { *ready = 1; return SO_OK; }
+    if (c->phase != kReducing) return SO_ERR_STATE;
+    *ready = check_arrived(c) ? 1 : 0;
     return SO_OK;
 }
 
@@ -893,6 +952,51 @@ so_status so_get_loss_scale(const so_ctx *c, double *scale)
     return SO_OK;
 }
 
+namespace {
+
+// Copy the committed fp32 state between the slot arenas and flat arrays in
+// parameter order, one asynchronous copy per bucket and array.
+so_status copy_state(so_ctx *c, void *flat[3], bool to_flat, cudaStream_t stream)
+{
+    float *arenas[3] = {c->master, c->mom, c->var};
+    for (int32_t b = 0; b < c->n_buckets; ++b) {
+        const size_t n = (size_t)elems_of(c, b);
+        const size_t flat_off = (size_t)b * (size_t)c->bucket_elems;
+        const size_t slot_off = (size_t)c->slot_of[b] * (size_t)c->stride;
+        for (int k = 0; k < 3; ++k) {
+            if (!flat[k]) continue;
+            float *in_arena = arenas[k] + slot_off;
+            float *in_flat = static_cast<float *>(flat[k]) + flat_off;
+            const cudaError_t e = cudaMemcpyAsync(to_flat ? in_flat : in_arena,
+                                                  to_flat ? in_arena : in_flat, n * sizeof(float),
+                                                  cudaMemcpyDefault, stream);
+            if (e != cudaSuccess) return cuda_fail(c, e);
+        }
+    }
+    return SO_OK;
+}
+
+}  // namespace
+
+so_status so_state_export(so_ctx *c, void *master, void *m, void *v, void *stream)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (!c->bound || c->phase != kIdle) return SO_ERR_STATE;
+    if (c->dry_run) return SO_ERR_UNSUPPORTED;
+    void *flat[3] = {master, m, v};
+    return copy_state(c, flat, /*to_flat=*/true, static_cast<cudaStream_t>(stream));
+}
+
+so_status so_state_import(so_ctx *c, const void *master, const void *m, const void *v,
+                          void *stream)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (!c->bound || c->phase != kIdle) return SO_ERR_STATE;
+    if (c->dry_run) return SO_ERR_UNSUPPORTED;
+    void *flat[3] = {const_cast<void *>(master), const_cast<void *>(m), const_cast<void *>(v)};
+    return copy_state(c, flat, /*to_flat=*/false, static_cast<cudaStream_t>(stream));
+}
+
 so_status so_bucket_slot(const so_ctx *c, int32_t bucket, int32_t *slot)
 {
     if (!c || !slot || bucket < 0 || bucket >= c->n_buckets) return SO_ERR_INVALID_ARG;
@@ -951,6 +1055,7 @@ void so_destroy(so_ctx *c)
 {
     if (!c) return;
     for (cudaEvent_t ev : c->events) cudaEventDestroy(ev);
+    if (c->reduce_done) cudaEventDestroy(c->reduce_done);
     if (c->copy_in) cudaStreamDestroy(c->copy_in);
     if (c->copy_out) cudaStreamDestroy(c->copy_out);
     if (c->h_stats) {

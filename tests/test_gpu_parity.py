@@ -334,3 +334,70 @@ def test_fp16_static_scale_register_variant_and_check_first_flow():
     b, _ = run_lockstep(w, steps=4, undo_slots=0, speculative=False)
     assert a.decisions == b.decisions == [R] * 4
     assert a.loss_scales == b.loss_scales == [2.0 ** 12] * 4
+
+
+# ---------------------------------------------------------------------------
+# validation off the critical path; checkpoint and resume
+# ---------------------------------------------------------------------------
+
+def test_deferred_validation_gives_the_same_bits():
+    """so_validate_begin, other work on the stream (a stand-in for the next
+    forward pass), then the verdict: identical to validating at once."""
+    w = W.tiny()
+    hp = hparams_of(w)
+    stream = torch.cuda.current_stream()
+    ref = _run_device_only(w, 8, undo_slots=B.SO_ALL, speculative=True)
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, B.SO_ALL)
+    opt.load_state(W.initial_master(w, device="cuda"))
+    opt.cast_params(stream=stream)
+    a = torch.randn(2048, 2048, device="cuda")
+    trace = []
+    for step in range(1, 9):
+        opt.load_grads(W.gradients(w, step, device="cuda"))
+        opt.step_speculative(hp, B.SO_ALL, stream)
+        B.so_validate_begin(opt.ctx, hp, stream)
+        for _ in range(4):
+            a = torch.tanh(a @ a.t() * 1e-3)                 # "forward pass" behind the reduction
+        polls = 0
+        while not B.so_validate_poll(opt.ctx):
+            polls += 1
+            assert polls < 10_000_000
+        res = opt.validate(hp, stream)
+        trace.append((res.decision, res.stats.sumsq, res.stats.norm, res.stats.clip_coef,
+                      res.stats.nonfinite, res.step_after))
+    torch.cuda.synchronize()
+    assert trace == ref[0] and _state_bytes(opt) == ref[1]
+
+
+def test_checkpoint_export_import_resumes_bit_for_bit():
+    w = W.tiny_ragged()
+    hp = hparams_of(w)
+    stream = torch.cuda.current_stream()
+    straight = _run_device_only(w, 6, undo_slots=B.SO_ALL, speculative=True)
+
+    first = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, B.SO_ALL)
+    first.load_state(W.initial_master(w, device="cuda"))
+    first.cast_params(stream=stream)
+    for step in (1, 2, 3):
+        first.load_grads(W.gradients(w, step, device="cuda"))
+        first.iteration(hp, stream=stream)
+    n = w.total
+    ckpt = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(2)]
+    host_v = torch.empty(n, dtype=torch.float32, pin_memory=True)      # one array via the host
+    B.so_state_export(first.ctx, ckpt[0].data_ptr(), ckpt[1].data_ptr(), host_v.data_ptr(), stream)
+    torch.cuda.synchronize()
+    t = first.step_count
+    gathered = first.gather_state()
+    assert torch.equal(ckpt[0], gathered[0]) and torch.equal(ckpt[1], gathered[1])
+    assert torch.equal(host_v.cuda(), gathered[2])
+
+    second = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, 2)    # a different undo window
+    B.so_state_import(second.ctx, ckpt[0].data_ptr(), ckpt[1].data_ptr(), host_v.data_ptr(), stream)
+    B.so_set_step(second.ctx, t)
+    second.cast_params(stream=stream)
+    for step in (4, 5, 6):
+        second.load_grads(W.gradients(w, step, device="cuda"))
+        second.iteration(hp, stream=stream)
+    torch.cuda.synchronize()
+    assert second.step_count == straight[0][-1][5]
+    assert _state_bytes(second) == straight[1]

@@ -304,3 +304,25 @@ def test_loss_scale_is_only_for_fp16_contexts_and_validates_its_arguments():
     B.so_adam_step_speculative(ctx, HP(), 0)
     assert _status(B.so_loss_scale_config, ctx, 2048.0) == B.SO_ERR_STATE        # mid-iteration
     B.so_destroy(ctx)
+
+
+def test_deferred_validation_state_machine():
+    ctx, _ = _dry_ctx([1000], 256)
+    hp = HP(max_grad_norm=0.0)
+    assert _status(B.so_validate_poll, ctx) == B.SO_ERR_STATE           # nothing in flight
+    B.so_adam_step_speculative(ctx, hp, 0)
+    B.so_validate_begin(ctx, hp)                                         # scans buckets 1..3
+    assert B.so_get_counters(ctx).elems_checked == 1000 - 256
+    assert B.so_validate_poll(ctx) is True
+    assert _status(B.so_adam_step_speculative, ctx, hp, 1) == B.SO_ERR_STATE
+    assert _status(B.so_grad_check, ctx, None, 1) == B.SO_ERR_STATE
+    assert _status(B.so_validate_begin, ctx, hp) == B.SO_ERR_STATE       # already begun
+    st = B.so_grad_check(ctx, hp, B.SO_ALL)                              # finishing is allowed
+    assert st.nonfinite == 0
+    assert B.so_validate_poll(ctx) is True
+    r = B.so_validate_commit_or_rollback(ctx, hp)
+    assert r.decision == B.SO_DECISION_COMMIT and r.step_after == 1
+    B.so_validate_begin(ctx, hp)                                         # check-first flow, deferred
+    r = B.so_validate_commit_or_rollback(ctx, hp)
+    assert r.step_after == 2 and r.buckets_speculated == 0
+    B.so_destroy(ctx)
