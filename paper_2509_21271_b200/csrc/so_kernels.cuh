@@ -198,6 +198,16 @@ __device__ __forceinline__ void store_quad_bf16(uint16_t *base, uint32_t idx, ui
     }
 }
 
+// Sum of a tile, fixed order.  A lane keeps four running sums, one per
+// position in its quad, each advanced in row order (four independent chains
+// instead of one 32-long one: the adds have a long latency); they are combined
+// as (s0 + s1) + (s2 + s3) and then folded across the warp with an xor tree.
+__device__ __forceinline__ double warp_fold(double x);
+__device__ __forceinline__ double tile_fold(const double (&acc)[4])
+{
+    return warp_fold(__dadd_rn(__dadd_rn(acc[0], acc[1]), __dadd_rn(acc[2], acc[3])));
+}
+
 // Fold a per-lane double across the warp with a fixed xor tree.
 __device__ __forceinline__ double warp_fold(double x)
 {
@@ -306,7 +316,7 @@ __global__ void __launch_bounds__(kThreads, 2) adamw_step_kernel(const __grid_co
         float *p_out = a.master + dst, *m_out = a.mom + dst, *v_out = a.var + dst;
         uint16_t *pb = a.param_bf16 + (int64_t)e.bucket * a.geo.stride;
 
-        double acc = 0.0;
+        double acc[4] = {0.0, 0.0, 0.0, 0.0};
 #pragma unroll 1
         for (int r0 = 0; r0 < kRowsPerTile; r0 += kRowsInFlight) {
             if (base + r0 * kRowElems >= n) break;
@@ -325,7 +335,7 @@ __global__ void __launch_bounds__(kThreads, 2) adamw_step_kernel(const __grid_co
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     adamw_element<!kSpec, grad_traits<GradT>::kUnscale>(gq[u][q], pq[u][q], mq[u][q],
-                                                                         vq[u][q], a.k, acc);
+                                                                         vq[u][q], a.k, acc[q]);
                 const uint32_t idx = base + (r0 + u) * kRowElems + lane * 4;
                 if (idx < n) {
                     store_quad(p_out, idx, n, pq[u]);
@@ -336,56 +346,98 @@ __global__ void __launch_bounds__(kThreads, 2) adamw_step_kernel(const __grid_co
             }
         }
         if (kSpec) {
-            acc = warp_fold(acc);
-            if (lane == 0) a.partials[(int64_t)e.bucket * tps + lt] = acc;
+            const double tile_sum = tile_fold(acc);
+            if (lane == 0) a.partials[(int64_t)e.bucket * tps + lt] = tile_sum;
         }
     }
 }
 
 // ---------------------------------------------------------------------------
 // stand-alone gradient scan: tile sums of g^2 (same order as the fused kernel)
-// ---------------------------------------------------------------------------
+// ---------------------------------------------------------------------------//
+// Read-only, 2 (4) bytes per element: all that matters is bytes in flight.  A
+// warp keeps the eight row loads of its *next* tile in flight while it sums the
+// current one (two register buffers of raw quads).
+template <typename GradT> struct raw_quad { typedef uint2 type; };
+template <> struct raw_quad<float> { typedef float4 type; };
+
+template <typename GradT>
+__device__ __forceinline__ void unpack_quad(const typename raw_quad<GradT>::type &q, float (&x)[4])
+{
+    if constexpr (sizeof(GradT) == 2) {
+        unpack2<GradT>(q.x, x[0], x[1]);
+        unpack2<GradT>(q.y, x[2], x[3]);
+    } else {
+        x[0] = q.x; x[1] = q.y; x[2] = q.z; x[3] = q.w;
+    }
+}
+
+struct CheckTile { uint32_t n, base, lt; int32_t bucket; bool valid; };
+
 template <typename GradT>
 __global__ void __launch_bounds__(kThreads) grad_check_kernel(const __grid_constant__ CheckArgs a)
 {
+    using Raw = typename raw_quad<GradT>::type;
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     const uint32_t tps = a.geo.tiles_per_slot;
     const uint32_t total_tiles = (uint32_t)a.n_entries * tps;
 
-    for (uint32_t tile = warp; tile < total_tiles; tile += n_warps) {
-        const uint32_t j = tile / tps;
-        const uint32_t lt = tile - j * tps;
-        const int32_t b = a.bucket[j];
-        const uint32_t n = (b == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
-        const uint32_t base = lt * kTileElems;
-        if (base >= n) continue;
-        const GradT *g = static_cast<const GradT *>(a.grad) + (int64_t)b * a.geo.stride;
-
-        float gq[kRowsPerTile][4];
-#pragma unroll
-        for (int r = 0; r < kRowsPerTile; ++r) {
-            const uint32_t idx = base + r * kRowElems + lane * 4;
-            if (idx < n) {
-                load_quad(g, idx, n, gq[r]);
-            } else {
-                gq[r][0] = gq[r][1] = gq[r][2] = gq[r][3] = 0.0f;
+    // first tile at or after `tile` (stepping by n_warps) that lies inside its bucket
+    auto seek = [&](uint32_t tile, CheckTile &t) {
+        for (; tile < total_tiles; tile += n_warps) {
+            const uint32_t j = tile / tps;
+            const uint32_t lt = tile - j * tps;
+            const int32_t b = a.bucket[j];
+            const uint32_t n = (b == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
+            if (lt * kTileElems < n) {
+                t.n = n; t.base = lt * kTileElems; t.lt = lt; t.bucket = b; t.valid = true;
+                return tile;
             }
         }
-        double acc = 0.0;
+        t.valid = false;
+        return tile;
+    };
+    // issue the vector loads of a tile's full quads (ragged ends are read later, guarded)
+    auto prefetch = [&](const CheckTile &t, Raw (&raw)[kRowsPerTile]) {
+        const GradT *g = static_cast<const GradT *>(a.grad) + (int64_t)t.bucket * a.geo.stride;
 #pragma unroll
         for (int r = 0; r < kRowsPerTile; ++r) {
+            const uint32_t idx = t.base + r * kRowElems + lane * 4;
+            if (idx + 4 <= t.n) raw[r] = __ldcs(reinterpret_cast<const Raw *>(g + idx));
+        }
+    };
+
+    CheckTile cur, nxt;
+    Raw buf_cur[kRowsPerTile], buf_nxt[kRowsPerTile];
+    uint32_t tile = seek(warp, cur);
+    if (cur.valid) prefetch(cur, buf_cur);
+    while (cur.valid) {
+        tile = seek(tile + n_warps, nxt);
+        if (nxt.valid) prefetch(nxt, buf_nxt);
+
+        const GradT *g = static_cast<const GradT *>(a.grad) + (int64_t)cur.bucket * a.geo.stride;
+        double acc[4] = {0.0, 0.0, 0.0, 0.0};
+#pragma unroll
+        for (int r = 0; r < kRowsPerTile; ++r) {
+            const uint32_t idx = cur.base + r * kRowElems + lane * 4;
+            float x[4];
+            if (idx + 4 <= cur.n) unpack_quad<GradT>(buf_cur[r], x);
+            else load_quad(g, idx, cur.n, x);               // guarded: zeros past the end
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                const double gd = grad_traits<GradT>::kUnscale
-                                      ? __dmul_rn((double)gq[r][q], a.unscale)
-                                      : (double)gq[r][q];
-                acc = __dadd_rn(acc, __dmul_rn(gd, gd));
+                const double gd = grad_traits<GradT>::kUnscale ? __dmul_rn((double)x[q], a.unscale)
+                                                               : (double)x[q];
+                acc[q] = __dadd_rn(acc[q], __dmul_rn(gd, gd));
             }
         }
-        acc = warp_fold(acc);
-        if (lane == 0) a.partials[(int64_t)b * tps + lt] = acc;
+        const double tile_sum = tile_fold(acc);
+        if (lane == 0) a.partials[(int64_t)cur.bucket * tps + cur.lt] = tile_sum;
+
+        cur = nxt;
+#pragma unroll
+        for (int r = 0; r < kRowsPerTile; ++r) buf_cur[r] = buf_nxt[r];
     }
 }
 

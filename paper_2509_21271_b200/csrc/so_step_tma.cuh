@@ -285,7 +285,7 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
 
     uint32_t phases = 0;               // parity bit per input stage
     int stage = 0, ostage = 0;
-    double acc = 0.0;
+    double acc[4] = {0.0, 0.0, 0.0, 0.0};
     bool failed = false;
 
 #pragma unroll 1
@@ -333,7 +333,7 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     adamw_element<!kSpec, grad_traits<GradT>::kUnscale>(gq[q], pq[q], mq[q], vq[q],
-                                                                         a.k, acc);
+                                                                         a.k, acc[q]);
                 *reinterpret_cast<float4 *>(out + off * 4) = make_float4(pq[0], pq[1], pq[2], pq[3]);
                 *reinterpret_cast<float4 *>(out + L::kF32Bytes + off * 4) =
                     make_float4(mq[0], mq[1], mq[2], mq[3]);
@@ -371,7 +371,7 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
                     adamw_element<!kSpec, grad_traits<GradT>::kUnscale>(gq[q], pq[q], mq[q], vq[q],
-                                                                         a.k, acc);
+                                                                         a.k, acc[q]);
                 if (idx < d.n) {
                     store_quad(a.master + dst, idx, d.n, pq);
                     store_quad(a.mom + dst, idx, d.n, mq);
@@ -385,10 +385,10 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
 
         if (d.flags & kLastOfTile) {
             if (kSpec) {
-                const double tile_sum = warp_fold(acc);
+                const double tile_sum = tile_fold(acc);
                 if (lane == 0) a.partials[(int64_t)d.bucket * tps + d.tile_in_bucket] = tile_sum;
             }
-            acc = 0.0;
+            acc[0] = acc[1] = acc[2] = acc[3] = 0.0;
         }
         stage = (stage + 1 == kStagesIn) ? 0 : stage + 1;
     }
