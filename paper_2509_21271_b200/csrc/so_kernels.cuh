@@ -8,14 +8,15 @@
 // and no block-level synchronisation at all (the reduction is per warp).
 //
 // Work decomposition.  A bucket is cut into *tiles* of 1024 consecutive
-// elements; one warp owns one tile at a time (tiles are dealt round-robin to
-// all warps of the grid).  Inside a tile a warp sweeps 8 *rows* of 128
+// elements; one warp owns one tile at a time (dealt round-robin to all warps
+// of the grid here, claimed from a counter in the bulk-copy step kernel).  Inside a tile a warp sweeps 8 *rows* of 128
 // elements; lane l owns the *quad* of elements [4l, 4l+4) of each row, so a
 // warp-wide fp32 access is one contiguous 512-byte line set and a bf16 access
 // one contiguous 256-byte one.  The sum of squares of a tile is accumulated
-// per lane in row order, then folded across lanes with an xor-shuffle tree and
-// stored as one double per tile; a second tiny kernel folds the tiles of each
-// bucket in a fixed order.  The summation order therefore depends on nothing
+// per lane in four chains (one per quad position, each in row order), combined
+// pairwise, folded across lanes with an xor-shuffle tree and stored as one
+// double per tile; a second tiny kernel folds the tiles of each bucket in a
+// fixed order.  The summation order therefore depends on nothing
 // but the data and the bucket geometry: the same bits come out whatever the
 // grid size, and whether the sums were produced by the fused step kernel or by
 // the stand-alone check kernel.
@@ -43,7 +44,6 @@ struct Geometry {
     int32_t last_bucket;                  // its index (-1 if none)
 };
 
-// Per-step constants, all derived on the host in double precision.
 // Gradient element types: uint16_t carries bf16 bit patterns, half_t IEEE
 // binary16 bit patterns (the only type that is used with a loss scale), float
 // plain fp32.
@@ -52,6 +52,7 @@ struct half_t { uint16_t bits; };
 template <typename GradT> struct grad_traits { static constexpr bool kUnscale = false; };
 template <> struct grad_traits<half_t> { static constexpr bool kUnscale = true; };
 
+// Per-step constants, all derived on the host in double precision.
 struct AdamScalars {
     double beta1, omb1;                   // beta1, 1 - beta1
     double beta2, omb2;
