@@ -224,6 +224,19 @@ so_status so_validate_begin(so_ctx *ctx, const so_hparams *hp, void *stream);
 so_status so_validate_poll(so_ctx *ctx, int32_t *ready);
 
 /*
+ * so_set_global_grad_stats -- the hook for sharded optimizer states (Section
+ * 4.7: with ZeRO-style partitioning each process updates only its own subset
+ * of the parameters).  The norm and the NaN/Inf check are global quantities:
+ * a process that holds a shard calls so_grad_check(SO_ALL) to get its LOCAL
+ * sum of squares and flag, combines them with the other shards' (one 16-byte
+ * all-reduce: sum of the sums, OR of the flags), hands the result back here,
+ * and then calls so_validate_commit_or_rollback, which decides and acts on the
+ * global values.  Only after so_grad_check(SO_ALL) and before validation
+ * (SO_ERR_STATE otherwise).  Host-only.
+ */
+so_status so_set_global_grad_stats(so_ctx *ctx, double global_sumsq, int32_t global_nonfinite);
+
+/*
  * so_cast_params -- fp32 master -> bf16 parameter copy, round to nearest even
  * (Section 4.5: the cast runs on the GPU).  bucket >= 0 or SO_ALL.  Only
  * between iterations (SO_ERR_STATE while buckets are covered).  Enqueues only.

@@ -73,7 +73,7 @@ _lib = None
 
 EXPORTS = ["so_layout_init", "so_layout_get_info", "so_layout_tensor", "so_layout_bind",
            "so_grad_check", "so_adam_step_speculative", "so_validate_commit_or_rollback",
-           "so_validate_begin", "so_validate_poll", "so_cast_params", "so_iteration_host", "so_grad_check_static", "so_loss_scale_config",
+           "so_validate_begin", "so_validate_poll", "so_set_global_grad_stats", "so_cast_params", "so_iteration_host", "so_grad_check_static", "so_loss_scale_config",
            "so_get_loss_scale", "so_state_export", "so_state_import", "so_bucket_slot", "so_get_step", "so_set_step",
            "so_pending_buckets", "so_get_counters", "so_last_cuda_error", "so_strerror",
            "so_destroy", "so_debug_set_dry_run", "so_debug_set_bucket_stats",
@@ -102,6 +102,7 @@ def lib() -> C.CDLL:
         "so_validate_commit_or_rollback": [vp, P(so_hparams), vp, P(so_step_result)],
         "so_validate_begin": [vp, P(so_hparams), vp],
         "so_validate_poll": [vp, P(i32)],
+        "so_set_global_grad_stats": [vp, dbl, i32],
         "so_cast_params": [vp, i32, vp],
         "so_iteration_host": [vp, P(so_hparams), vp, vp, vp, P(so_step_result)],
         "so_grad_check_static": [vp, i64, i32, dbl, vp, vp],
@@ -228,6 +229,11 @@ def so_validate_poll(ctx) -> bool:
     ready = C.c_int32()
     _ok(ctx, lib().so_validate_poll(ctx, C.byref(ready)), "so_validate_poll")
     return bool(ready.value)
+
+
+def so_set_global_grad_stats(ctx, global_sumsq: float, global_nonfinite: int) -> None:
+    _ok(ctx, lib().so_set_global_grad_stats(ctx, global_sumsq, int(global_nonfinite)),
+        "so_set_global_grad_stats")
 
 
 def so_cast_params(ctx, bucket: int = SO_ALL, stream=None) -> None:

@@ -298,7 +298,10 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
         uint16_t *pb = a.param_bf16 + (int64_t)d.bucket * stride;
 
         if (bulk) {
-            if (!mbar_wait_bounded(bars + stage * 8, (phases >> stage) & 1u)) {
+            // every lane polls the same barrier; the verdict is made warp-wide so
+            // that no lane leaves the loop while others go on to a __syncwarp
+            if (!__all_sync(0xFFFFFFFFu,
+                            mbar_wait_bounded(bars + stage * 8, (phases >> stage) & 1u))) {
                 failed = true;
                 break;
             }

@@ -815,6 +815,18 @@ so_status so_validate_begin(so_ctx *c, const so_hparams *hp, void *stream)
     return SO_OK;
 }
 
+so_status so_set_global_grad_stats(so_ctx *c, double global_sumsq, int32_t global_nonfinite)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (c->phase != kChecked) return SO_ERR_STATE;
+    if (std::isnan(global_sumsq) ? false : global_sumsq < 0.0) return SO_ERR_INVALID_ARG;
+    c->stats.sumsq = global_sumsq;
+    c->stats.norm = std::sqrt(global_sumsq);
+    c->stats.nonfinite = (global_nonfinite != 0 || !std::isfinite(global_sumsq)) ? 1 : 0;
+    c->stats.clip_coef = clip_coef_of(c->stats.norm, c->hp_iter.max_grad_norm);
+    return SO_OK;
+}
+
 so_status so_validate_poll(so_ctx *c, int32_t *ready)
 {
     if (!c || !ready) return SO_ERR_INVALID_ARG;
@@ -870,8 +882,8 @@ so_status so_iteration_host(so_ctx *c, const so_hparams *hp, const void *host_gr
     // the copy streams start after whatever the caller queued on `stream`
     e = cudaEventRecord(start, main);
     if (e != cudaSuccess) return cuda_fail(c, e);
-    cudaStreamWaitEvent(c->copy_in, start, 0);
-    cudaStreamWaitEvent(c->copy_out, start, 0);
+    if ((e = cudaStreamWaitEvent(c->copy_in, start, 0)) != cudaSuccess) return cuda_fail(c, e);
+    if ((e = cudaStreamWaitEvent(c->copy_out, start, 0)) != cudaSuccess) return cuda_fail(c, e);
 
     for (int32_t b = 0; b < c->n_buckets; ++b) {
         const size_t n = (size_t)elems_of(c, b);
@@ -879,8 +891,8 @@ so_status so_iteration_host(so_ctx *c, const so_hparams *hp, const void *host_gr
                             hg + (size_t)b * (size_t)c->bucket_elems * gsz, n * gsz,
                             cudaMemcpyHostToDevice, c->copy_in);
         if (e != cudaSuccess) return cuda_fail(c, e);
-        cudaEventRecord(c->events[2 * b], c->copy_in);
-        cudaStreamWaitEvent(main, c->events[2 * b], 0);
+        if ((e = cudaEventRecord(c->events[2 * b], c->copy_in)) != cudaSuccess) return cuda_fail(c, e);
+        if ((e = cudaStreamWaitEvent(main, c->events[2 * b], 0)) != cudaSuccess) return cuda_fail(c, e);
         so_status s;
         bool speculated = false;
         if (!c->free_slots.empty()) {
@@ -891,8 +903,8 @@ so_status so_iteration_host(so_ctx *c, const so_hparams *hp, const void *host_gr
         }
         if (s != SO_OK) return s;
         if (speculated && hp_out) {
-            cudaEventRecord(c->events[2 * b + 1], main);
-            cudaStreamWaitEvent(c->copy_out, c->events[2 * b + 1], 0);
+            if ((e = cudaEventRecord(c->events[2 * b + 1], main)) != cudaSuccess) return cuda_fail(c, e);
+            if ((e = cudaStreamWaitEvent(c->copy_out, c->events[2 * b + 1], 0)) != cudaSuccess) return cuda_fail(c, e);
             e = cudaMemcpyAsync(hp_out + (size_t)b * (size_t)c->bucket_elems * 2,
                                 c->param_bf16 + (size_t)b * (size_t)c->stride, n * 2,
                                 cudaMemcpyDeviceToHost, c->copy_out);
@@ -905,8 +917,8 @@ so_status so_iteration_host(so_ctx *c, const so_hparams *hp, const void *host_gr
     if (s != SO_OK) return s;
     if (hp_out) {
         // whatever validation (re)wrote after the speculative copies went out
-        cudaEventRecord(start, main);
-        cudaStreamWaitEvent(c->copy_out, start, 0);
+        if ((e = cudaEventRecord(start, main)) != cudaSuccess) return cuda_fail(c, e);
+        if ((e = cudaStreamWaitEvent(c->copy_out, start, 0)) != cudaSuccess) return cuda_fail(c, e);
         for (int32_t b = 0; b < c->n_buckets; ++b) {
             const bool sent = was_speculated[b] == kSpeculated;
             if (sent && res.decision == SO_DECISION_COMMIT) continue;
