@@ -401,3 +401,45 @@ def test_checkpoint_export_import_resumes_bit_for_bit():
     torch.cuda.synchronize()
     assert second.step_count == straight[0][-1][5]
     assert _state_bytes(second) == straight[1]
+
+
+# ---------------------------------------------------------------------------
+# launch structure: batches of more than 128 buckets, several streams
+# ---------------------------------------------------------------------------
+
+def test_three_hundred_small_buckets_lockstep():
+    """301 buckets of 4096 elements: a batched call splits into three launches
+    (128 buckets each at most), each with its own tile counter."""
+    w = W.Workload(name="many_buckets", numel=[300 * 4096 + 17], bucket_elems=4096,
+                   sigma_g=1e-2, steps=4,
+                   faults=(W.Fault(step=3, flat_index=200 * 4096 + 5, kind="nan"),))
+    rep, opt = run_lockstep(w, steps=4)
+    assert opt.n_buckets == 301 and rep.decisions == [R, R, S, R]
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+
+
+def test_per_bucket_launches_on_two_streams_give_the_same_bits():
+    """Buckets stepped one call at a time, alternating between two streams whose
+    kernels may overlap on the GPU (each launch claims tiles from its own
+    counter), against the single batched launch."""
+    w = W.tiny_ragged()
+    hp = hparams_of(w)
+    ref = _run_device_only(w, 6, undo_slots=B.SO_ALL, speculative=True)
+    main = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, B.SO_ALL)
+    opt.load_state(W.initial_master(w, device="cuda"))
+    opt.cast_params(stream=main)
+    trace = []
+    for step in range(1, 7):
+        opt.load_grads(W.gradients(w, step, device="cuda"))
+        side.wait_stream(main)
+        for b in range(opt.n_buckets):
+            opt.step_speculative(hp, b, side if b % 2 else main)
+        main.wait_stream(side)
+        res = opt.validate(hp, main)
+        side.wait_stream(main)                      # re-steps / re-casts finish before reuse
+        trace.append((res.decision, res.stats.sumsq, res.stats.norm, res.stats.clip_coef,
+                      res.stats.nonfinite, res.step_after))
+    torch.cuda.synchronize()
+    assert trace == ref[0] and _state_bytes(opt) == ref[1]
