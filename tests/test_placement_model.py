@@ -1,0 +1,50 @@
+"""The paper's closed-form models (Eq. 1-5) against the one number it states
+for them and against hand arithmetic."""
+from __future__ import annotations
+
+import os
+
+import pytest
+
+from paper_2509_21271_b200 import placement_model as M
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "efficiency_statement.txt")
+
+
+def _golden():
+    out = {}
+    with open(GOLDEN) as fh:
+        for line in fh:
+            parts = line.split("#")[0].split()
+            if len(parts) == 2:
+                out[parts[0]] = float(parts[1])
+    return out
+
+
+def test_batch_four_is_the_first_to_pass_sixty_percent():
+    g = _golden()
+    b = M.min_batch_for_efficiency(g["target"], g["seq"], g["peak_flops"], g["link_bytes_per_s"])
+    assert b == int(g["min_batch"])
+    e3 = M.forward_efficiency(7e9, 3, g["seq"], g["peak_flops"], g["link_bytes_per_s"])
+    e4 = M.forward_efficiency(7e9, 4, g["seq"], g["peak_flops"], g["link_bytes_per_s"])
+    assert e3 < 0.60 < e4
+    # Eq. 3 by hand for batch 4: comp = 2*4*1024*P/989e12, comm = 2*P/450e9
+    comp, comm = 2 * 4 * 1024 / 989e12, 2 / 450e9
+    assert e4 == pytest.approx(comp / (comp + comm), rel=1e-12)
+    # the model size cancels out
+    assert M.forward_efficiency(1.0, 4, 1024, 989e12, 450e9) == pytest.approx(e4, rel=1e-12)
+
+
+def test_gpu_resident_buckets_by_hand():
+    # 64 M-element buckets; link 100 G elem/s each way, CPU step 12.5 G/s (Table 3's
+    # GraceAdam rate), backward 50 G params/s, GPU step 230 G params/s (measured here)
+    r = M.Rates(move_grad=100e9, move_param=100e9, step_cpu=12.5e9, step_gpu=230e9, bwd=50e9)
+    bucket = 64e6
+    exposed = bucket / 100e9 + bucket / 12.5e9 + bucket / 100e9          # 6.4 ms
+    cover = bucket / 50e9 + bucket / 230e9                               # 1.558 ms per bucket
+    n = M.gpu_resident_buckets(bucket, 100, r)
+    assert (n - 1) * cover < exposed <= n * cover and n == 5
+    # a CPU as fast as the GPU path needs fewer resident buckets; never more than exist
+    fast = M.Rates(100e9, 100e9, 230e9, 230e9, 50e9)
+    assert M.gpu_resident_buckets(bucket, 100, fast) < n
+    assert M.gpu_resident_buckets(bucket, 3, r) == 3
