@@ -73,11 +73,12 @@ _lib = None
 
 EXPORTS = ["so_layout_init", "so_layout_get_info", "so_layout_tensor", "so_layout_bind",
            "so_grad_check", "so_adam_step_speculative", "so_validate_commit_or_rollback",
-           "so_validate_begin", "so_validate_poll", "so_set_global_grad_stats", "so_cast_params", "so_iteration_host", "so_grad_check_static", "so_loss_scale_config",
-           "so_get_loss_scale", "so_state_export", "so_state_import", "so_bucket_slot", "so_get_step", "so_set_step",
-           "so_pending_buckets", "so_get_counters", "so_last_cuda_error", "so_strerror",
-           "so_destroy", "so_debug_set_dry_run", "so_debug_set_bucket_stats",
-           "so_debug_set_step_variant"]
+           "so_validate_begin", "so_validate_poll", "so_set_global_grad_stats",
+           "so_cast_params", "so_iteration_host", "so_grad_check_static",
+           "so_loss_scale_config", "so_get_loss_scale", "so_state_export", "so_state_import",
+           "so_bucket_slot", "so_get_step", "so_set_step", "so_pending_buckets",
+           "so_get_counters", "so_last_cuda_error", "so_strerror", "so_destroy",
+           "so_debug_set_dry_run", "so_debug_set_bucket_stats", "so_debug_set_step_variant"]
 
 
 def lib() -> C.CDLL:
