@@ -9,17 +9,17 @@
 //
 // Work decomposition.  A bucket is cut into *tiles* of 1024 consecutive
 // elements; one warp owns one tile at a time (dealt round-robin to all warps
-// of the grid here, claimed from a counter in the bulk-copy step kernel).  Inside a tile a warp sweeps 8 *rows* of 128
-// elements; lane l owns the *quad* of elements [4l, 4l+4) of each row, so a
-// warp-wide fp32 access is one contiguous 512-byte line set and a bf16 access
-// one contiguous 256-byte one.  The sum of squares of a tile is accumulated
+// of the grid here, claimed from a counter in the bulk-copy step kernel).
+// Inside a tile a warp sweeps 8 *rows* of 128 elements; lane l owns the *quad*
+// of elements [4l, 4l+4) of each row, so a warp-wide fp32 access is one
+// contiguous 512-byte line set and a bf16 access one contiguous 256-byte one.  The sum of squares of a tile is accumulated
 // per lane in four chains (one per quad position, each in row order), combined
 // pairwise, folded across lanes with an xor-shuffle tree and stored as one
 // double per tile; a second tiny kernel folds the tiles of each bucket in a
-// fixed order.  The summation order therefore depends on nothing
-// but the data and the bucket geometry: the same bits come out whatever the
-// grid size, and whether the sums were produced by the fused step kernel or by
-// the stand-alone check kernel.
+// fixed order.  The summation order therefore depends on nothing but the data
+// and the bucket geometry: the same bits come out whatever the grid size, and
+// whether the sums were produced by the fused step kernel or by the
+// stand-alone check kernel.
 #pragma once
 
 #include <cuda_fp16.h>
@@ -237,13 +237,15 @@ __device__ __forceinline__ double warp_fold(double x)
 // steps on g ~ sqrt(x), h ~ 1/(2 sqrt(x)).  Straight-line code: the library
 // routine's range checks and slow path are not needed here (x is a finite,
 // non-negative, never subnormal second moment).  The seed is taken of
-// max(x, 1e-290): for every real input that changes nothing, and for x = 0 it
-// keeps the seed finite so that g = 0 * seed = 0 comes out exactly.  A NaN/Inf
-// input only occurs in a speculative step that validation discards.
+// x + 1e-300: every non-zero second moment is at least 1e-93 (the square of the
+// smallest fp32 denormal times 1 - beta2), so the addition returns x itself,
+// and for x = 0 it keeps the seed finite so that g = 0 * seed = 0 comes out
+// exactly.  A NaN/Inf input only occurs in a speculative step that validation
+// discards.
 __device__ __forceinline__ double sqrt_nonneg(double x)
 {
     double y;
-    const double xs = fmax(x, 1e-290);
+    const double xs = __dadd_rn(x, 1e-300);
     asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(xs));
     double g = __dmul_rn(x, y);
     double h = __dmul_rn(0.5, y);
