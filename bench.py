@@ -32,6 +32,7 @@ if ROOT not in sys.path:
 METRIC = "optimizer_params_per_sec"
 UNIT = "params/s"
 BYTES_PER_PARAM = {"bf16": 28, "fp16": 28, "fp32": 30}      # algorithmic HBM bytes of the fused step
+GRAD_BYTES = {"bf16": 2, "fp16": 2, "fp32": 4}
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per parameter of the fused step
 # kernel (gpt2_small capture: 1.742 GB read + 1.688 GB written per launch of
@@ -226,6 +227,10 @@ def main():
     ap.add_argument("--undo-slots", type=int, default=-1)
     ap.add_argument("--per-bucket", action="store_true",
                     help="one speculative-step call per bucket instead of one batched call")
+    ap.add_argument("--order", default="stv", choices=["stv", "ste"],
+                    help="stv: speculate, then validate (default); ste: gradient check first, "
+                         "then the step and cast in place (the synchronous order the paper "
+                         "starts from), for comparison")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--step-variant", type=int, default=0,
@@ -284,7 +289,9 @@ def main():
     nb = opt.n_buckets
 
     def one_step(ev=None):
-        if args.per_bucket:
+        if args.order == "ste":
+            B.so_grad_check(opt.ctx, hp, B.SO_ALL, stream)
+        elif args.per_bucket:
             for b in range(nb):
                 try:
                     B.so_adam_step_speculative(opt.ctx, hp, b, stream)
@@ -333,13 +340,13 @@ def main():
     spec_buckets = min(nb, opt.info.undo_slots)
     spec_params = sum(opt.bucket_range(b)[1] - opt.bucket_range(b)[0] for b in range(spec_buckets))
     kernel_ms = None
-    if not args.per_bucket:
+    if not args.per_bucket and args.order == "stv":
         times = [a.elapsed_time(b) for a, b in kernel_events.values()]
         kernel_ms = sum(times) / len(times)
 
     # ---- end to end through the host-buffer entry point -------------------
     e2e = None
-    if not args.no_e2e and N <= (1 << 31):
+    if not args.no_e2e and args.order == "stv" and N <= (1 << 31):
         gsz = 4 if w.grad_dtype == "fp32" else 2
         host_g = torch.empty(N, dtype=opt.grad_torch_dtype, pin_memory=True)
         for start, piece in W.iter_gradients(w, 1, device="cuda", loss_scale=w.loss_scale):
@@ -391,12 +398,15 @@ def main():
                    "undo_slots": opt.info.undo_slots, "grad_dtype": w.grad_dtype,
                    "max_grad_norm": w.max_grad_norm,
                    "decisions": sorted(B.DECISION_NAMES[d] for d in decisions),
+                   "order": args.order,
                    "launch_mode": "per_bucket" if args.per_bucket else "batched",
                    "step_kernel": "bulk_copy_pipeline" if args.step_variant == 0 else "registers",
                    "parallelism": "replicas" if world > 1 else "single",
                    "l2": f"working set {16 * N / 1e6:.0f} MB resident + undo slots, "
                          "larger than the 126 MB L2; no flush"},
-        "hbm_gbs_whole_step": world * bpp * N / (ms_per_step * 1e-3) / 1e9,
+        # check-first reads the gradients twice: once to check, once to step
+        "hbm_gbs_whole_step": world * (bpp + (GRAD_BYTES[w.grad_dtype] if args.order == "ste" else 0))
+                              * N / (ms_per_step * 1e-3) / 1e9,
         "gpu_launches": launches,
         "clocks": clocks,
     }

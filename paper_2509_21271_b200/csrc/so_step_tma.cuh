@@ -333,10 +333,21 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                     const float4 g4 = *reinterpret_cast<const float4 *>(in + 3 * L::kF32Bytes + off * 4);
                     gq[0] = g4.x; gq[1] = g4.y; gq[2] = g4.z; gq[3] = g4.w;
                 }
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    adamw_element<!kSpec, grad_traits<GradT>::kUnscale>(gq[q], pq[q], mq[q], vq[q],
-                                                                         a.k, acc[q]);
+                adamw_quad<!kSpec, grad_traits<GradT>::kUnscale>(
+                    gq, pq, mq, vq, a.k, acc,
+                    [&](float4 &g0, float4 &p0, float4 &m0, float4 &v0) {
+                        // the input stage is refilled only after this loop
+                        p0 = *reinterpret_cast<const float4 *>(in + off * 4);
+                        m0 = *reinterpret_cast<const float4 *>(in + L::kF32Bytes + off * 4);
+                        v0 = *reinterpret_cast<const float4 *>(in + 2 * L::kF32Bytes + off * 4);
+                        if constexpr (sizeof(GradT) == 2) {
+                            const uint2 h2 = *reinterpret_cast<const uint2 *>(in + 3 * L::kF32Bytes + off * 2);
+                            unpack2<GradT>(h2.x, g0.x, g0.y);
+                            unpack2<GradT>(h2.y, g0.z, g0.w);
+                        } else {
+                            g0 = *reinterpret_cast<const float4 *>(in + 3 * L::kF32Bytes + off * 4);
+                        }
+                    });
                 *reinterpret_cast<float4 *>(out + off * 4) = make_float4(pq[0], pq[1], pq[2], pq[3]);
                 *reinterpret_cast<float4 *>(out + L::kF32Bytes + off * 4) =
                     make_float4(mq[0], mq[1], mq[2], mq[3]);
@@ -371,10 +382,14 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                 load_quad(a.master + src, idx, d.n, pq);
                 load_quad(a.mom + src, idx, d.n, mq);
                 load_quad(a.var + src, idx, d.n, vq);
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    adamw_element<!kSpec, grad_traits<GradT>::kUnscale>(gq[q], pq[q], mq[q], vq[q],
-                                                                         a.k, acc[q]);
+                adamw_quad<!kSpec, grad_traits<GradT>::kUnscale>(
+                    gq, pq, mq, vq, a.k, acc,
+                    [&](float4 &g0, float4 &p0, float4 &m0, float4 &v0) {
+                        g0 = load_quad4(g, idx, d.n);  // not stored yet: still the inputs
+                        p0 = load_quad4(a.master + src, idx, d.n);
+                        m0 = load_quad4(a.mom + src, idx, d.n);
+                        v0 = load_quad4(a.var + src, idx, d.n);
+                    });
                 if (idx < d.n) {
                     store_quad(a.master + dst, idx, d.n, pq);
                     store_quad(a.mom + dst, idx, d.n, mq);

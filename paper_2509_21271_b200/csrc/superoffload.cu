@@ -131,6 +131,9 @@ AdamScalars scalars_for(const so_hparams &hp, int64_t step_index, double scale, 
     k.step_size = hp.lr / bc1;
     k.decay = 1.0 - hp.lr * hp.weight_decay;
     k.eps = hp.eps;
+    k.lr = hp.lr;
+    k.bc1 = bc1;
+    k.bc2 = bc2;
     k.scale = scale;
     k.unscale = unscale;
     return k;
@@ -248,13 +251,13 @@ so_status launch_steps(so_ctx *c, const std::vector<BucketEntry> &entries, const
             if (c->step_variant != 1) {
                 launch_tma_variant(c, a, n, speculative, stream);
             } else if (speculative) {
-                if (dt == SO_GRAD_BF16) adamw_step_kernel<uint16_t, true, 4><<<grid, kThreads, 0, stream>>>(a);
-                else if (dt == SO_GRAD_FP16) adamw_step_kernel<half_t, true, 4><<<grid, kThreads, 0, stream>>>(a);
-                else adamw_step_kernel<float, true, 4><<<grid, kThreads, 0, stream>>>(a);
+                if (dt == SO_GRAD_BF16) adamw_step_kernel<uint16_t, true, 2><<<grid, kThreads, 0, stream>>>(a);
+                else if (dt == SO_GRAD_FP16) adamw_step_kernel<half_t, true, 2><<<grid, kThreads, 0, stream>>>(a);
+                else adamw_step_kernel<float, true, 2><<<grid, kThreads, 0, stream>>>(a);
             } else {
-                if (dt == SO_GRAD_BF16) adamw_step_kernel<uint16_t, false, 4><<<grid, kThreads, 0, stream>>>(a);
-                else if (dt == SO_GRAD_FP16) adamw_step_kernel<half_t, false, 4><<<grid, kThreads, 0, stream>>>(a);
-                else adamw_step_kernel<float, false, 4><<<grid, kThreads, 0, stream>>>(a);
+                if (dt == SO_GRAD_BF16) adamw_step_kernel<uint16_t, false, 2><<<grid, kThreads, 0, stream>>>(a);
+                else if (dt == SO_GRAD_FP16) adamw_step_kernel<half_t, false, 2><<<grid, kThreads, 0, stream>>>(a);
+                else adamw_step_kernel<float, false, 2><<<grid, kThreads, 0, stream>>>(a);
             }
         }
         const so_status s = after_launch(c);
@@ -584,12 +587,12 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
         const int dt = c->grad_dtype;
         e = dt == SO_GRAD_BF16
                 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                      &c->occ_step, adamw_step_kernel<uint16_t, true, 4>, kThreads, 0)
+                      &c->occ_step, adamw_step_kernel<uint16_t, true, 2>, kThreads, 0)
             : dt == SO_GRAD_FP16
                 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                      &c->occ_step, adamw_step_kernel<half_t, true, 4>, kThreads, 0)
+                      &c->occ_step, adamw_step_kernel<half_t, true, 2>, kThreads, 0)
                 : cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                      &c->occ_step, adamw_step_kernel<float, true, 4>, kThreads, 0);
+                      &c->occ_step, adamw_step_kernel<float, true, 2>, kThreads, 0);
         if (e != cudaSuccess) return cuda_fail(c, e);
         e = dt == SO_GRAD_BF16
                 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(

@@ -8,6 +8,8 @@ oracle's replay uses the coefficient the device found (compared separately
 against the oracle's own, to the norm tolerance)."""
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
 from dataclasses import dataclass, field
 
 import numpy as np
@@ -71,7 +73,10 @@ def compare_state(dev, orc, rep: Report) -> None:
     for name, a, b in zip(("p", "m", "v"), dev, orc):
         d = ulp_distance(a, b)
         mx = int(d.max()) if d.size else 0
-        assert mx <= MAX_ULP_STATE, f"{name}: {mx} ulp from the oracle"
+        if mx > MAX_ULP_STATE:
+            i = int(d.argmax())
+            raise AssertionError(f"{name}[{i}]: {mx} ulp from the oracle "
+                                 f"(device {float(a[i])!r}, oracle {float(b[i])!r})")
         rep.max_ulp[name] = max(rep.max_ulp[name], mx)
         rep.n_diff[name] += int((d != 0).sum())
     rep.n_elems += dev[0].size
@@ -168,6 +173,38 @@ def _bucket_state_numpy(opt: BucketedAdamW, b: int):
     return [p.cpu().numpy(), m.cpu().numpy(), v.cpu().numpy()], bf16_to_numpy(pb)
 
 
+# The oracle is single-threaded C and stays that way.  The host work of these
+# big cases is spread over threads only where the split cannot change a result:
+# a bucket's sum of squares is still one sequential pass (buckets are folded in
+# bucket order afterwards), and an element update depends on nothing outside
+# its own index, so stepping disjoint ranges concurrently is the same update.
+_POOL = ThreadPoolExecutor(max_workers=max(1, min(16, (os.cpu_count() or 2) - 1)))
+_STEP_CHUNK = 1 << 23
+
+
+def _oracle_check_all_buckets(opt: BucketedAdamW):
+    window, pending, results = 4, [], []
+    for b in range(opt.n_buckets):
+        gb = _bucket_grads_numpy(opt, b)
+        pending.append(_POOL.submit(oracle.grad_check_range, gb, 0, gb.size))
+        if len(pending) >= window:
+            results.append(pending.pop(0).result())
+    results += [f.result() for f in pending]
+    total, flag = 0.0, 0
+    for s, f in results:                  # bucket order
+        total += s
+        flag |= f
+    return total, flag
+
+
+def _oracle_step_chunked(p, m, v, g, scale, tt, hp) -> None:
+    futures = [_POOL.submit(oracle.adamw_step_range, p, m, v, g, lo, min(lo + _STEP_CHUNK, p.size),
+                            scale, tt, hp)
+               for lo in range(0, p.size, _STEP_CHUNK)]
+    for f in futures:
+        f.result()
+
+
 def run_sampled(w: W.Workload, steps: int, pick_buckets, undo_slots: int = B.SO_ALL,
                 expect_decisions=None):
     """Parity on a large workload: norm, coefficient, flag and decision are
@@ -192,12 +229,7 @@ def run_sampled(w: W.Workload, steps: int, pick_buckets, undo_slots: int = B.SO_
         res = opt.iteration(hp, stream=stream)
         torch.cuda.synchronize()
 
-        total, flag = 0.0, 0
-        for b in range(opt.n_buckets):
-            gb = _bucket_grads_numpy(opt, b)
-            s, f = oracle.grad_check_range(gb, 0, gb.size)
-            total += s
-            flag |= f
+        total, flag = _oracle_check_all_buckets(opt)
         norm = float(np.sqrt(np.float64(total)))
         own_coef = oracle.clip_coef(norm, hp.max_grad_norm)
         own_decision = oracle.decision(flag, own_coef)
@@ -211,7 +243,7 @@ def run_sampled(w: W.Workload, steps: int, pick_buckets, undo_slots: int = B.SO_
             gb = _bucket_grads_numpy(opt, b)
             if res.decision != B.SO_DECISION_SKIP:
                 scale = res.stats.clip_coef if res.decision == B.SO_DECISION_CLIP_RESTEP else 1.0
-                oracle.adamw_step_range(p, m, v, gb, 0, p.size, scale, t + 1, hp)
+                _oracle_step_chunked(p, m, v, gb, scale, t + 1, hp)
                 pb = oracle.bf16_rne(p)
             dev, pb_dev = _bucket_state_numpy(opt, b)
             compare_state(dev, (p, m, v), rep)

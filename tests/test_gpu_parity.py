@@ -10,7 +10,7 @@ import torch
 
 import oracle
 from gpu_harness import (Report, bf16_to_numpy, grads_to_numpy, hparams_of, run_lockstep)
-from helpers import is_bf16_nan
+from helpers import bf16_bits_to_f32, is_bf16_nan, ulp_distance
 from paper_2509_21271_b200 import binding as B
 from paper_2509_21271_b200 import build as so_build
 from paper_2509_21271_b200 import workloads as W
@@ -443,3 +443,74 @@ def test_per_bucket_launches_on_two_streams_give_the_same_bits():
                       res.stats.nonfinite, res.step_after))
     torch.cuda.synchronize()
     assert trace == ref[0] and _state_bytes(opt) == ref[1]
+
+
+# ---------------------------------------------------------------------------
+# cancelling updates: p*(1 - lr*wd) and the Adam update nearly equal
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("t0,clip", [(0, False), (0, True), (5, False)])
+def test_cancelling_update_stays_within_tolerance(t0, clip):
+    """When the decayed parameter and the update cancel, the new parameter is
+    orders of magnitude smaller than either, and an fp64 rounding error in the
+    update that is harmless elsewhere becomes whole fp32 ulps of the result.
+    Masters are placed next to the update (relative distance 2^-8 .. 2^-50
+    before their own rounding to fp32), so most of the new parameters are
+    1e-7 .. 1e-12 of the old ones.  The 2-ulp bound has to hold there too, and
+    deep inside the zone the result has to be the oracle's bit for bit."""
+    n, bucket = 1 << 20, 1 << 18
+    rng = np.random.default_rng(11 + t0 + int(clip))
+    hp = oracle.HParams(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01,
+                        max_grad_norm=1.0 if clip else 0.0)
+    g32 = (rng.standard_normal(n) * 1e-2).astype(np.float32)
+    g_t = torch.from_numpy(g32).cuda().to(torch.bfloat16)
+    g_bits = grads_to_numpy(g_t)
+    g = bf16_bits_to_f32(g_bits).astype(np.float64)
+    if t0:
+        m0 = (rng.standard_normal(n) * 3e-3).astype(np.float32)
+        v0 = (rng.random(n) * 1e-4 + 1e-8).astype(np.float32)
+    else:
+        m0 = np.zeros(n, np.float32)
+        v0 = np.zeros(n, np.float32)
+    coef = 1.0
+    if clip:
+        _, norm, _ = oracle.global_grad_check(g_bits, bucket)
+        coef = oracle.clip_coef(norm, hp.max_grad_norm)
+        assert coef < 1.0
+    # where the update will land (input construction only; the expected values
+    # below come from the oracle)
+    gs = g * coef
+    m1 = hp.beta1 * m0 + (1 - hp.beta1) * gs
+    v1 = hp.beta2 * v0 + (1 - hp.beta2) * gs * gs
+    tt = t0 + 1
+    u = hp.lr * (m1 / (1 - hp.beta1 ** tt)) / (np.sqrt(v1 / (1 - hp.beta2 ** tt)) + hp.eps)
+    delta = np.ldexp(1.0, -rng.integers(8, 51, n)) * rng.choice([-1.0, 1.0], n)
+    p0 = (u / (1 - hp.lr * hp.weight_decay) * (1 + delta)).astype(np.float32)
+
+    stream = torch.cuda.current_stream()
+    for variant in (0, 1):
+        opt = BucketedAdamW([n], bucket, "bf16", B.SO_ALL, step_variant=variant)
+        opt.load_state(torch.from_numpy(p0).cuda(), torch.from_numpy(m0).cuda(),
+                       torch.from_numpy(v0).cuda())
+        B.so_set_step(opt.ctx, t0)
+        opt.cast_params(stream=stream)
+        opt.load_grads(g_t)
+        res = opt.iteration(hp, stream=stream)
+        torch.cuda.synchronize()
+        assert res.decision == (R if clip else C)
+
+        p, m, v = p0.copy(), m0.copy(), v0.copy()
+        pb = oracle.bf16_rne(p)
+        orc = oracle.iteration_stv(p, m, v, pb, g_bits, bucket, t0, hp,
+                                   forced_coef=res.stats.clip_coef if clip else None)
+        assert orc.decision == res.decision
+        dev = [x.cpu().numpy() for x in opt.gather_state()]
+        ratio = np.abs(p.astype(np.float64)) / np.abs(p0.astype(np.float64))
+        assert np.count_nonzero(ratio < 2.0 ** -24) > n // 4     # the zone is populated
+        d = ulp_distance(dev[0], p)
+        assert d.max() <= 2, f"variant {variant}: p {d.max()} ulp from the oracle"
+        deep = ratio < 2.0 ** -17
+        assert np.array_equal(dev[0][deep].view(np.uint32), p[deep].view(np.uint32))
+        assert dev[1].tobytes() == m.tobytes() and dev[2].tobytes() == v.tobytes()
+        assert np.array_equal(bf16_to_numpy(opt.gather_param_bf16()), oracle.bf16_rne(dev[0]))
+        opt.close()
