@@ -109,3 +109,38 @@ def test_sweep_one_bucket_per_combination(bucket_mi, grad_dtype):
     write_report(w.name, rep, {"undo_slots": undo})
     opt.close()
     del opt
+
+
+# ---------------------------------------------------------------------------
+# the recipes at their full number of steps (about 50 minutes; on request)
+# ---------------------------------------------------------------------------
+
+full_length = pytest.mark.skipif(os.environ.get("SO_FULL_LENGTH") != "1",
+                                 reason="set SO_FULL_LENGTH=1 for the 20- and 100-step recipes")
+
+
+@full_length
+@pytest.mark.parametrize("clip", [False, True])
+def test_gpt2_small_twenty_steps(clip):
+    """Config 2 as stated: 20 AdamW steps, every element compared on every step."""
+    rep, opt = run_lockstep(W.gpt2_small(clip=clip), steps=20, guard_bands=False)
+    assert rep.decisions == [R if clip else C] * 20
+    write_report("gpt2_small_clip_20_steps" if clip else "gpt2_small_20_steps", rep)
+    opt.close()
+
+
+@full_length
+def test_llama_1b_hundred_steps():
+    """Config 3 as stated: the norm alternates 0.5 / 3.0, a NaN on steps 50 and
+    100.  Decision, norm and coefficient on every step; all 13 buckets on steps
+    1, 2, 49-51 and 100, one rotating bucket on the others."""
+    w = W.llama_1b()
+    nb = w.n_buckets
+    full = {1, 2, 49, 50, 51, 100}
+    rep, opt = run_sampled(w, steps=100,
+                           pick_buckets=lambda s: list(range(nb)) if s in full else [(s * 5) % nb])
+    want = [S if s % 50 == 0 else (C if s % 2 else R) for s in range(1, 101)]
+    assert rep.decisions == want
+    assert opt.step_count == 98
+    write_report("llama_1b_100_steps", rep)
+    opt.close()
