@@ -449,8 +449,9 @@ def test_per_bucket_launches_on_two_streams_give_the_same_bits():
 # cancelling updates: p*(1 - lr*wd) and the Adam update nearly equal
 # ---------------------------------------------------------------------------
 
-@pytest.mark.parametrize("t0,clip", [(0, False), (0, True), (5, False)])
-def test_cancelling_update_stays_within_tolerance(t0, clip):
+@pytest.mark.parametrize("t0,clip,dtype", [(0, False, "bf16"), (0, True, "bf16"), (5, False, "bf16"),
+                                           (5, True, "fp32"), (3, True, "fp16")])
+def test_cancelling_update_stays_within_tolerance(t0, clip, dtype):
     """When the decayed parameter and the update cancel, the new parameter is
     orders of magnitude smaller than either, and an fp64 rounding error in the
     update that is harmless elsewhere becomes whole fp32 ulps of the result.
@@ -462,10 +463,13 @@ def test_cancelling_update_stays_within_tolerance(t0, clip):
     rng = np.random.default_rng(11 + t0 + int(clip))
     hp = oracle.HParams(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01,
                         max_grad_norm=1.0 if clip else 0.0)
-    g32 = (rng.standard_normal(n) * 1e-2).astype(np.float32)
-    g_t = torch.from_numpy(g32).cuda().to(torch.bfloat16)
-    g_bits = grads_to_numpy(g_t)
-    g = bf16_bits_to_f32(g_bits).astype(np.float64)
+    loss_scale = 4096.0 if dtype == "fp16" else 1.0
+    unscale = 1.0 / loss_scale
+    g32 = (rng.standard_normal(n) * 1e-2 * loss_scale).astype(np.float32)
+    torch_dtype = {"bf16": torch.bfloat16, "fp32": torch.float32, "fp16": torch.float16}[dtype]
+    g_t = torch.from_numpy(g32).cuda().to(torch_dtype)
+    g_host = grads_to_numpy(g_t)             # what the oracle takes: bf16 bits, or fp32 / fp16 values
+    g = (bf16_bits_to_f32(g_host) if dtype == "bf16" else g_host).astype(np.float64) * unscale
     if t0:
         m0 = (rng.standard_normal(n) * 3e-3).astype(np.float32)
         v0 = (rng.random(n) * 1e-4 + 1e-8).astype(np.float32)
@@ -474,7 +478,7 @@ def test_cancelling_update_stays_within_tolerance(t0, clip):
         v0 = np.zeros(n, np.float32)
     coef = 1.0
     if clip:
-        _, norm, _ = oracle.global_grad_check(g_bits, bucket)
+        _, norm, _ = oracle.global_grad_check(g_host, bucket, unscale)
         coef = oracle.clip_coef(norm, hp.max_grad_norm)
         assert coef < 1.0
     # where the update will land (input construction only; the expected values
@@ -489,10 +493,12 @@ def test_cancelling_update_stays_within_tolerance(t0, clip):
 
     stream = torch.cuda.current_stream()
     for variant in (0, 1):
-        opt = BucketedAdamW([n], bucket, "bf16", B.SO_ALL, step_variant=variant)
+        opt = BucketedAdamW([n], bucket, dtype, B.SO_ALL, step_variant=variant)
         opt.load_state(torch.from_numpy(p0).cuda(), torch.from_numpy(m0).cuda(),
                        torch.from_numpy(v0).cuda())
         B.so_set_step(opt.ctx, t0)
+        if dtype == "fp16":
+            B.so_loss_scale_config(opt.ctx, loss_scale, 2.0, 0.5, 1000)
         opt.cast_params(stream=stream)
         opt.load_grads(g_t)
         res = opt.iteration(hp, stream=stream)
@@ -501,11 +507,14 @@ def test_cancelling_update_stays_within_tolerance(t0, clip):
 
         p, m, v = p0.copy(), m0.copy(), v0.copy()
         pb = oracle.bf16_rne(p)
-        orc = oracle.iteration_stv(p, m, v, pb, g_bits, bucket, t0, hp,
-                                   forced_coef=res.stats.clip_coef if clip else None)
+        orc = oracle.iteration_stv(p, m, v, pb, g_host, bucket, t0, hp,
+                                   forced_coef=res.stats.clip_coef if clip else None,
+                                   unscale=unscale)
         assert orc.decision == res.decision
         dev = [x.cpu().numpy() for x in opt.gather_state()]
         ratio = np.abs(p.astype(np.float64)) / np.abs(p0.astype(np.float64))
+        # with a clip, the device's coefficient differs from the one the masters
+        # were placed with by ~1e-13 relative, which bounds the cancellation
         assert np.count_nonzero(ratio < 2.0 ** -24) > n // 4     # the zone is populated
         d = ulp_distance(dev[0], p)
         assert d.max() <= 2, f"variant {variant}: p {d.max()} ulp from the oracle"
