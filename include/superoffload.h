@@ -109,6 +109,7 @@ typedef struct {
     int64_t commits, skips, clip_resteps;      /* validated iterations by outcome    */
     int64_t kernel_launches;                   /* kernels this context has launched  */
     int64_t elems_stepped, elems_checked, elems_cast;  /* work done by those kernels */
+    int64_t timeouts;                          /* iterations given up with SO_ERR_TIMEOUT */
 } so_counters;
 
 /*
@@ -204,6 +205,15 @@ so_status so_adam_step_speculative(so_ctx *ctx, const so_hparams *hp, int32_t bu
  * `hp` must equal the hyper-parameters of this iteration's speculative steps.
  * `out` (host, may be NULL) receives the decision, statistics and step count.
  * Follow-up kernels are enqueued on `stream`; the call does not wait for them.
+ * SO_ERR_TIMEOUT (also from so_grad_check(SO_ALL)): a kernel gave up a bounded
+ * wait for one of its own copies, so tiles are missing.  The iteration is given
+ * up: speculative slots are released, the bf16 copy of the speculated buckets is
+ * derived again from the committed master, step count and loss scale stay, and
+ * the context is idle (the iteration may be repeated).  The committed fp32
+ * state is untouched if the kernel was one of this iteration's (speculative
+ * steps, scans).  Kernels that validation itself enqueues (in-place steps,
+ * re-steps) report one iteration late, through the same status; if one of
+ * those can have been the cause, restore the state with so_state_import.
  */
 so_status so_validate_commit_or_rollback(so_ctx *ctx, const so_hparams *hp, void *stream,
                                          so_step_result *out);
@@ -357,7 +367,9 @@ void so_destroy(so_ctx *ctx);
 /*
  * Host-logic test hooks.  In dry-run mode no CUDA call is made: launches are
  * only counted, and the per-bucket check results come from
- * so_debug_set_bucket_stats instead of the device.  This lets the slot map and
+ * so_debug_set_bucket_stats instead of the device (with bucket == SO_ALL it
+ * sets, from `nonfinite`, the device status word the next check will read, which
+ * is how the SO_ERR_TIMEOUT handling is tested).  This lets the slot map and
  * the per-iteration state machine be exercised on a machine without a GPU.
  */
 so_status so_debug_set_dry_run(so_ctx *ctx, int32_t on);

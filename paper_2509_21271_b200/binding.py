@@ -56,7 +56,8 @@ class so_step_result(C.Structure):
 class so_counters(C.Structure):
     _fields_ = [("commits", C.c_int64), ("skips", C.c_int64), ("clip_resteps", C.c_int64),
                 ("kernel_launches", C.c_int64), ("elems_stepped", C.c_int64),
-                ("elems_checked", C.c_int64), ("elems_cast", C.c_int64)]
+                ("elems_checked", C.c_int64), ("elems_cast", C.c_int64),
+                ("timeouts", C.c_int64)]
 
 
 class SuperOffloadError(RuntimeError):

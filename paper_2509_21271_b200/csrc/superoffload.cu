@@ -73,6 +73,7 @@ struct so_ctx {
     int32_t last_cuda_error = 0;
     bool dry_run = false;
     std::vector<BucketStats> injected;
+    int32_t injected_status = 0;
     // ---- host-fed iteration: copy streams and ordering events (lazy) ----
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     std::vector<cudaEvent_t> events;
@@ -382,6 +383,27 @@ bool check_arrived(so_ctx *c)
     return cudaEventQuery(c->reduce_done) == cudaSuccess;
 }
 
+void end_iteration(so_ctx *c);
+
+// A kernel of this iteration gave up waiting for one of its own copies: give
+// the iteration up.  Speculative slots go back to the free list (the committed
+// slots were never written), the bf16 copy of the speculated buckets - partly
+// overwritten - is derived again from the committed master, and the context is
+// idle again with step count and loss scale as they were.
+so_status abandon_iteration(so_ctx *c)
+{
+    std::vector<BucketEntry> recast;
+    for (int32_t b = 0; b < c->n_buckets; ++b)
+        if (c->cover[b] == kSpeculated) {
+            recast.push_back(BucketEntry{b, c->slot_of[b], 0});
+            c->free_slots.push_back(c->spec_slot[b]);
+        }
+    if (!recast.empty()) launch_casts(c, recast, c->reduce_stream);   // best effort
+    c->counters.timeouts += 1;
+    end_iteration(c);
+    return SO_ERR_TIMEOUT;
+}
+
 // Second half: wait for the per-bucket records to reach the host, fold over
 // buckets in index order, derive norm and clip coefficient.
 so_status finish_check(so_ctx *c, const so_hparams &hp)
@@ -421,10 +443,14 @@ so_status finish_check(so_ctx *c, const so_hparams &hp)
                 // counters may be left mid-way, so re-arm the whole control block
                 cudaMemsetAsync(c->d_ctrl, 0, sizeof(ControlBlock), c->reduce_stream);
                 if (c->h_stats_dev) std::memset(&c->h_stats[c->n_buckets], 0, sizeof(BucketStats));
-                return SO_ERR_TIMEOUT;
+                return abandon_iteration(c);
             }
         } else {
             for (int32_t b = 0; b < c->n_buckets; ++b) c->h_stats[b] = c->injected[b];
+            if (c->injected_status != 0) {
+                c->injected_status = 0;
+                return abandon_iteration(c);
+            }
         }
     }
     double sumsq = 0.0;
@@ -1098,6 +1124,10 @@ so_status so_debug_set_step_variant(so_ctx *c, int32_t variant)
 
 so_status so_debug_set_bucket_stats(so_ctx *c, int32_t bucket, double sumsq, int32_t nonfinite)
 {
+    if (c && bucket == SO_ALL) {          // the device status word of the next check
+        c->injected_status = nonfinite;
+        return SO_OK;
+    }
     if (!c || bucket < 0 || bucket >= c->n_buckets) return SO_ERR_INVALID_ARG;
     c->injected[bucket] = BucketStats{sumsq, nonfinite, 0};
     return SO_OK;

@@ -326,3 +326,37 @@ def test_deferred_validation_state_machine():
     r = B.so_validate_commit_or_rollback(ctx, hp)
     assert r.step_after == 2 and r.buckets_speculated == 0
     B.so_destroy(ctx)
+
+
+def test_device_timeout_gives_the_iteration_up_and_leaves_the_context_usable():
+    """A raised device status word (a kernel gave up a bounded wait) must end
+    the iteration as if it had not happened: slots released, slot map, step
+    count and loss scale unchanged, bf16 of the speculated buckets re-derived,
+    and the same iteration can be run again."""
+    ctx, _ = _dry_ctx([1000], 256, undo=3)
+    hp = HP()
+    for b in range(4):
+        B.so_debug_set_bucket_stats(ctx, b, 0.01, 0)
+    B.so_adam_step_speculative(ctx, hp, B.SO_ALL)            # buckets 0..2 speculated
+    B.so_debug_set_bucket_stats(ctx, B.SO_ALL, 0.0, 1)       # status word of the next check
+    assert _status(B.so_validate_commit_or_rollback, ctx, hp) == B.SO_ERR_TIMEOUT
+    assert [B.so_bucket_slot(ctx, b) for b in range(4)] == [0, 1, 2, 3]
+    assert B.so_get_step(ctx) == 0 and B.so_pending_buckets(ctx) == 4
+    c = B.so_get_counters(ctx)
+    assert c.timeouts == 1 and (c.commits, c.skips, c.clip_resteps) == (0, 0, 0)
+    assert c.elems_cast == 768                               # bf16 of buckets 0..2 again
+    # the status was consumed; the iteration runs again, all three slots free
+    B.so_adam_step_speculative(ctx, hp, B.SO_ALL)
+    r = B.so_validate_commit_or_rollback(ctx, hp)
+    assert r.decision == B.SO_DECISION_COMMIT and r.buckets_speculated == 3 and r.step_after == 1
+    # also on the blocking check and on the deferred path
+    B.so_debug_set_bucket_stats(ctx, B.SO_ALL, 0.0, 1)
+    assert _status(B.so_grad_check, ctx, hp, B.SO_ALL) == B.SO_ERR_TIMEOUT
+    B.so_adam_step_speculative(ctx, hp, 0)
+    B.so_validate_begin(ctx, hp)
+    B.so_debug_set_bucket_stats(ctx, B.SO_ALL, 0.0, 1)
+    assert _status(B.so_validate_commit_or_rollback, ctx, hp) == B.SO_ERR_TIMEOUT
+    assert B.so_get_step(ctx) == 1 and B.so_get_counters(ctx).timeouts == 3
+    r = B.so_validate_commit_or_rollback(ctx, hp)
+    assert r.decision == B.SO_DECISION_COMMIT and r.step_after == 2
+    B.so_destroy(ctx)
