@@ -217,6 +217,80 @@ def run_reference(args, w):
     print(json.dumps(line))
 
 
+def run_overlap(args, w, opt, hp, B, torch):
+    """Speculative steps behind a synthetic bucket-by-bucket backward pass.
+
+    The paper's speculation-then-validation schedule takes the optimizer off the
+    critical path by stepping each bucket as soon as its gradients exist, while
+    the backward pass goes on (critical path of an iteration: its Eq. 7 against
+    Eq. 6).  Here both run on one GPU: the stand-in backward is a chain of bf16
+    matmuls per bucket on one stream (library GEMMs: not part of the path, only
+    something compute-bound to hide behind), the speculative step of bucket b
+    waits on an event recorded after bucket b's matmuls and runs on a second
+    stream, validation follows the last step.  Three timings over the same
+    number of iterations: backward alone, steps + validation alone, both."""
+    main = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
+    nb = opt.n_buckets
+    dim = 4096
+    a = torch.randn(dim, dim, device="cuda", dtype=torch.bfloat16)
+    b = torch.randn(dim, dim, device="cuda", dtype=torch.bfloat16)
+    out = torch.empty(dim, dim, device="cuda", dtype=torch.bfloat16)
+    events = [torch.cuda.Event() for _ in range(nb)]
+
+    def steps_only():
+        for bk in range(nb):
+            B.so_adam_step_speculative(opt.ctx, hp, bk, side)
+        B.so_validate_commit_or_rollback(opt.ctx, hp, side)
+
+    def timed(fn, iters):
+        torch.cuda.synchronize()
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record(main)
+        side.wait_event(t0)
+        for _ in range(iters):
+            fn()
+        done = torch.cuda.Event()
+        done.record(side)
+        main.wait_event(done)
+        t1.record(main)
+        torch.cuda.synchronize()
+        return t0.elapsed_time(t1) / iters
+
+    for _ in range(3):
+        steps_only()
+    t_steps = timed(steps_only, args.steps)
+    # matmuls per bucket so that the backward takes about bwd_ratio x the steps
+    def backward_only(k):
+        for bk in range(nb):
+            for _ in range(k):
+                torch.matmul(a, b, out=out)
+            events[bk].record(main)
+    backward_only(4)
+    t_mm = timed(lambda: backward_only(4), 3) / (4 * nb)
+    k = max(1, round(args.bwd_ratio * t_steps / (nb * t_mm)))
+    backward_only(k)
+    t_bwd = timed(lambda: backward_only(k), args.steps)
+
+    def overlapped():
+        for bk in range(nb):
+            for _ in range(k):
+                torch.matmul(a, b, out=out)
+            events[bk].record(main)
+            side.wait_event(events[bk])
+            B.so_adam_step_speculative(opt.ctx, hp, bk, side)
+        B.so_validate_commit_or_rollback(opt.ctx, hp, side)
+    for _ in range(3):
+        overlapped()
+    t_both = timed(overlapped, args.steps)
+    return {"ms_backward_alone": t_bwd, "ms_steps_and_validation_alone": t_steps,
+            "ms_overlapped": t_both, "ms_exposed": t_both - t_bwd,
+            "ms_serial_sum": t_bwd + t_steps,
+            "ms_last_bucket_step": t_steps / nb,
+            "matmuls_per_bucket": k, "matmul": f"{dim}x{dim}x{dim} bf16 (library GEMM stand-in)",
+            "buckets": nb, "step_launches": "one per bucket, second stream"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -231,6 +305,10 @@ def main():
                     help="stv: speculate, then validate (default); ste: gradient check first, "
                          "then the step and cast in place (the synchronous order the paper "
                          "starts from), for comparison")
+    ap.add_argument("--overlap", action="store_true",
+                    help="also time per-bucket speculative steps behind a synthetic backward pass")
+    ap.add_argument("--bwd-ratio", type=float, default=4.0,
+                    help="--overlap: length of the synthetic backward in units of the optimizer step")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--step-variant", type=int, default=0,
@@ -416,6 +494,8 @@ def main():
         line["e2e"] = {"value": world * N / (e2e["ms"] * 1e-3), "unit": UNIT,
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                        "ms_per_step": e2e["ms"]}
+    if args.overlap and world == 1:
+        line["overlap"] = run_overlap(args, w, opt, hp, B, torch)
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = _oracle_sample(w, 20, 1)[0]
     print(json.dumps(line))
