@@ -97,8 +97,11 @@ def check_stats(stats, orc_res, max_grad_norm: float, rep: Report) -> None:
 
 
 def run_lockstep(w: W.Workload, steps: int, undo_slots: int = B.SO_ALL,
-                 speculative: bool = True, guard_bands: bool = True, step_variant: int = 0):
-    """Full element-by-element parity over `steps` iterations of workload w."""
+                 speculative: bool = True, guard_bands: bool = True, step_variant: int = 0,
+                 drive=None):
+    """Full element-by-element parity over `steps` iterations of workload w.
+    `drive(opt, hp, stream, step)`, if given, issues the iteration's calls itself
+    (in whatever order and granularity) and returns the validation result."""
     hp = hparams_of(w)
     stream = torch.cuda.current_stream()
     opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, undo_slots,
@@ -123,7 +126,10 @@ def run_lockstep(w: W.Workload, steps: int, undo_slots: int = B.SO_ALL,
         g = W.gradients(w, step, device="cuda", loss_scale=loss_scale)
         opt.load_grads(g)
         g_host = grads_to_numpy(g)
-        res = opt.iteration(hp, stream=stream, speculative=speculative)
+        if drive is not None:
+            res = drive(opt, hp, stream, step)
+        else:
+            res = opt.iteration(hp, stream=stream, speculative=speculative)
         torch.cuda.synchronize()
 
         # oracle replay from the device's pre-step state

@@ -523,3 +523,57 @@ def test_cancelling_update_stays_within_tolerance(t0, clip, dtype):
         assert dev[1].tobytes() == m.tobytes() and dev[2].tobytes() == v.tobytes()
         assert np.array_equal(bf16_to_numpy(opt.gather_param_bf16()), oracle.bf16_rne(dev[0]))
         opt.close()
+
+
+# ---------------------------------------------------------------------------
+# random call sequences: any legal order and granularity gives the oracle's result
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("seed,undo,dtype", [(0, B.SO_ALL, "bf16"), (1, 5, "bf16"),
+                                             (2, 0, "fp32"), (3, 11, "fp32")])
+def test_random_call_sequences_lockstep(seed, undo, dtype):
+    """22 ragged buckets; per iteration the buckets are visited in random order
+    and each is stepped speculatively, scanned, or left to validation; the
+    check is finished by so_grad_check(SO_ALL), so_validate_begin, or validation
+    itself; norms fall on both sides of the clip threshold and two iterations
+    carry a non-finite gradient.  Every iteration is compared with the oracle."""
+    import random
+    rng = random.Random(seed)
+    w = W.tiny_ragged()
+    w.name = f"random_walk_{seed}"
+    w.bucket_elems = 50_003
+    w.grad_dtype = dtype
+    w.seed = 100 + seed
+    w.target_norm = lambda step: (0.4, 2.5, 0.9, 7.0)[(step * 7 + seed) % 4]
+    w.faults = (W.Fault(step=4, flat_index=3 * 50_003 + 11, kind="nan"),
+                W.Fault(step=9, flat_index=w.total - 1, kind="-inf"))
+    exhausted = [0]
+
+    def drive(opt, hp, stream, step):
+        order = list(range(opt.n_buckets))
+        rng.shuffle(order)
+        for b in order:
+            r = rng.random()
+            try:
+                if r < 0.6:
+                    B.so_adam_step_speculative(opt.ctx, hp, b, stream)
+                elif r < 0.8:
+                    B.so_grad_check(opt.ctx, None, b, stream)
+            except B.SuperOffloadError as e:
+                assert e.status == B.SO_ERR_UNDO_EXHAUSTED
+                exhausted[0] += 1
+        mode = rng.random()
+        if mode < 0.3:
+            B.so_validate_begin(opt.ctx, hp, stream)
+        elif mode < 0.5:
+            B.so_grad_check(opt.ctx, hp, B.SO_ALL, stream)
+        return B.so_validate_commit_or_rollback(opt.ctx, hp, stream)
+
+    rep, opt = run_lockstep(w, steps=12, undo_slots=undo, drive=drive)
+    assert {C, S, R} <= set(rep.decisions), rep.decisions
+    assert rep.decisions[3] == S and rep.decisions[8] == S
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+    assert opt.step_count == 10
+    if undo not in (B.SO_ALL,):
+        assert exhausted[0] > 0
+    opt.close()
