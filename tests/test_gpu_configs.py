@@ -144,3 +144,36 @@ def test_llama_1b_hundred_steps():
     assert opt.step_count == 98
     write_report("llama_1b_100_steps", rep)
     opt.close()
+
+
+def _soak_workload(dtype: str, steps: int) -> W.Workload:
+    """The ragged 1 Mi-parameter case with norms on both sides of the clip
+    threshold and a non-finite gradient every 97 steps."""
+    w = W.tiny_ragged()
+    w.name = f"soak_{dtype}"
+    w.grad_dtype = dtype
+    w.seed = 77
+    w.target_norm = lambda step: (0.3, 0.8, 1.5, 4.0, 0.99)[step % 5]
+    w.faults = tuple(W.Fault(step=s, flat_index=(s * 7919) % w.total,
+                             kind=("nan", "inf", "-inf")[s % 3]) for s in range(37, steps, 97))
+    return w
+
+
+def _soak(dtype: str, steps: int):
+    rep, opt = run_lockstep(_soak_workload(dtype, steps), steps=steps, undo_slots=3)
+    skips = len(range(37, steps, 97))
+    assert rep.decisions.count(S) == skips and opt.step_count == steps - skips
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+    write_report(f"soak_{dtype}_{steps}_steps", rep)
+    opt.close()
+
+
+def test_soak_two_hundred_steps():
+    """200 iterations in lock-step (windowed undo, all three decisions)."""
+    _soak("bf16", 200)
+
+
+@full_length
+@pytest.mark.parametrize("dtype,steps", [("bf16", 1200), ("fp32", 600)])
+def test_soak_long(dtype, steps):
+    _soak(dtype, steps)
