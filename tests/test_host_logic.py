@@ -360,3 +360,49 @@ def test_device_timeout_gives_the_iteration_up_and_leaves_the_context_usable():
     r = B.so_validate_commit_or_rollback(ctx, hp)
     assert r.decision == B.SO_DECISION_COMMIT and r.step_after == 2
     B.so_destroy(ctx)
+
+
+def test_header_is_plain_c_and_a_c_program_can_drive_the_library(tmp_path):
+    """The boundary is a C ABI: the header must compile as C99 with no CUDA or
+    C++ in sight, and a program written in C must be able to link against the
+    shared library and run the host-side calls (dry run: no GPU needed)."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    src = tmp_path / "drive.c"
+    src.write_text(r'''
+#include <stdio.h>
+#include <stdint.h>
+#include "superoffload.h"
+int main(void) {
+    int64_t numel[3] = {1000, 0, 537};
+    so_ctx *ctx = 0;
+    so_layout_info info;
+    if (so_layout_init(&ctx, 3, numel, 256, SO_GRAD_BF16, SO_ALL, &info) != SO_OK) return 1;
+    if (info.n_buckets != 7 || info.total_elems != 1537) return 2;
+    if (so_debug_set_dry_run(ctx, 1) != SO_OK) return 3;
+    char *base = (char *)0x10000000;
+    if (so_layout_bind(ctx, base, base + 0x1000000, base + 0x2000000, base + 0x3000000,
+                       base + 0x4000000, base + 0x5000000) != SO_OK) return 4;
+    so_hparams hp = {1e-3, 0.9, 0.999, 1e-8, 0.01, 1.0};
+    for (int b = 0; b < 7; ++b) so_debug_set_bucket_stats(ctx, b, 1.0, 0);
+    if (so_adam_step_speculative(ctx, &hp, SO_ALL, 0) != SO_OK) return 5;
+    so_step_result r;
+    if (so_validate_commit_or_rollback(ctx, &hp, 0, &r) != SO_OK) return 6;
+    printf("%d %d %lld %.6f\n", (int)r.decision, (int)r.buckets_speculated,
+           (long long)r.step_after, r.stats.norm);
+    so_destroy(ctx);
+    return 0;
+}
+''')
+    inc = os.path.join(ROOT, "include")
+    exe = tmp_path / "drive"
+    subprocess.run([gcc, "-std=c99", "-Wall", "-Werror", "-pedantic", "-fsyntax-only",
+                    "-I", inc, "-x", "c", os.path.join(inc, "superoffload.h")], check=True)
+    libdir = os.path.dirname(so_build.LIB_PATH)
+    subprocess.run([gcc, "-std=c99", "-Wall", "-Werror", "-I", inc, str(src), "-o", str(exe),
+                    "-L", libdir, "-lsuperoffload", f"-Wl,-rpath,{libdir}"], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()
+    assert out == [str(B.SO_DECISION_CLIP_RESTEP), "7", "1", f"{7 ** 0.5:.6f}"]
