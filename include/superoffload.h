@@ -182,7 +182,9 @@ so_status so_grad_check(so_ctx *ctx, const so_hparams *hp, int32_t bucket, void 
  *   bucket == SO_ALL : every uncovered bucket, in index order, for as long as
  *                 slots are free (batched launches); never UNDO_EXHAUSTED.
  * All speculative steps of one iteration must use equal hyper-parameters.
- * Enqueues only; no synchronisation.
+ * Enqueues only; no synchronisation.  Calls for different buckets may go to
+ * different streams and their kernels may overlap; at most 4096 step launches
+ * of one context may be outstanding (enqueued and unfinished) at any time.
  */
 so_status so_adam_step_speculative(so_ctx *ctx, const so_hparams *hp, int32_t bucket,
                                    void *stream);

@@ -41,7 +41,13 @@
 namespace so {
 
 constexpr uint32_t kSpinLimit = 1u << 20;              // bounded mbarrier polling
-constexpr int kCounterPairs = 64;                      // launches that may overlap in time
+// Launches of one context that may be outstanding at a time (enqueued and not
+// yet finished, on whatever streams).  A launch takes the next pair of the ring;
+// within one stream a pair's previous user has finished and re-armed it long
+// before it comes round again, and across streams the ring is long enough that
+// one stream would have to run 4096 launches ahead of another for two running
+// kernels to meet on a pair.
+constexpr int kCounterPairs = 4096;
 
 // Control block in scratch (zeroed once at bind time): a status record and a
 // ring of {next tile, finished warps} counter pairs, one pair per launch.
