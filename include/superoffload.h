@@ -19,7 +19,11 @@
  *   - `stream` arguments are cudaStream_t values passed as void* (NULL = the
  *     legacy default stream).  Calls that launch work enqueue it and return;
  *     only calls that fill a host struct from device results wait for the
- *     device (stated per function).
+ *     device (stated per function).  The library adds no dependencies
+ *     between streams: when the per-bucket calls of an iteration go to several
+ *     streams, the stream given to so_grad_check(SO_ALL) / so_validate_* must
+ *     have been made to wait for the others (an event per stream), and the
+ *     others must wait for it before the next iteration touches the buckets.
  *   - The device that is current when so_layout_bind is called must be current
  *     for every later call on that context.  A context is not thread-safe;
  *     separate contexts are independent.
