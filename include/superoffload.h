@@ -273,7 +273,8 @@ so_status so_cast_params(so_ctx *ctx, int32_t bucket, void *stream);
  *   host_param_bf16  flat bf16 output of N elements, or NULL for none
  * Buckets beyond the undo capacity are scanned instead of stepped and receive
  * their step inside validation.  Uses two internal copy streams created on
- * first use.  Returns after all copies have completed (synchronises).
+ * first use.  Returns after all copies have completed (synchronises); on an
+ * error too, so that no copy is left in flight from or into the host buffers.
  */
 so_status so_iteration_host(so_ctx *ctx, const so_hparams *hp, const void *host_grad,
                             void *host_param_bf16, void *stream, so_step_result *out);

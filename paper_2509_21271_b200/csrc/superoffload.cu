@@ -881,6 +881,9 @@ so_status so_cast_params(so_ctx *c, int32_t bucket, void *stream)
     return launch_casts(c, entries, static_cast<cudaStream_t>(stream));
 }
 
+static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void *host_grad,
+                                     void *host_param_bf16, void *stream, so_step_result *out);
+
 so_status so_iteration_host(so_ctx *c, const so_hparams *hp, const void *host_grad,
                             void *host_param_bf16, void *stream, so_step_result *out)
 {
@@ -888,6 +891,19 @@ so_status so_iteration_host(so_ctx *c, const so_hparams *hp, const void *host_gr
     if (!c->bound || c->phase != kIdle) return SO_ERR_STATE;
     if (!hparams_ok(hp) || (c->n_buckets > 0 && !host_grad)) return SO_ERR_INVALID_ARG;
     if (c->dry_run) return SO_ERR_UNSUPPORTED;
+    const so_status s = iteration_host_body(c, hp, host_grad, host_param_bf16, stream, out);
+    if (s != SO_OK && c->copy_in) {
+        // leave no copy in flight from or into the caller's buffers
+        cudaStreamSynchronize(c->copy_in);
+        cudaStreamSynchronize(c->copy_out);
+        cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    }
+    return s;
+}
+
+static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void *host_grad,
+                                     void *host_param_bf16, void *stream, so_step_result *out)
+{
     cudaStream_t main = static_cast<cudaStream_t>(stream);
     cudaError_t e;
     if (!c->copy_in) {
