@@ -319,7 +319,7 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
             const unsigned char *in = wbase + stage * L::kInStage;
             unsigned char *out = out_base + ostage * L::kOutStage;
             // one row (4 elements per lane) at a time: keeps the register
-            // footprint small enough for 16 warps per SM
+            // footprint small (the alternate 16-warp shape has 128 registers per thread)
 #pragma unroll 1
             for (int r = 0; r < kChunkRows; ++r) {
                 const uint32_t off = r * kRowElems + lane * 4;     // element within the chunk
