@@ -449,17 +449,21 @@ def test_per_bucket_launches_on_two_streams_give_the_same_bits():
 # cancelling updates: p*(1 - lr*wd) and the Adam update nearly equal
 # ---------------------------------------------------------------------------
 
-@pytest.mark.parametrize("t0,clip,dtype", [(0, False, "bf16"), (0, True, "bf16"), (5, False, "bf16"),
-                                           (5, True, "fp32"), (3, True, "fp16")])
-def test_cancelling_update_stays_within_tolerance(t0, clip, dtype):
+@pytest.mark.parametrize("t0,clip,dtype,undo", [(0, False, "bf16", B.SO_ALL), (0, True, "bf16", B.SO_ALL),
+                                                (5, False, "bf16", B.SO_ALL), (5, True, "fp32", B.SO_ALL),
+                                                (3, True, "fp16", B.SO_ALL),
+                                                (5, False, "bf16", 0), (2, True, "fp32", 0)])
+def test_cancelling_update_stays_within_tolerance(t0, clip, dtype, undo):
     """When the decayed parameter and the update cancel, the new parameter is
     orders of magnitude smaller than either, and an fp64 rounding error in the
     update that is harmless elsewhere becomes whole fp32 ulps of the result.
     Masters are placed next to the update (relative distance 2^-8 .. 2^-50
     before their own rounding to fp32), so most of the new parameters are
     1e-7 .. 1e-12 of the old ones.  The 2-ulp bound has to hold there too, and
-    deep inside the zone the result has to be the oracle's bit for bit."""
-    n, bucket = 1 << 20, 1 << 18
+    deep inside the zone the result has to be the oracle's bit for bit.
+    undo = 0 takes the check-first route (steps in place); the 13 elements past
+    the last full bucket take the kernels' guarded, non-staged path."""
+    n, bucket = (1 << 20) + 13, 1 << 18
     rng = np.random.default_rng(11 + t0 + int(clip))
     hp = oracle.HParams(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.01,
                         max_grad_norm=1.0 if clip else 0.0)
@@ -493,7 +497,7 @@ def test_cancelling_update_stays_within_tolerance(t0, clip, dtype):
 
     stream = torch.cuda.current_stream()
     for variant in (0, 1):
-        opt = BucketedAdamW([n], bucket, dtype, B.SO_ALL, step_variant=variant)
+        opt = BucketedAdamW([n], bucket, dtype, undo, step_variant=variant)
         opt.load_state(torch.from_numpy(p0).cuda(), torch.from_numpy(m0).cuda(),
                        torch.from_numpy(v0).cuda())
         B.so_set_step(opt.ctx, t0)
