@@ -289,13 +289,15 @@ def test_gpt2_small_clip_path_lockstep():
 # the host-fed, bucket-pipelined iteration
 # ---------------------------------------------------------------------------
 
-@pytest.mark.parametrize("name,undo", [("tiny", B.SO_ALL), ("tiny_ragged", 2), ("tiny", 0)])
-def test_host_fed_iteration_is_bitwise_the_device_fed_one(name, undo):
+@pytest.mark.parametrize("name,undo,dtype", [("tiny", B.SO_ALL, "bf16"), ("tiny_ragged", 2, "bf16"),
+                                             ("tiny", 0, "bf16"), ("tiny_ragged", 3, "fp32")])
+def test_host_fed_iteration_is_bitwise_the_device_fed_one(name, undo, dtype):
     """so_iteration_host (pinned gradients in, bf16 parameters out, copies
     overlapped per bucket) must leave exactly the state, statistics and
     decisions of the ordinary call sequence, and deliver the committed bf16
     parameters to the host -- through commits, clip re-steps and a skip."""
     w = W.by_name(name)
+    w.grad_dtype = dtype
     hp = hparams_of(w)
     stream = torch.cuda.current_stream()
     ref = _run_device_only(w, 8, undo_slots=undo, speculative=True)
@@ -303,7 +305,7 @@ def test_host_fed_iteration_is_bitwise_the_device_fed_one(name, undo):
     opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, undo)
     opt.load_state(W.initial_master(w, device="cuda"))
     opt.cast_params(stream=stream)
-    host_g = torch.empty(w.total, dtype=torch.bfloat16, pin_memory=True)
+    host_g = torch.empty(w.total, dtype=opt.grad_torch_dtype, pin_memory=True)
     host_p = torch.empty(w.total, dtype=torch.bfloat16, pin_memory=True)
     trace = []
     for step in range(1, 9):
