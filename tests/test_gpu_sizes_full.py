@@ -177,3 +177,26 @@ def test_soak_two_hundred_steps():
 @pytest.mark.parametrize("dtype,steps", [("bf16", 1200), ("fp32", 600)])
 def test_soak_long(dtype, steps):
     _soak(dtype, steps)
+
+
+@full_length
+def test_llama_8b_clip_and_nan_through_the_undo_window():
+    """The 8 B-parameter workload with the clip active on every other step and
+    a NaN on steps 4 and 8: re-steps write speculated buckets from their old
+    slot into the new one and step the others in place; a skip re-derives the
+    bf16 copy of the speculated ones.  Three buckets per step in lock-step,
+    from both sides of the window."""
+    w = W.llama_8b()
+    w.max_grad_norm = 1.0
+    w.target_norm = lambda step: 0.5 if step % 2 == 1 else 3.0
+    w.nan_every = 4
+    undo = _undo_that_fits(w)
+    nb = w.n_buckets
+    assert 0 < undo < nb
+    pick = lambda s: [(s * 3) % undo, undo + (s * 5) % (nb - undo), nb - 1 if s % 2 else 0]
+    rep, opt = run_sampled(w, steps=8, pick_buckets=pick, undo_slots=undo,
+                           expect_decisions=[C, R, C, S, C, R, C, S])
+    assert opt.step_count == 6
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+    write_report("llama_8b_clip_nan_8_steps", rep, {"undo_slots": undo})
+    opt.close()
