@@ -587,6 +587,9 @@ static __global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(co
     __shared__ double s_sum[kReduceThreads];
     __shared__ int s_bad[kReduceThreads];
     __shared__ int s_last;
+    // launched as a programmatic dependent of the kernel before it: nothing of
+    // that kernel's output may be read before this returns
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int32_t b = (int32_t)(blockIdx.x / a.segs_per_slot);
     const uint32_t seg = blockIdx.x - (uint32_t)b * a.segs_per_slot;
     const uint32_t n = (b == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;

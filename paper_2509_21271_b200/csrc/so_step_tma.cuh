@@ -417,6 +417,9 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
         stage = (stage + 1 == kStagesIn) ? 0 : stage + 1;
     }
 
+    // this warp has no more tiles to claim: a dependent kernel may be set up
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     if (failed) {
         // a copy never completed: tell the host, then give the copies that are
         // still in flight a bounded chance to land before this block's shared

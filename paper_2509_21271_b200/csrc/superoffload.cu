@@ -354,7 +354,20 @@ so_status begin_check(so_ctx *c, cudaStream_t stream)
             r.segs_per_slot = (uint32_t)c->segs_per_slot;
             r.n_buckets = c->n_buckets;
             const int64_t blocks = (int64_t)c->n_buckets * c->segs_per_slot;
-            bucket_reduce_kernel<<<(unsigned)blocks, kReduceThreads, 0, stream>>>(r);
+            // Programmatic dependent launch: the reduction's blocks may be set up
+            // while the step (or scan) kernel before it in the stream drains; they
+            // wait for its completion and memory flush before reading anything.
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)blocks);
+            cfg.blockDim = dim3(kReduceThreads);
+            cfg.dynamicSmemBytes = 0;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            cudaLaunchKernelEx(&cfg, bucket_reduce_kernel, r);
         }
         const so_status s = after_launch(c);
         if (s != SO_OK) return s;
