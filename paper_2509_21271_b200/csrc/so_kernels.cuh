@@ -340,9 +340,22 @@ static __device__ __noinline__ float4 adamw_exact_quad(float4 g, float4 p, float
     return r;
 }
 
-// The four elements of a lane's quad; `reload` fetches the original inputs of
-// the quad again (they have been overwritten in registers by then) and is only
-// called when one of the four cancelled.
+// The same, fetching the original inputs itself from global memory (they have
+// not been overwritten there yet): the call site passes four pointers and an
+// index instead of sixteen values.
+template <typename GradT, bool kScaled>
+static __device__ __noinline__ float4 adamw_exact_quad_at(const GradT *g, const float *p,
+                                                          const float *m, const float *v,
+                                                          uint32_t idx, uint32_t n,
+                                                          const AdamScalars &k)
+{
+    return adamw_exact_quad<kScaled, grad_traits<GradT>::kUnscale>(
+        load_quad4(g, idx, n), load_quad4(p, idx, n), load_quad4(m, idx, n), load_quad4(v, idx, n), k);
+}
+
+// The four elements of a lane's quad; `reload` forms the quad again in the
+// textbook order from its original inputs (they have been overwritten in
+// registers by then) and is only called when one of the four cancelled.
 template <bool kScaled, bool kUnscale, typename Reload>
 __device__ __forceinline__ void adamw_quad(const float (&gq)[4], float (&pq)[4], float (&mq)[4],
                                            float (&vq)[4], const AdamScalars &k, double (&acc)[4],
@@ -353,9 +366,7 @@ __device__ __forceinline__ void adamw_quad(const float (&gq)[4], float (&pq)[4],
     for (int q = 0; q < 4; ++q)
         redo |= adamw_element<kScaled, kUnscale>(gq[q], pq[q], mq[q], vq[q], k, acc[q]);
     if (__builtin_expect(redo, false)) {
-        float4 g0, p0, m0, v0;
-        reload(g0, p0, m0, v0);
-        const float4 e = adamw_exact_quad<kScaled, kUnscale>(g0, p0, m0, v0, k);
+        const float4 e = reload();
         pq[0] = e.x; pq[1] = e.y; pq[2] = e.z; pq[3] = e.w;
     }
 }
@@ -412,11 +423,8 @@ __global__ void __launch_bounds__(kThreads, 2) adamw_step_kernel(const __grid_co
                 const uint32_t idx = base + (r0 + u) * kRowElems + lane * 4;
                 adamw_quad<!kSpec, grad_traits<GradT>::kUnscale>(
                     gq[u], pq[u], mq[u], vq[u], a.k, acc,
-                    [&](float4 &g0, float4 &p0, float4 &m0, float4 &v0) {
-                        g0 = load_quad4(g, idx, n);    // not stored yet: still the inputs
-                        p0 = load_quad4(p_in, idx, n);
-                        m0 = load_quad4(m_in, idx, n);
-                        v0 = load_quad4(v_in, idx, n);
+                    [&]() {                    // not stored yet: still the inputs
+                        return adamw_exact_quad_at<GradT, !kSpec>(g, p_in, m_in, v_in, idx, n, a.k);
                     });
                 if (idx < n) {
                     store_quad(p_out, idx, n, pq[u]);

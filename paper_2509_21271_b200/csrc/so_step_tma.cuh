@@ -341,11 +341,12 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                 }
                 adamw_quad<!kSpec, grad_traits<GradT>::kUnscale>(
                     gq, pq, mq, vq, a.k, acc,
-                    [&](float4 &g0, float4 &p0, float4 &m0, float4 &v0) {
+                    [&]() {
                         // the input stage is refilled only after this loop
-                        p0 = *reinterpret_cast<const float4 *>(in + off * 4);
-                        m0 = *reinterpret_cast<const float4 *>(in + L::kF32Bytes + off * 4);
-                        v0 = *reinterpret_cast<const float4 *>(in + 2 * L::kF32Bytes + off * 4);
+                        float4 g0;
+                        const float4 p0 = *reinterpret_cast<const float4 *>(in + off * 4);
+                        const float4 m0 = *reinterpret_cast<const float4 *>(in + L::kF32Bytes + off * 4);
+                        const float4 v0 = *reinterpret_cast<const float4 *>(in + 2 * L::kF32Bytes + off * 4);
                         if constexpr (sizeof(GradT) == 2) {
                             const uint2 h2 = *reinterpret_cast<const uint2 *>(in + 3 * L::kF32Bytes + off * 2);
                             unpack2<GradT>(h2.x, g0.x, g0.y);
@@ -353,6 +354,7 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                         } else {
                             g0 = *reinterpret_cast<const float4 *>(in + 3 * L::kF32Bytes + off * 4);
                         }
+                        return adamw_exact_quad<!kSpec, grad_traits<GradT>::kUnscale>(g0, p0, m0, v0, a.k);
                     });
                 *reinterpret_cast<float4 *>(out + off * 4) = make_float4(pq[0], pq[1], pq[2], pq[3]);
                 *reinterpret_cast<float4 *>(out + L::kF32Bytes + off * 4) =
@@ -390,11 +392,9 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                 load_quad(a.var + src, idx, d.n, vq);
                 adamw_quad<!kSpec, grad_traits<GradT>::kUnscale>(
                     gq, pq, mq, vq, a.k, acc,
-                    [&](float4 &g0, float4 &p0, float4 &m0, float4 &v0) {
-                        g0 = load_quad4(g, idx, d.n);  // not stored yet: still the inputs
-                        p0 = load_quad4(a.master + src, idx, d.n);
-                        m0 = load_quad4(a.mom + src, idx, d.n);
-                        v0 = load_quad4(a.var + src, idx, d.n);
+                    [&]() {                    // not stored yet: still the inputs
+                        return adamw_exact_quad_at<GradT, !kSpec>(g, a.master + src, a.mom + src,
+                                                                  a.var + src, idx, d.n, a.k);
                     });
                 if (idx < d.n) {
                     store_quad(a.master + dst, idx, d.n, pq);
