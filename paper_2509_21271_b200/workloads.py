@@ -174,10 +174,21 @@ def sweep(bucket_mi: int, grad_dtype: str = "bf16", total: int = 4 << 30) -> Wor
                     grad_dtype=grad_dtype, loss_scale=4096.0 if grad_dtype == "fp16" else 1.0)
 
 
+def _with_grad_dtype(w: Workload, dtype: str) -> Workload:
+    """The same list with fp32 gradients, or fp16 gradients under a static loss scale."""
+    w.name = f"{w.name}_{dtype}"
+    w.grad_dtype = dtype
+    if dtype == "fp16":
+        w.loss_scale = 4096.0
+    return w
+
+
 def by_name(name: str) -> Workload:
     table = {"tiny": tiny, "tiny_ragged": tiny_ragged, "tiny_fp16": tiny_fp16,
              "gpt2_small": gpt2_small,
              "gpt2_small_clip": lambda: gpt2_small(clip=True),
+             "gpt2_small_fp32": lambda: _with_grad_dtype(gpt2_small(), "fp32"),
+             "gpt2_small_fp16": lambda: _with_grad_dtype(gpt2_small(), "fp16"),
              "llama_1b": llama_1b, "llama_8b": llama_8b}
     if name in table:
         return table[name]()
