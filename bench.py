@@ -34,6 +34,10 @@ UNIT = "params/s"
 BYTES_PER_PARAM = {"bf16": 28, "fp16": 28, "fp32": 30}      # algorithmic HBM bytes of the fused step
 GRAD_BYTES = {"bf16": 2, "fp16": 2, "fp32": 4}
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0             # vendor figure for B200 HBM3e, quoted for context
+# The largest configuration that fits one GPU: Llama-3-8B-shaped, 8.03 G
+# parameters in 41 buckets of 200 M elements, 128.5 GB resident.
+DEFAULT_WORKLOAD = "llama_8b"
 # dram__bytes_read.sum + dram__bytes_write.sum per parameter of the fused step
 # kernel (gpt2_small capture: 1.742 GB read + 1.688 GB written per launch of
 # 124 439 808 parameters; profiles/adamw_step_tma_kernel_gpt2_small.md), scaled
@@ -171,34 +175,102 @@ def _hparams(w, oracle_mod=None):
     return so_hparams(w.lr, w.beta1, w.beta2, w.eps, w.weight_decay, w.max_grad_norm)
 
 
-def _oracle_sample(w, steps, warmup):
-    """The CPU oracle, as it stands, on the first bucket of the workload."""
+ORACLE_SAMPLE_ELEMS = 64 << 20       # slice of the workload the CPU legs run on
+ORACLE_THREAD_ELEMS = 4 << 20       # bucket each thread of the all-cores leg owns
+
+
+def _oracle_inputs(w, n):
+    """Seeded inputs of the first n parameters of the workload, as numpy."""
     import numpy as np
     import torch
 
     import oracle
     from paper_2509_21271_b200 import workloads as W
 
-    n = min(w.bucket_elems, w.total)
     sample = W.Workload(name=w.name + "_sample", numel=[n], bucket_elems=n, sigma_g=w.sigma_g,
                         seed=w.seed, max_grad_norm=w.max_grad_norm, grad_dtype=w.grad_dtype)
     hp = oracle.HParams(lr=w.lr, beta1=w.beta1, beta2=w.beta2, eps=w.eps,
                         weight_decay=w.weight_decay, max_grad_norm=w.max_grad_norm)
     p = W.initial_master(sample).numpy()
+    g = W.gradients(sample, 1, loss_scale=w.loss_scale)
+    g = g.view(torch.int16).numpy().view(np.uint16) if g.dtype == torch.bfloat16 else g.numpy()
+    return p, g, hp
+
+
+def _oracle_sample(w, steps, warmup):
+    """The CPU oracle, as it stands (one thread), on a bounded slice of the
+    workload: the first min(bucket, 64 Mi) parameters."""
+    import numpy as np
+
+    import oracle
+
+    n = min(w.bucket_elems, w.total, ORACLE_SAMPLE_ELEMS)
+    p, g, hp = _oracle_inputs(w, n)
     m, v = np.zeros_like(p), np.zeros_like(p)
     pb = oracle.bf16_rne(p)
-    g = W.gradients(sample, 1)
-    g = g.view(torch.int16).numpy().view(np.uint16) if g.dtype == torch.bfloat16 else g.numpy()
+    unscale = 1.0 / w.loss_scale
     t = 0
     for _ in range(warmup):
-        t = oracle.iteration_ste(p, m, v, pb, g, n, t, hp).step_after
+        t = oracle.iteration_ste(p, m, v, pb, g, n, t, hp, unscale=unscale).step_after
     t0 = time.perf_counter()
     for _ in range(steps):
-        t = oracle.iteration_ste(p, m, v, pb, g, n, t, hp).step_after
+        t = oracle.iteration_ste(p, m, v, pb, g, n, t, hp, unscale=unscale).step_after
     dt = time.perf_counter() - t0
     return {"value": n * steps / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"first bucket ({n} params) of {w.name}, {steps} steps of check+AdamW+cast, "
+            "sample": f"first {n} params of {w.name}, {steps} steps of check+AdamW+cast, "
                       f"single thread, {dt:.1f} s"}, dt / steps, n
+
+
+def _cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as fh:
+            for line in fh:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
+def _oracle_all_cores(w, seconds: float = 8.0):
+    """The same oracle loop, one bucket per thread on every host core: each
+    thread owns a 4 Mi-parameter bucket (its own arrays) and repeats
+    check+AdamW+cast on it until the time is up.  The oracle itself stays
+    single-threaded C; the threads only run independent copies of it (ctypes
+    releases the interpreter lock during the call)."""
+    import numpy as np
+    from concurrent.futures import ThreadPoolExecutor
+
+    import oracle
+
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+    n = min(ORACLE_THREAD_ELEMS, w.total)
+    p0, g, hp = _oracle_inputs(w, n)
+    unscale = 1.0 / w.loss_scale
+
+    def make():
+        p = p0.copy()
+        return p, np.zeros_like(p), np.zeros_like(p), oracle.bf16_rne(p)
+    states = [make() for _ in range(cores)]
+    deadline = [0.0]
+
+    def work(i):
+        p, m, v, pb = states[i]
+        t, done = 0, 0
+        while True:
+            t = oracle.iteration_ste(p, m, v, pb, g, n, t, hp, unscale=unscale).step_after
+            done += 1
+            if time.perf_counter() >= deadline[0]:
+                return done
+    with ThreadPoolExecutor(max_workers=cores) as pool:
+        t0 = time.perf_counter()
+        deadline[0] = t0 + seconds
+        counts = list(pool.map(work, range(cores)))
+        dt = time.perf_counter() - t0
+    return {"value": n * sum(counts) / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "cpu_model": _cpu_model(),
+            "sample": f"{cores} threads, one {n}-param bucket of {w.name} each, "
+                      f"{sum(counts)} bucket steps of check+AdamW+cast in {dt:.1f} s"}
 
 
 def run_reference(args, w):
@@ -212,6 +284,7 @@ def run_reference(args, w):
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": w.name, "sample_params": n, "bucket_elems": w.bucket_elems},
             "cpu_baseline": base,
+            "cpu_baseline_all_cores": _oracle_all_cores(w, 5.0),
             "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0,
                     "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -294,10 +367,10 @@ def run_overlap(args, w, opt, hp, B, torch):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="gpt2_small")
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--undo-slots", type=int, default=-1)
     ap.add_argument("--per-bucket", action="store_true",
                     help="one speculative-step call per bucket instead of one batched call")
@@ -394,10 +467,11 @@ def main():
     for _ in range(args.warmup):
         one_step()
     # the fused step kernel is timed on every 4th step of the timed region (an
-    # event pair costs a few microseconds of an iteration that lasts ~0.5 ms)
+    # event pair costs a few microseconds of an iteration)
     sampled = set(range(0, args.steps, 4))
     kernel_events = {k: (torch.cuda.Event(enable_timing=True),
                          torch.cuda.Event(enable_timing=True)) for k in sampled}
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     launches0 = opt.counters().kernel_launches
     sampler = ClockSampler(local_rank)
     if rank == 0:
@@ -405,14 +479,15 @@ def main():
         time.sleep(0.05)
     barrier()
     mark0 = sampler.mark()
-    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     decisions = set()
-    t_start.record(stream)
+    marks[0].record(stream)
     for k in range(args.steps):
         decisions.add(one_step(kernel_events.get(k)).decision)
-    t_end.record(stream)
+        marks[k + 1].record(stream)
     barrier()
-    elapsed_ms = t_start.elapsed_time(t_end)
+    elapsed_ms = marks[0].elapsed_time(marks[-1])
+    per_step = sorted(marks[k].elapsed_time(marks[k + 1]) for k in range(args.steps))
+    median_ms, best_ms = per_step[len(per_step) // 2], per_step[0]
     launches = opt.counters().kernel_launches - launches0
     clocks = sampler.stop(mark0, sampler.mark()) if rank == 0 else None
     spec_buckets = min(nb, opt.info.undo_slots)
@@ -424,29 +499,39 @@ def main():
 
     # ---- end to end through the host-buffer entry point -------------------
     e2e = None
-    if not args.no_e2e and args.order == "stv" and N <= (1 << 31):
+    if not args.no_e2e and args.order == "stv":
         gsz = 4 if w.grad_dtype == "fp32" else 2
-        host_g = torch.empty(N, dtype=opt.grad_torch_dtype, pin_memory=True)
-        for start, piece in W.iter_gradients(w, 1, device="cuda", loss_scale=w.loss_scale):
-            host_g[start:start + piece.numel()].copy_(piece)
-        host_p = torch.empty(N, dtype=torch.bfloat16, pin_memory=True)
-        for _ in range(3):
-            B.so_iteration_host(opt.ctx, hp, host_g.data_ptr(), host_p.data_ptr(), stream)
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        n_e2e = max(3, min(args.steps, 10))
-        e0.record(stream)
-        for _ in range(n_e2e):
-            B.so_iteration_host(opt.ctx, hp, host_g.data_ptr(), host_p.data_ptr(), stream)
-        e1.record(stream)
-        barrier()
-        e2e_ms = e0.elapsed_time(e1) / n_e2e
-        e2e = {"ms": e2e_ms, "h2d": N * gsz, "d2h": N * 2 + 40}
+        try:
+            host_g = torch.empty(N, dtype=opt.grad_torch_dtype, pin_memory=True)
+            host_p = torch.empty(N, dtype=torch.bfloat16, pin_memory=True)
+        except RuntimeError as exc:       # the host refused to pin N * (gsz + 2) bytes
+            host_g = host_p = None
+            e2e = {"unavailable": f"could not pin {N * (gsz + 2)} bytes of host memory: "
+                                  f"{str(exc).splitlines()[0][:120]}"}
+        if host_g is not None:
+            for start, piece in W.iter_gradients(w, 1, device="cuda", loss_scale=w.loss_scale):
+                host_g[start:start + piece.numel()].copy_(piece)
+            n_warm = 3 if N < (1 << 31) else 1
+            for _ in range(n_warm):
+                B.so_iteration_host(opt.ctx, hp, host_g.data_ptr(), host_p.data_ptr(), stream)
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            n_e2e = max(3, min(args.steps, 10)) if N < (1 << 31) else 3
+            e0.record(stream)
+            for _ in range(n_e2e):
+                B.so_iteration_host(opt.ctx, hp, host_g.data_ptr(), host_p.data_ptr(), stream)
+            e1.record(stream)
+            barrier()
+            e2e_ms = e0.elapsed_time(e1) / n_e2e
+            e2e = {"ms": e2e_ms, "h2d": N * gsz, "d2h": N * 2 + 40, "steps": n_e2e}
+            del host_g, host_p
 
     # ---- max over ranks ----------------------------------------------------
     if dist is not None:
-        elapsed_ms, e2e_ms = max_over_ranks([elapsed_ms, e2e["ms"] if e2e else 0.0], "cuda")
-        if e2e:
+        have_e2e = bool(e2e) and "ms" in e2e
+        elapsed_ms, e2e_ms, median_ms, best_ms = max_over_ranks(
+            [elapsed_ms, e2e["ms"] if have_e2e else 0.0, median_ms, best_ms], "cuda")
+        if have_e2e:
             e2e["ms"] = e2e_ms
     if rank != 0:
         if dist is not None:
@@ -463,13 +548,15 @@ def main():
         roofline = {"bound": "hbm", "kernel": "adamw_step_tma_kernel (fused speculative AdamW step + bf16 cast + tile sums)",
                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}",
                     "unit": "GB/s", "frac": achieved / peak,
+                    "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                     "traffic": (NCU_TRAFFIC_BYTES_PER_PARAM * spec_params
                                 if NCU_TRAFFIC_BYTES_PER_PARAM else None),
                     "bytes_per_param": bpp, "params_per_launch": spec_params,
                     "kernel_ms": kernel_ms, "launches_timed": len(kernel_events)}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "median_ms": median_ms,
+        "best_ms": best_ms, "timed_region_s": elapsed_ms * 1e-3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": w.name, "params": N, "tensors": len(w.numel),
                    "bucket_elems": w.bucket_elems, "n_buckets": nb,
@@ -485,19 +572,30 @@ def main():
         # check-first reads the gradients twice: once to check, once to step
         "hbm_gbs_whole_step": world * (bpp + (GRAD_BYTES[w.grad_dtype] if args.order == "ste" else 0))
                               * N / (ms_per_step * 1e-3) / 1e9,
+        # bytes the step actually moves: buckets beyond the undo window are
+        # scanned first (one more gradient read) and stepped in place afterwards
+        "hbm_gbs_whole_step_moved": world * (bpp * N + GRAD_BYTES[w.grad_dtype] *
+                                             (N if args.order == "ste" else N - spec_params))
+                                    / (ms_per_step * 1e-3) / 1e9,
         "gpu_launches": launches,
         "clocks": clocks,
     }
+    if clocks and clocks.get("sm_mhz"):
+        line["ms_per_step_x_sm_mhz"] = ms_per_step * clocks["sm_mhz"]
     if roofline:
         line["roofline"] = roofline
-    if e2e:
+    if e2e and "ms" in e2e:
         line["e2e"] = {"value": world * N / (e2e["ms"] * 1e-3), "unit": UNIT,
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
-                       "ms_per_step": e2e["ms"]}
+                       "ms_per_step": e2e["ms"], "steps": e2e["steps"],
+                       "link_gbs_each_way": e2e["h2d"] / (e2e["ms"] * 1e-3) / 1e9}
+    elif e2e:
+        line["e2e"] = e2e
     if args.overlap and world == 1:
         line["overlap"] = run_overlap(args, w, opt, hp, B, torch)
     if not args.no_cpu_baseline and world == 1:
-        line["cpu_baseline"] = _oracle_sample(w, 20, 1)[0]
+        line["cpu_baseline"] = _oracle_sample(w, 10, 1)[0]
+        line["cpu_baseline_all_cores"] = _oracle_all_cores(w)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -82,6 +82,7 @@ struct CheckArgs {
     const void *grad;
     double *partials;
     double unscale;                       // 1 / loss scale (fp16 gradients), else 1
+    int32_t unscale_is_pow2;              // the product with `unscale` is exact
     Geometry geo;
     int32_t n_entries;
     int32_t bucket[kMaxBatch];
@@ -461,72 +462,117 @@ __device__ __forceinline__ void unpack_quad(const typename raw_quad<GradT>::type
     }
 }
 
-struct CheckTile { uint32_t n, base, lt; int32_t bucket; bool valid; };
+// A tile of the scan: `n` = elements in its bucket (0: no tile), `base` = its
+// first element within the bucket.
+struct CheckTile { uint32_t n, base; int32_t bucket; };
+
+// Resident blocks per SM the scan is compiled for (its two register buffers of
+// raw quads are twice as large with 4-byte gradients).
+template <typename GradT> struct check_shape { static constexpr int kBlocksPerSm = 4; };
+template <> struct check_shape<float> { static constexpr int kBlocksPerSm = 2; };
 
 template <typename GradT>
-__global__ void __launch_bounds__(kThreads) grad_check_kernel(const __grid_constant__ CheckArgs a)
+__global__ void __launch_bounds__(kThreads, check_shape<GradT>::kBlocksPerSm)
+grad_check_kernel(const __grid_constant__ CheckArgs a)
 {
     using Raw = typename raw_quad<GradT>::type;
+    constexpr bool kUnscale = grad_traits<GradT>::kUnscale;
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     const uint32_t tps = a.geo.tiles_per_slot;
-    const uint32_t total_tiles = (uint32_t)a.n_entries * tps;
+    const uint32_t n_entries = (uint32_t)a.n_entries;
+    const GradT *grad = static_cast<const GradT *>(a.grad);
 
-    // first tile at or after `tile` (stepping by n_warps) that lies inside its bucket
-    auto seek = [&](uint32_t tile, CheckTile &t) {
-        for (; tile < total_tiles; tile += n_warps) {
-            const uint32_t j = tile / tps;
-            const uint32_t lt = tile - j * tps;
-            const int32_t b = a.bucket[j];
+    // Position of the next tile to fetch, kept as (entry, tile within the slot)
+    // and advanced by the grid's stride without a division.
+    uint32_t ent = warp / tps, lt = warp - ent * tps;
+
+    // Describe the tile at the position (skipping slot padding), issue its
+    // vector loads (a ragged end is read later, guarded), start the tile this
+    // warp takes after it on its way from DRAM into L2 (no registers held for
+    // it), and move the position on.
+    auto fetch_next = [&](CheckTile &t, Raw (&raw)[kRowsPerTile]) {
+        for (;;) {
+            if (ent >= n_entries) { t.n = 0; return; }
+            const int32_t b = a.bucket[ent];
             const uint32_t n = (b == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
-            if (lt * kTileElems < n) {
-                t.n = n; t.base = lt * kTileElems; t.lt = lt; t.bucket = b; t.valid = true;
-                return tile;
+            const uint32_t base = lt * kTileElems;
+            if (base < n) {
+                t.n = n; t.base = base; t.bucket = b;
+                const GradT *slot = grad + (int64_t)b * a.geo.stride;
+                const GradT *g = slot + base + lane * 4;
+                if (base + kTileElems <= n) {
+#pragma unroll
+                    for (int r = 0; r < kRowsPerTile; ++r)
+                        raw[r] = __ldcs(reinterpret_cast<const Raw *>(g + r * kRowElems));
+                } else {
+#pragma unroll
+                    for (int r = 0; r < kRowsPerTile; ++r)
+                        if (base + r * kRowElems + lane * 4 + 4 <= n)
+                            raw[r] = __ldcs(reinterpret_cast<const Raw *>(g + r * kRowElems));
+                }
+                constexpr uint32_t kLines = kTileElems * sizeof(GradT) / 128;
+                const uint64_t ahead = (uint64_t)(lt + n_warps) * kTileElems;
+                if (ahead + kTileElems <= n && lane < kLines)
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(
+                        reinterpret_cast<const char *>(slot + ahead) + lane * 128));
             }
-        }
-        t.valid = false;
-        return tile;
-    };
-    // issue the vector loads of a tile's full quads (ragged ends are read later, guarded)
-    auto prefetch = [&](const CheckTile &t, Raw (&raw)[kRowsPerTile]) {
-        const GradT *g = static_cast<const GradT *>(a.grad) + (int64_t)t.bucket * a.geo.stride;
-#pragma unroll
-        for (int r = 0; r < kRowsPerTile; ++r) {
-            const uint32_t idx = t.base + r * kRowElems + lane * 4;
-            if (idx + 4 <= t.n) raw[r] = __ldcs(reinterpret_cast<const Raw *>(g + idx));
+            lt += n_warps;
+            while (lt >= tps) { lt -= tps; ++ent; }
+            if (base < n) return;
         }
     };
-
-    CheckTile cur, nxt;
-    Raw buf_cur[kRowsPerTile], buf_nxt[kRowsPerTile];
-    uint32_t tile = seek(warp, cur);
-    if (cur.valid) prefetch(cur, buf_cur);
-    while (cur.valid) {
-        tile = seek(tile + n_warps, nxt);
-        if (nxt.valid) prefetch(nxt, buf_nxt);
-
-        const GradT *g = static_cast<const GradT *>(a.grad) + (int64_t)cur.bucket * a.geo.stride;
+    // The square of a bf16 or fp32 value has at most 48 significant bits: it is
+    // exact in double, so one fused multiply-add rounds exactly like the
+    // multiply and the add it replaces.  The same holds for a binary16 value
+    // times a power of two (the usual loss scales); with any other scale the
+    // unscaled value has a full double mantissa and keeps the two separately
+    // rounded operations.
+    const bool exact_square = !kUnscale || a.unscale_is_pow2 != 0;
+    auto square_add = [&](float x, double &acc) {
+        const double gd = kUnscale ? __dmul_rn((double)x, a.unscale) : (double)x;
+        if (exact_square) acc = __fma_rn(gd, gd, acc);
+        else acc = __dadd_rn(acc, __dmul_rn(gd, gd));
+    };
+    auto consume = [&](const CheckTile &t, const Raw (&raw)[kRowsPerTile]) {
         double acc[4] = {0.0, 0.0, 0.0, 0.0};
+        if (t.base + kTileElems <= t.n) {
+            // the usual case, straight-line: no bounds to check
 #pragma unroll
-        for (int r = 0; r < kRowsPerTile; ++r) {
-            const uint32_t idx = cur.base + r * kRowElems + lane * 4;
-            float x[4];
-            if (idx + 4 <= cur.n) unpack_quad<GradT>(buf_cur[r], x);
-            else load_quad(g, idx, cur.n, x);               // guarded: zeros past the end
+            for (int r = 0; r < kRowsPerTile; ++r) {
+                float x[4];
+                unpack_quad<GradT>(raw[r], x);
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const double gd = grad_traits<GradT>::kUnscale ? __dmul_rn((double)x[q], a.unscale)
-                                                               : (double)x[q];
-                acc[q] = __dadd_rn(acc[q], __dmul_rn(gd, gd));
+                for (int q = 0; q < 4; ++q) square_add(x[q], acc[q]);
+            }
+        } else {
+            const GradT *g = grad + (int64_t)t.bucket * a.geo.stride;
+#pragma unroll
+            for (int r = 0; r < kRowsPerTile; ++r) {
+                const uint32_t idx = t.base + r * kRowElems + lane * 4;
+                float x[4];
+                if (idx + 4 <= t.n) unpack_quad<GradT>(raw[r], x);
+                else load_quad(g, idx, t.n, x);                 // guarded: zeros past the end
+#pragma unroll
+                for (int q = 0; q < 4; ++q) square_add(x[q], acc[q]);
             }
         }
         const double tile_sum = tile_fold(acc);
-        if (lane == 0) a.partials[(int64_t)cur.bucket * tps + cur.lt] = tile_sum;
+        if (lane == 0) a.partials[(int64_t)t.bucket * tps + t.base / kTileElems] = tile_sum;
+    };
 
-        cur = nxt;
-#pragma unroll
-        for (int r = 0; r < kRowsPerTile; ++r) buf_cur[r] = buf_nxt[r];
+    // Two register buffers used alternately: while one tile is summed the loads
+    // of the next are in flight and the one after that is coming into L2.
+    CheckTile t0, t1;
+    Raw buf0[kRowsPerTile], buf1[kRowsPerTile];
+    fetch_next(t0, buf0);
+    while (t0.n) {
+        fetch_next(t1, buf1);
+        consume(t0, buf0);
+        if (!t1.n) break;
+        fetch_next(t0, buf0);
+        consume(t1, buf1);
     }
 }
 

@@ -138,6 +138,7 @@ extern "C" so_status so_grad_check_static(const void *grad, int64_t n_elems, int
         a.grad = grad;
         a.partials = d->tile_sums;
         a.unscale = 1.0;
+        a.unscale_is_pow2 = 1;
         a.geo.stride = 0;
         a.geo.tiles_per_slot = n_tiles;
         a.geo.bucket_elems = (uint32_t)n_elems;

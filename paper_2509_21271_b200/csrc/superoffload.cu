@@ -276,6 +276,8 @@ so_status launch_checks(so_ctx *c, const std::vector<int32_t> &buckets, cudaStre
         a.grad = c->grad;
         a.partials = c->d_partials;
         a.unscale = c->iter_unscale;
+        int exponent = 0;
+        a.unscale_is_pow2 = std::frexp(a.unscale, &exponent) == 0.5 ? 1 : 0;
         a.geo = geo;
         a.n_entries = n;
         for (int i = 0; i < n; ++i) {
