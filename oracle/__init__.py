@@ -59,6 +59,10 @@ def _load():
     lib.orc_bf16_rne.argtypes = [c.c_float]
     lib.orc_cast_params.restype = None
     lib.orc_cast_params.argtypes = [vp, vp, i64]
+    lib.orc_fp16_rne.restype = c.c_uint16
+    lib.orc_fp16_rne.argtypes = [c.c_float]
+    lib.orc_cast_params_fp16.restype = None
+    lib.orc_cast_params_fp16.argtypes = [vp, vp, i64]
     lib.orc_grad_check_range.restype = c.c_int
     lib.orc_grad_check_range.argtypes = [vp, c.c_int, i64, i64, dbl, pd]
     lib.orc_global_grad_check.restype = c.c_int
@@ -132,6 +136,14 @@ def bf16_rne(x: np.ndarray) -> np.ndarray:
     x = _check(np.ascontiguousarray(x), np.float32)
     out = np.empty(x.shape, dtype=np.uint16)
     _load().orc_cast_params(_ptr(x), _ptr(out), x.size)
+    return out
+
+
+def fp16_rne(x: np.ndarray) -> np.ndarray:
+    """fp32 -> IEEE binary16 bit patterns (uint16), round to nearest even."""
+    x = _check(np.ascontiguousarray(x), np.float32)
+    out = np.empty(x.shape, dtype=np.uint16)
+    _load().orc_cast_params_fp16(_ptr(x), _ptr(out), x.size)
     return out
 
 

@@ -103,6 +103,49 @@ void orc_cast_params(const float *p, uint16_t *pb, int64_t n)
     for (int64_t i = 0; i < n; ++i) pb[i] = orc_bf16_rne(p[i]);
 }
 
+/*
+ * fp32 -> IEEE binary16, round to nearest, ties to even (Section 4.5 names the
+ * FP32 <-> FP16 casts of the paper's own mixed-precision runs).  Written out on
+ * the bit fields: binary16 keeps 10 mantissa bits and exponents -14..15; below
+ * 2^-14 its numbers are the multiples of 2^-24 (subnormals); a value that
+ * rounds to 2^16 or more becomes infinity (65520, halfway between the largest
+ * finite 65504 and 2^16, is the first such value: the tie goes to the even
+ * neighbour, which is 2^16).  NaN maps to a quiet NaN with the sign kept.
+ */
+uint16_t orc_fp16_rne(float x)
+{
+    const uint32_t u = f32_bits(x);
+    const uint16_t sign = (uint16_t)((u >> 16) & 0x8000u);
+    const uint32_t magnitude = u & 0x7FFFFFFFu;
+    const int exponent = (int)(magnitude >> 23) - 127;         /* unbiased, of a normal fp32 */
+    if (magnitude > 0x7F800000u) return (uint16_t)(sign | 0x7E00u);       /* NaN */
+    if (magnitude == 0x7F800000u) return (uint16_t)(sign | 0x7C00u);      /* infinity */
+    if (exponent < -26) return sign;          /* below 2^-26 (fp32 subnormals included): under half of 2^-24 */
+    {
+        /* 24-bit significand with its leading one; the result keeps its top
+         * bits down to the binary16 quantum: 2^(exponent-10) for a normal
+         * result, 2^-24 below 2^-14 */
+        const uint32_t significand = (magnitude & 0x7FFFFFu) | 0x800000u;
+        const int shift = exponent >= -14 ? 13 : 13 + (-14 - exponent);
+        uint32_t kept = significand >> shift;
+        const uint32_t dropped = significand & ((1u << shift) - 1u);
+        const uint32_t half = 1u << (shift - 1);
+        uint32_t bits;
+        if (dropped > half || (dropped == half && (kept & 1u))) kept += 1u;
+        if (exponent >= -14)
+            bits = ((uint32_t)(exponent + 14) << 10) + kept;   /* kept includes the leading one: +1 on the exponent field */
+        else
+            bits = kept;                                       /* subnormal, or 0x400 = 2^-14 after rounding up */
+        if (bits >= 0x7C00u) bits = 0x7C00u;                   /* rounded past the largest finite value */
+        return (uint16_t)(sign | bits);
+    }
+}
+
+void orc_cast_params_fp16(const float *p, uint16_t *ph, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) ph[i] = orc_fp16_rne(p[i]);
+}
+
 /* ---- gradient check (Section 4.4: global norm + NaN/Inf check) ---------- */
 
 static double grad_at(const void *g, int grad_dtype, int64_t i)

@@ -451,6 +451,81 @@ def test_bf16_rne_golden_table():
             assert out == int(want, 16), (hex(pattern), hex(out))
 
 
+def _golden_rows(name):
+    rows = []
+    with open(os.path.join(GOLDEN, name)) as fh:
+        for line in fh:
+            line = line.split("#")[0].split()
+            if len(line) == 2:
+                rows.append((int(line[0], 16), line[1]))
+    return rows
+
+
+def _is_fp16_nan(bits: np.ndarray) -> np.ndarray:
+    b = bits.astype(np.uint32)
+    return ((b & 0x7C00) == 0x7C00) & ((b & 0x03FF) != 0)
+
+
+def test_fp16_rne_golden_table():
+    rows = _golden_rows("fp16_rne_table.txt")
+    assert len(rows) >= 35
+    src = np.array([r[0] for r in rows], np.uint32).view(np.float32)
+    got = oracle.fp16_rne(src)
+    for (pattern, want), out in zip(rows, got):
+        if want == "nan":
+            assert _is_fp16_nan(np.array([out]))[0], hex(pattern)
+        else:
+            assert out == int(want, 16), (hex(pattern), hex(out))
+
+
+def test_fp16_rne_against_numpy_conversion():
+    """Library cross-check: numpy's float32 -> float16 conversion (IEEE round
+    to nearest even) on every upper half x lower halves that decide a rounding
+    at each possible cut (the cut moves down the word in the subnormal range),
+    plus eight million random patterns."""
+    rng = np.random.default_rng(15)
+    hi = np.arange(65536, dtype=np.uint32) << 16
+    lows = np.array([0, 1, 0x0FFF, 0x1000, 0x1001, 0x1FFF, 0x2000, 0x2FFF, 0x3000, 0x3001,
+                     0x7FFF, 0x8000, 0x8001, 0xEFFF, 0xF000, 0xFFFF], np.uint32)
+    pats = np.concatenate([(hi[:, None] | lows[None, :]).reshape(-1),
+                           rng.integers(0, 1 << 32, 1 << 23, dtype=np.uint64).astype(np.uint32),
+                           # dense around the subnormal range and the overflow threshold
+                           rng.integers(0x32000000, 0x39000000, 1 << 21, dtype=np.uint64).astype(np.uint32),
+                           rng.integers(0x477F0000, 0x47810000, 1 << 18, dtype=np.uint64).astype(np.uint32)])
+    x = pats.view(np.float32)
+    got = oracle.fp16_rne(x)
+    with np.errstate(over="ignore", invalid="ignore"):
+        ref = x.astype(np.float16).view(np.uint16)
+    nan = np.isnan(x)
+    assert _is_fp16_nan(got[nan]).all()
+    assert np.array_equal(got[~nan], ref[~nan])
+    # the sign of a NaN is kept
+    assert np.array_equal(got[nan] >> 15, (pats[nan] >> 31).astype(np.uint16))
+
+
+def test_fp16_rne_round_trip_and_monotonicity():
+    """Every binary16 value widened to fp32 casts back to itself, and the cast
+    never decreases when its argument increases (both fix the rounding
+    direction of every interval without reference to another implementation)."""
+    h = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    finite_or_inf = ~_is_fp16_nan(h)
+    wide = oracle.fp16_to_f32(h)
+    back = oracle.fp16_rne(wide)
+    assert np.array_equal(back[finite_or_inf], h[finite_or_inf])
+    pats = np.sort(np.random.default_rng(16).integers(0, 0x7F800000, 1 << 20, dtype=np.uint64)
+                   .astype(np.uint32))
+    out = oracle.fp16_rne(pats.view(np.float32)).astype(np.int64)
+    assert (np.diff(out) >= 0).all()
+    # halfway points between neighbours go to the neighbour with the even pattern
+    lo = np.arange(0, 0x7BFF, dtype=np.uint32).astype(np.uint16)
+    a = oracle.fp16_to_f32(lo).astype(np.float64)
+    b = oracle.fp16_to_f32((lo + 1).astype(np.uint16)).astype(np.float64)
+    mid = ((a + b) / 2).astype(np.float32)          # exact: 12 significant bits
+    assert np.array_equal(mid.astype(np.float64), (a + b) / 2)
+    want = np.where(lo % 2 == 0, lo, lo + 1).astype(np.uint16)
+    assert np.array_equal(oracle.fp16_rne(mid), want)
+
+
 def test_bf16_rne_against_torch_conversion():
     """Library cross-check on every upper half x the decisive lower halves,
     plus four million random patterns."""
