@@ -67,6 +67,7 @@ enum {
 };
 
 enum { SO_GRAD_BF16 = 0, SO_GRAD_FP32 = 1, SO_GRAD_FP16 = 2 };
+enum { SO_PARAM_BF16 = 0, SO_PARAM_FP16 = 1 };   /* dtype of the low-precision parameter copy */
 enum { SO_DECISION_COMMIT = 0, SO_DECISION_SKIP = 1, SO_DECISION_CLIP_RESTEP = 2 };
 #define SO_ALL (-1)
 
@@ -144,14 +145,48 @@ so_status so_layout_tensor(const so_ctx *ctx, int32_t i, int64_t *flat_offset,
 /*
  * so_layout_bind -- hand the caller-owned DEVICE arenas to the context.
  * Sizes as reported by so_layout_init; pointers 256-byte aligned; master, m, v
- * are fp32, grad is bf16, fp16 or fp32 per grad_dtype, param_bf16 is bf16.  The
+ * are fp32, grad is bf16, fp16 or fp32 per grad_dtype, param_bf16 is the 2-byte
+ * low-precision parameter copy (bf16, or binary16 after so_param_dtype_config).  The
  * caller fills master/m/v slot b with bucket b's initial state (m = v = 0 for
  * a fresh optimizer) and normally calls so_cast_params(SO_ALL) once.  Scratch
- * needs no initialisation by the caller (bind zeroes a small control
- * block and the per-bucket reduction counters with synchronous cudaMemsets).  Records the current device.
+ * needs no initialisation by the caller (bind zeroes a small control block and
+ * the reduction counters and uploads the slot tables, synchronously; with an
+ * empty tensor list it touches no device memory and all pointers may be NULL).
+ * Records the current device.
  */
 so_status so_layout_bind(so_ctx *ctx, void *master, void *m, void *v, void *grad,
                          void *param_bf16, void *scratch);
+
+/*
+ * so_param_dtype_config -- dtype of the low-precision parameter copy (Section
+ * 4.5 casts FP32 <-> FP16: the paper's runs keep FP16 parameters; bf16 is the
+ * default here).  With SO_PARAM_FP16 the fused step and so_cast_params write
+ * IEEE binary16, round to nearest even (values beyond 65504 + half an ulp
+ * become infinities, subnormals are kept).  Only between iterations; call
+ * so_cast_params(SO_ALL) afterwards to re-derive the copy.  Host-only.
+ */
+so_status so_param_dtype_config(so_ctx *ctx, int32_t param_dtype);
+
+/*
+ * so_layout_pack_grads / so_layout_unpack_params -- the device part of the
+ * flattening (Section 4.3: model states are flattened into buckets).  One
+ * kernel launch copies every tensor's gradient from its own buffer into the
+ * gradient arena (pack), or every tensor's low-precision parameters from the
+ * parameter arena back into its own buffer (unpack).
+ *   tensor_grads / tensor_params   HOST array of n_tensors DEVICE pointers in
+ *                the order given to so_layout_init, each to numel[i] elements
+ *                of the gradient dtype (pack) or of 2 bytes (unpack), aligned
+ *                to its element size; an empty tensor's pointer may be NULL.
+ *                The array is read before the call returns.
+ * Tensors may start at any element alignment and straddle buckets; interior
+ * runs move as 128-bit accesses, ragged heads and tails element by element.
+ * Pack only between iterations (SO_ERR_STATE once a bucket is covered); unpack
+ * at any time, ordered on `stream` like any other work.  Enqueues only (a
+ * second call on the same context first waits for `stream`, because the
+ * pointer list is staged in one pinned buffer).
+ */
+so_status so_layout_pack_grads(so_ctx *ctx, const void *const *tensor_grads, void *stream);
+so_status so_layout_unpack_params(so_ctx *ctx, void *const *tensor_params, void *stream);
 
 /*
  * so_grad_check -- the global gradient check (Section 4.4: the global
@@ -197,17 +232,21 @@ so_status so_adam_step_speculative(so_ctx *ctx, const so_hparams *hp, int32_t bu
  * so_validate_commit_or_rollback -- end the iteration (Section 4.4: after
  * validation, either keep the speculative update, skip the iteration when a
  * NaN/Inf was found, or revert it and re-execute with clipped gradients).
- * Completes the gradient check if so_grad_check(SO_ALL) has not run
- * (blocks until its results have reached the host), then
- *   nonfinite          -> SKIP: speculative slots are dropped, the bf16 copy of
- *                         those buckets is re-derived from the untouched master,
- *                         the step count does not advance;
+ * If a validation begun with so_validate_begin is pending, this call collects
+ * it.  Otherwise it enqueues the end of the open iteration -- the scan of
+ * uncovered buckets, the reduction with the verdict formed on the device (or,
+ * after so_grad_check(SO_ALL), a one-block kernel that applies the statistics
+ * the host holds), and the follow-up launch -- and then waits for the verdict
+ * to reach the host; the follow-up kernels run meanwhile.  On the device
+ *   nonfinite          -> SKIP: speculative slots are dropped, the low-precision
+ *                         copy of those buckets is re-derived from the untouched
+ *                         master, the step count does not advance;
  *   else clip_coef < 1 -> CLIP_RESTEP: every bucket is stepped from its
  *                         untouched prior state with gradients scaled by
  *                         clip_coef (same step index), then committed;
  *   else               -> COMMIT: speculated buckets are re-pointed at their new
- *                         slot (no device work); buckets that were only checked
- *                         are stepped in place with scale 1.
+ *                         slot (the follow-up launch returns at once); buckets
+ *                         that were only checked are stepped in place, scale 1.
  * `hp` must equal the hyper-parameters of this iteration's speculative steps.
  * `out` (host, may be NULL) receives the decision, statistics and step count.
  * Follow-up kernels are enqueued on `stream`; the call does not wait for them.
@@ -227,14 +266,29 @@ so_status so_validate_commit_or_rollback(so_ctx *ctx, const so_hparams *hp, void
 /*
  * so_validate_begin / so_validate_poll -- validation off the critical path
  * (Section 4.4: validation runs while the GPU executes the next forward pass,
- * and the result is consulted after it).  so_validate_begin scans whatever is
- * still uncovered and launches the reduction; its records make their own way
- * to the host and the call returns at once.  The caller then enqueues other
- * work (the next forward pass) and later calls
- * so_validate_commit_or_rollback, which by then finds the verdict waiting;
- * so_validate_poll tells without blocking whether it has arrived (*ready = 1).
- * Between so_validate_begin and so_validate_commit_or_rollback no bucket may be
- * stepped or scanned (SO_ERR_STATE).
+ * and the result is consulted after it).  so_validate_begin enqueues the whole
+ * end of the iteration and returns at once: the scan of whatever is still
+ * uncovered, the reduction, whose last block forms the verdict ON THE DEVICE
+ * (norm, clip coefficient, decision) and re-points the speculated buckets if
+ * the iteration is kept, and one follow-up launch that reads that verdict and
+ * does what it entails (see so_validate_commit_or_rollback).  No host round
+ * trip separates these kernels.  The verdict also travels to mapped host
+ * memory; so_validate_poll tells without blocking whether it has arrived
+ * (*ready = 1), and so_validate_commit_or_rollback, called later, collects it
+ * for the host's bookkeeping (step count, loss scale, counters, slot map).
+ * Until it has been collected:
+ *   - the NEXT iteration may already be assembled: so_adam_step_speculative and
+ *     so_grad_check(bucket) are accepted and enqueue kernels that carry the
+ *     constants (step index, loss scale) for each way the pending iteration can
+ *     end and choose among them on the device;
+ *   - so_grad_check(SO_ALL) waits for the pending verdict and reports its
+ *     statistics without collecting it (only while no new iteration is open);
+ *   - so_validate_begin, so_cast_params, so_layout_bind, so_set_step, state
+ *     export / import and the loss-scale / dtype setters return SO_ERR_STATE;
+ *   - so_validate_commit_or_rollback collects the pending verdict and leaves
+ *     the newly opened iteration alone.
+ * All of one context's kernels must be ordered by the caller's streams as
+ * before: the next iteration's steps after the follow-up launch of this one.
  */
 so_status so_validate_begin(so_ctx *ctx, const so_hparams *hp, void *stream);
 so_status so_validate_poll(so_ctx *ctx, int32_t *ready);
@@ -384,10 +438,18 @@ so_status so_debug_set_bucket_stats(so_ctx *ctx, int32_t bucket, double sumsq,
                                     int32_t nonfinite);
 
 /* Which implementation of the fused step runs: 0 (default) stages bulk copies
- * through shared memory, 1 keeps everything in registers, 10 and 11 are the
- * default with other pipeline shapes.  All produce the same bits; the switch
- * exists for measurements and for testing them against each other. */
+ * through shared memory, 1 keeps everything in registers.  Both produce the
+ * same bits; the switch exists for measurements and for testing them against
+ * each other. */
 so_status so_debug_set_step_variant(so_ctx *ctx, int32_t variant);
+
+/* How many times the bulk-copy step kernel polls for a chunk's loads before it
+ * gives the launch up (0 .. 2^20, the default).  The waits that drain copies in
+ * flight before a block exits always use the full limit, so a small value makes
+ * the kernel raise its status word (SO_ERR_TIMEOUT at the next check) without
+ * leaving anything in flight: this is how the give-up path is tested.  Applies
+ * to launches made after the call. */
+so_status so_debug_set_spin_limit(so_ctx *ctx, int64_t polls);
 
 #ifdef __cplusplus
 }

@@ -19,6 +19,7 @@ SO_ERR_TIMEOUT = -7
 SO_ERR_TOO_LARGE = -8
 SO_STATIC_CHECK_MAX_ELEMS = 1 << 26
 SO_GRAD_BF16, SO_GRAD_FP32, SO_GRAD_FP16 = 0, 1, 2
+SO_PARAM_BF16, SO_PARAM_FP16 = 0, 1
 SO_DECISION_COMMIT, SO_DECISION_SKIP, SO_DECISION_CLIP_RESTEP = 0, 1, 2
 SO_ALL = -1
 DECISION_NAMES = {0: "COMMIT", 1: "SKIP", 2: "CLIP_RESTEP"}
@@ -73,6 +74,8 @@ class SuperOffloadError(RuntimeError):
 _lib = None
 
 EXPORTS = ["so_layout_init", "so_layout_get_info", "so_layout_tensor", "so_layout_bind",
+           "so_param_dtype_config", "so_layout_pack_grads", "so_layout_unpack_params",
+           "so_debug_set_spin_limit",
            "so_grad_check", "so_adam_step_speculative", "so_validate_commit_or_rollback",
            "so_validate_begin", "so_validate_poll", "so_set_global_grad_stats",
            "so_cast_params", "so_iteration_host", "so_grad_check_static",
@@ -99,6 +102,10 @@ def lib() -> C.CDLL:
         "so_layout_get_info": [vp, P(so_layout_info)],
         "so_layout_tensor": [vp, i32, P(i64), P(i32), P(i32)],
         "so_layout_bind": [vp, vp, vp, vp, vp, vp, vp],
+        "so_param_dtype_config": [vp, i32],
+        "so_layout_pack_grads": [vp, P(vp), vp],
+        "so_layout_unpack_params": [vp, P(vp), vp],
+        "so_debug_set_spin_limit": [vp, i64],
         "so_grad_check": [vp, P(so_hparams), i32, vp, P(so_grad_stats)],
         "so_adam_step_speculative": [vp, P(so_hparams), i32, vp],
         "so_validate_commit_or_rollback": [vp, P(so_hparams), vp, P(so_step_result)],
@@ -193,6 +200,26 @@ def so_layout_bind(ctx, master: int, m: int, v: int, grad: int, param_bf16: int,
     """Arguments are raw device addresses (e.g. ``tensor.data_ptr()``)."""
     _ok(ctx, lib().so_layout_bind(ctx, master, m, v, grad, param_bf16, scratch),
         "so_layout_bind")
+
+
+def so_param_dtype_config(ctx, param_dtype: int) -> None:
+    _ok(ctx, lib().so_param_dtype_config(ctx, param_dtype), "so_param_dtype_config")
+
+
+def _ptr_array(ptrs):
+    return (C.c_void_p * max(len(ptrs), 1))(*[C.c_void_p(int(p) or None) for p in ptrs])
+
+
+def so_layout_pack_grads(ctx, tensor_grads, stream=None) -> None:
+    """`tensor_grads`: one raw device address per tensor, in layout order."""
+    _ok(ctx, lib().so_layout_pack_grads(ctx, _ptr_array(tensor_grads), _stream(stream)),
+        "so_layout_pack_grads")
+
+
+def so_layout_unpack_params(ctx, tensor_params, stream=None) -> None:
+    """`tensor_params`: one raw device address per tensor, in layout order."""
+    _ok(ctx, lib().so_layout_unpack_params(ctx, _ptr_array(tensor_params), _stream(stream)),
+        "so_layout_unpack_params")
 
 
 def so_grad_check(ctx, hp, bucket: int = SO_ALL, stream=None):
@@ -322,6 +349,10 @@ def so_debug_set_dry_run(ctx, on: bool) -> None:
 def so_debug_set_bucket_stats(ctx, bucket: int, sumsq: float, nonfinite: int) -> None:
     _ok(ctx, lib().so_debug_set_bucket_stats(ctx, bucket, sumsq, nonfinite),
         "so_debug_set_bucket_stats")
+
+
+def so_debug_set_spin_limit(ctx, polls: int) -> None:
+    _ok(ctx, lib().so_debug_set_spin_limit(ctx, polls), "so_debug_set_spin_limit")
 
 
 def so_debug_set_step_variant(ctx, variant: int) -> None:

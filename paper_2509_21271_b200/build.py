@@ -11,7 +11,7 @@ CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libsuperoffload.so")
 SOURCES = [os.path.join(CSRC, "superoffload.cu"), os.path.join(CSRC, "so_static_check.cu")]
-_DEPS = SOURCES + [os.path.join(CSRC, "so_kernels.cuh"), os.path.join(CSRC, "so_step_tma.cuh"),
+_DEPS = SOURCES + [os.path.join(CSRC, "so_kernels.cuh"), os.path.join(CSRC, "so_step_tma.cuh"), os.path.join(CSRC, "so_types.h"), os.path.join(CSRC, "so_pack.cuh"),
                    os.path.join(INCLUDE, "superoffload.h")]
 
 

@@ -26,23 +26,9 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "so_types.h"
+
 namespace so {
-
-constexpr int kTileElems = 1024;          // elements per warp tile
-constexpr int kRowElems = 128;            // 32 lanes x 4 elements
-constexpr int kRowsPerTile = kTileElems / kRowElems;
-constexpr int kThreads = 256;             // threads per block (8 warps)
-constexpr int kWarpsPerBlock = kThreads / 32;
-constexpr int kMaxBatch = 128;            // buckets per launch
-constexpr int kReduceThreads = 512;
-
-struct Geometry {
-    int64_t stride;                       // elements between slots
-    uint32_t tiles_per_slot;
-    uint32_t bucket_elems;
-    uint32_t last_elems;                  // elements in the last bucket
-    int32_t last_bucket;                  // its index (-1 if none)
-};
 
 // Gradient element types: uint16_t carries bf16 bit patterns, half_t IEEE
 // binary16 bit patterns (the only type that is used with a loss scale), float
@@ -52,51 +38,48 @@ struct half_t { uint16_t bits; };
 template <typename GradT> struct grad_traits { static constexpr bool kUnscale = false; };
 template <> struct grad_traits<half_t> { static constexpr bool kUnscale = true; };
 
-// Per-step constants, all derived on the host in double precision.
-struct AdamScalars {
-    double beta1, omb1;                   // beta1, 1 - beta1
-    double beta2, omb2;
-    double rsqrt_bc2;                     // 1 / sqrt(1 - beta2^t)
-    double step_size;                     // lr / (1 - beta1^t)
-    double decay;                         // 1 - lr * wd
-    double eps;
-    double lr, bc1, bc2;                  // unhoisted: lr, 1 - beta1^t, 1 - beta2^t
-    double scale;                         // gradient scale (clip coefficient)
-    double unscale;                       // 1 / loss scale (fp16 gradients), else 1
-};
+// Every kernel of the library may be launched as a programmatic dependent of
+// the kernel before it in the stream (its blocks are set up while that kernel
+// drains): nothing written by an earlier kernel may be read before this returns.
+__device__ __forceinline__ void wait_for_prior_kernels()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
 
-struct BucketEntry { int32_t bucket, src_slot, dst_slot; };
+__device__ __forceinline__ void allow_dependent_launch()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 
-struct StepArgs {
-    const void *grad;
-    float *master, *mom, *var;
-    uint16_t *param_bf16;
-    double *partials;
-    Geometry geo;
-    AdamScalars k;
-    int32_t n_entries;
-    BucketEntry e[kMaxBatch];
-};
+// Which of the prepared constant sets applies: a launch enqueued while the
+// previous validation was still pending reads how it ended from the device.
+__device__ __forceinline__ int outcome_index(int32_t pick, const Verdict *verdict)
+{
+    if (!pick) return kAfterKept;
+    const int32_t d = __ldcg(&verdict->decision);
+    return d == kDecisionSkip ? kAfterSkipped : d == kDecisionAbandon ? kAfterAbandoned : kAfterKept;
+}
 
-struct CheckArgs {
-    const void *grad;
-    double *partials;
-    double unscale;                       // 1 / loss scale (fp16 gradients), else 1
-    int32_t unscale_is_pow2;              // the product with `unscale` is exact
-    Geometry geo;
-    int32_t n_entries;
-    int32_t bucket[kMaxBatch];
-};
+// The slot tables and the verdict are rewritten by one kernel and read by the
+// next, which may already be resident when they change (dependent launches):
+// they are always read from L2 (ld.global.cg), never from an SM's L1.
+struct ResolvedEntry { int32_t bucket, src_slot, dst_slot; };
 
-struct CastArgs {
-    const float *master;
-    uint16_t *param_bf16;
-    Geometry geo;
-    int32_t n_entries;
-    BucketEntry e[kMaxBatch];             // dst_slot unused
-};
+// Slots of a speculative step: read the committed slot, write the spare one.
+__device__ __forceinline__ ResolvedEntry resolve_speculative(const SlotTables &t, BucketEntry e)
+{
+    return ResolvedEntry{e.bucket, __ldcg(&t.slot_of[e.bucket]), __ldcg(&t.free_slot[e.free_idx])};
+}
 
-struct BucketStats { double sumsq; int32_t nonfinite; int32_t pad; };
+// Slots of a step that follows a kept verdict, whose slot swap has already
+// happened: a speculated bucket is stepped again from its prior state (now in
+// the spare slot) into its committed slot (clip re-step); a bucket that was
+// only checked is stepped in place.
+__device__ __forceinline__ ResolvedEntry resolve_after_verdict(const SlotTables &t, BucketEntry e)
+{
+    const int32_t cur = __ldcg(&t.slot_of[e.bucket]);
+    return ResolvedEntry{e.bucket, e.free_idx >= 0 ? __ldcg(&t.free_slot[e.free_idx]) : cur, cur};
+}
 
 // ---------------------------------------------------------------------------
 // streaming loads / stores of one quad (4 consecutive elements)
@@ -193,11 +176,26 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     return d;
 }
 
-__device__ __forceinline__ void store_quad_bf16(uint16_t *base, uint32_t idx, uint32_t n,
-                                                const float (&x)[4])
+// fp32 pair -> packed IEEE binary16 pair, round to nearest even (overflow goes
+// to infinity, subnormals are kept).
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi)
 {
-    const uint32_t w0 = pack_bf16x2(x[0], x[1]);
-    const uint32_t w1 = pack_bf16x2(x[2], x[3]);
+    uint32_t d;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+// The low-precision parameter copy is bf16 or, for the paper's FP16 runs, binary16.
+__device__ __forceinline__ uint32_t pack_lp(float lo, float hi, bool fp16)
+{
+    return fp16 ? pack_f16x2(lo, hi) : pack_bf16x2(lo, hi);
+}
+
+__device__ __forceinline__ void store_quad_lp(uint16_t *base, uint32_t idx, uint32_t n,
+                                              const float (&x)[4], bool fp16)
+{
+    const uint32_t w0 = pack_lp(x[0], x[1], fp16);
+    const uint32_t w1 = pack_lp(x[2], x[3], fp16);
     if (idx + 4 <= n) {
         __stcs(reinterpret_cast<uint2 *>(base + idx), make_uint2(w0, w1));
     } else {
@@ -256,8 +254,8 @@ __device__ __forceinline__ double warp_fold(double x)
 // x + 1e-300: every non-zero second moment is at least 1e-93 (the square of the
 // smallest fp32 denormal times 1 - beta2), so the addition returns x itself,
 // and for x = 0 it keeps the seed finite so that g = 0 * seed = 0 comes out
-// exactly.  A NaN/Inf input only occurs in a speculative step that validation
-// discards.
+// exactly.  For x = +Inf (a second moment that overflowed fp32) the result is
+// NaN (Inf * 0); the caller then forms the element again with IEEE operations.
 __device__ __forceinline__ double sqrt_nonneg(double x)
 {
     double y;
@@ -285,16 +283,16 @@ __device__ __forceinline__ double rcp_pos(double b)
 }
 
 // One element, fast order.  Returns true when the new parameter came out below
-// 2^-16 of the old one, i.e. when the caller has to replace it by
+// 2^-16 of the old one (or not a number), i.e. when the caller has to replace it by
 // adamw_exact_p() of the ORIGINAL inputs (the check costs a multiply and a
 // compare; taking the branch here, per element, would stop the compiler from
 // interleaving the four dependent chains of a quad).
 template <bool kScaled, bool kUnscale>
 __device__ __forceinline__ bool adamw_element(float g, float &p, float &m, float &v,
-                                              const AdamScalars &k, double &sumsq)
+                                              const AdamScalars &k, double scale, double &sumsq)
 {
     const double gd = kUnscale ? __dmul_rn((double)g, k.unscale) : (double)g;
-    const double gs = kScaled ? __dmul_rn(gd, k.scale) : gd;
+    const double gs = kScaled ? __dmul_rn(gd, scale) : gd;
     const double sq = __dmul_rn(gs, gs);
     if (!kScaled) sumsq = __dadd_rn(sumsq, sq);
     const double m64 = __dadd_rn(__dmul_rn(k.beta1, (double)m), __dmul_rn(k.omb1, gs));
@@ -302,7 +300,10 @@ __device__ __forceinline__ bool adamw_element(float g, float &p, float &m, float
     const double denom = __fma_rn(sqrt_nonneg(v64), k.rsqrt_bc2, k.eps);
     const double u = __dmul_rn(__dmul_rn(k.step_size, m64), rcp_pos(denom));
     const double p64 = __fma_rn((double)p, k.decay, -u);
-    const bool cancelled = fabs(p64) < __dmul_rn(fabs((double)p), 0x1p-16);
+    // negated >=, so that a NaN here (a second moment that reached +Inf makes the
+    // straight-line square root produce one) also takes the textbook order,
+    // whose IEEE operations handle infinities
+    const bool cancelled = !(fabs(p64) >= __dmul_rn(fabs((double)p), 0x1p-16));
     p = __double2float_rn(p64);
     m = __double2float_rn(m64);
     v = __double2float_rn(v64);
@@ -314,10 +315,10 @@ __device__ __forceinline__ bool adamw_element(float g, float &p, float &m, float
 // mhat = m'/bc1, vhat = v'/bc2, p' = p*(1 - lr*wd) - lr*(mhat/(sqrt(vhat) + eps)).
 template <bool kScaled, bool kUnscale>
 __device__ __forceinline__ float adamw_exact_p(float g, float p, float m, float v,
-                                               const AdamScalars &k)
+                                               const AdamScalars &k, double scale)
 {
     const double gd = kUnscale ? __dmul_rn((double)g, k.unscale) : (double)g;
-    const double gs = kScaled ? __dmul_rn(gd, k.scale) : gd;
+    const double gs = kScaled ? __dmul_rn(gd, scale) : gd;
     const double m64 = __dadd_rn(__dmul_rn(k.beta1, (double)m), __dmul_rn(k.omb1, gs));
     const double v64 = __dadd_rn(__dmul_rn(k.beta2, (double)v), __dmul_rn(k.omb2, __dmul_rn(gs, gs)));
     const double mhat = __ddiv_rn(m64, k.bc1);
@@ -331,13 +332,13 @@ __device__ __forceinline__ float adamw_exact_p(float g, float p, float m, float 
 // element past the end of a bucket is all zeros and stays zero).
 template <bool kScaled, bool kUnscale>
 static __device__ __noinline__ float4 adamw_exact_quad(float4 g, float4 p, float4 m, float4 v,
-                                                       const AdamScalars &k)
+                                                       const AdamScalars &k, double scale)
 {
     float4 r;
-    r.x = adamw_exact_p<kScaled, kUnscale>(g.x, p.x, m.x, v.x, k);
-    r.y = adamw_exact_p<kScaled, kUnscale>(g.y, p.y, m.y, v.y, k);
-    r.z = adamw_exact_p<kScaled, kUnscale>(g.z, p.z, m.z, v.z, k);
-    r.w = adamw_exact_p<kScaled, kUnscale>(g.w, p.w, m.w, v.w, k);
+    r.x = adamw_exact_p<kScaled, kUnscale>(g.x, p.x, m.x, v.x, k, scale);
+    r.y = adamw_exact_p<kScaled, kUnscale>(g.y, p.y, m.y, v.y, k, scale);
+    r.z = adamw_exact_p<kScaled, kUnscale>(g.z, p.z, m.z, v.z, k, scale);
+    r.w = adamw_exact_p<kScaled, kUnscale>(g.w, p.w, m.w, v.w, k, scale);
     return r;
 }
 
@@ -348,10 +349,11 @@ template <typename GradT, bool kScaled>
 static __device__ __noinline__ float4 adamw_exact_quad_at(const GradT *g, const float *p,
                                                           const float *m, const float *v,
                                                           uint32_t idx, uint32_t n,
-                                                          const AdamScalars &k)
+                                                          const AdamScalars &k, double scale)
 {
     return adamw_exact_quad<kScaled, grad_traits<GradT>::kUnscale>(
-        load_quad4(g, idx, n), load_quad4(p, idx, n), load_quad4(m, idx, n), load_quad4(v, idx, n), k);
+        load_quad4(g, idx, n), load_quad4(p, idx, n), load_quad4(m, idx, n), load_quad4(v, idx, n), k,
+        scale);
 }
 
 // The four elements of a lane's quad; `reload` forms the quad again in the
@@ -359,13 +361,13 @@ static __device__ __noinline__ float4 adamw_exact_quad_at(const GradT *g, const 
 // registers by then) and is only called when one of the four cancelled.
 template <bool kScaled, bool kUnscale, typename Reload>
 __device__ __forceinline__ void adamw_quad(const float (&gq)[4], float (&pq)[4], float (&mq)[4],
-                                           float (&vq)[4], const AdamScalars &k, double (&acc)[4],
-                                           Reload reload)
+                                           float (&vq)[4], const AdamScalars &k, double scale,
+                                           double (&acc)[4], Reload reload)
 {
     bool redo = false;
 #pragma unroll
     for (int q = 0; q < 4; ++q)
-        redo |= adamw_element<kScaled, kUnscale>(gq[q], pq[q], mq[q], vq[q], k, acc[q]);
+        redo |= adamw_element<kScaled, kUnscale>(gq[q], pq[q], mq[q], vq[q], k, scale, acc[q]);
     if (__builtin_expect(redo, false)) {
         const float4 e = reload();
         pq[0] = e.x; pq[1] = e.y; pq[2] = e.z; pq[3] = e.w;
@@ -376,24 +378,93 @@ __device__ __forceinline__ void adamw_quad(const float (&gq)[4], float (&pq)[4],
 // fused step: g, p, m, v in -> p', m', v', bf16(p') out (+ tile sums of g^2)
 // ---------------------------------------------------------------------------
 //
-// kSpec = true : speculative step (scale 1, tile sums written).
-// kSpec = false: step with a known scale (re-step after a clip, or the in-place
-//                step of a bucket that was only checked); no sums.
+// kSpec = true : speculative step (scale 1, tile sums written, new state into
+//                the bucket's spare slot).
+// kSpec = false: the step that follows a verdict, with the scale the verdict
+//                fixed and no sums: after a clip every bucket of the launch
+//                (speculated ones from their prior state, the others in
+//                place), after a commit only the buckets that were merely
+//                checked, after a skip nothing.
 // Source and destination slots may be the same slot (in-place): every element
 // is read and written by the same thread, reads first.
+
+// What a follow-up launch does, read from the device verdict.
+struct FollowUp { bool step_all, step_inplace, recast; double scale; };
+
+__device__ __forceinline__ FollowUp follow_up_of(const Verdict *verdict)
+{
+    const int32_t d = __ldcg(&verdict->decision);
+    FollowUp f;
+    f.step_all = d == kDecisionClip;
+    f.step_inplace = d == kDecisionCommit;
+    f.recast = d == kDecisionSkip || d == kDecisionAbandon;
+    f.scale = d == kDecisionClip ? __ldcg(&verdict->coef) : 1.0;
+    return f;
+}
+
+// bf16/fp16 copy of a speculated bucket derived again from its untouched
+// committed master (after a skip): tiles dealt round-robin to all warps.
+__device__ __forceinline__ void recast_speculated(const BucketEntry *e, int n_entries,
+                                                  const SlotTables &tab, const Geometry &geo,
+                                                  const float *master, uint16_t *param_lp, bool fp16,
+                                                  uint32_t warp, uint32_t n_warps, uint32_t lane)
+{
+    const uint32_t tps = geo.tiles_per_slot;
+    const uint32_t total_tiles = (uint32_t)n_entries * tps;
+    for (uint32_t tile = warp; tile < total_tiles; tile += n_warps) {
+        const uint32_t j = tile / tps;
+        const uint32_t lt = tile - j * tps;
+        if (e[j].free_idx < 0) continue;
+        const int32_t b = e[j].bucket;
+        const uint32_t n = (b == geo.last_bucket) ? geo.last_elems : geo.bucket_elems;
+        const uint32_t base = lt * kTileElems;
+        if (base >= n) continue;
+        const float *p = master + (int64_t)__ldcg(&tab.slot_of[b]) * geo.stride;
+        uint16_t *pb = param_lp + (int64_t)b * geo.stride;
+#pragma unroll 2
+        for (int r = 0; r < kRowsPerTile; ++r) {
+            const uint32_t idx = base + r * kRowElems + lane * 4;
+            if (idx < n) {
+                float pq[4];
+                load_quad(p, idx, n, pq);
+                store_quad_lp(pb, idx, n, pq, fp16);
+            }
+        }
+    }
+}
+
 template <typename GradT, bool kSpec, int kRowsInFlight>
 __global__ void __launch_bounds__(kThreads, 2) adamw_step_kernel(const __grid_constant__ StepArgs a)
 {
+    wait_for_prior_kernels();
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     const uint32_t tps = a.geo.tiles_per_slot;
     const uint32_t total_tiles = (uint32_t)a.n_entries * tps;
+    const AdamScalars &k = a.k[outcome_index(a.pick, a.tab.verdict)];
+    const bool fp16 = a.param_fp16 != 0;
+
+    FollowUp f{};
+    f.scale = 1.0;
+    if constexpr (kSpec) {
+        if (blockIdx.x == 0 && (int)threadIdx.x < a.n_entries)
+            a.tab.spec_idx[a.e[threadIdx.x].bucket] = a.e[threadIdx.x].free_idx;
+    } else {
+        f = follow_up_of(a.tab.verdict);
+        if (f.recast) {
+            recast_speculated(a.e, a.n_entries, a.tab, a.geo, a.master, a.param_lp, fp16, warp,
+                              n_warps, lane);
+            return;
+        }
+    }
 
     for (uint32_t tile = warp; tile < total_tiles; tile += n_warps) {
         const uint32_t j = tile / tps;
         const uint32_t lt = tile - j * tps;
-        const BucketEntry e = a.e[j];
+        if (!kSpec && !f.step_all && a.e[j].free_idx >= 0) continue;    // kept as speculated
+        const ResolvedEntry e = kSpec ? resolve_speculative(a.tab, a.e[j])
+                                      : resolve_after_verdict(a.tab, a.e[j]);
         const uint32_t n = (e.bucket == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
         const uint32_t base = lt * kTileElems;
         if (base >= n) continue;
@@ -403,7 +474,7 @@ __global__ void __launch_bounds__(kThreads, 2) adamw_step_kernel(const __grid_co
         const int64_t dst = (int64_t)e.dst_slot * a.geo.stride;
         const float *p_in = a.master + src, *m_in = a.mom + src, *v_in = a.var + src;
         float *p_out = a.master + dst, *m_out = a.mom + dst, *v_out = a.var + dst;
-        uint16_t *pb = a.param_bf16 + (int64_t)e.bucket * a.geo.stride;
+        uint16_t *pb = a.param_lp + (int64_t)e.bucket * a.geo.stride;
 
         double acc[4] = {0.0, 0.0, 0.0, 0.0};
 #pragma unroll 1
@@ -423,15 +494,16 @@ __global__ void __launch_bounds__(kThreads, 2) adamw_step_kernel(const __grid_co
             for (int u = 0; u < kRowsInFlight; ++u) {
                 const uint32_t idx = base + (r0 + u) * kRowElems + lane * 4;
                 adamw_quad<!kSpec, grad_traits<GradT>::kUnscale>(
-                    gq[u], pq[u], mq[u], vq[u], a.k, acc,
+                    gq[u], pq[u], mq[u], vq[u], k, f.scale, acc,
                     [&]() {                    // not stored yet: still the inputs
-                        return adamw_exact_quad_at<GradT, !kSpec>(g, p_in, m_in, v_in, idx, n, a.k);
+                        return adamw_exact_quad_at<GradT, !kSpec>(g, p_in, m_in, v_in, idx, n, k,
+                                                                  f.scale);
                     });
                 if (idx < n) {
                     store_quad(p_out, idx, n, pq[u]);
                     store_quad(m_out, idx, n, mq[u]);
                     store_quad(v_out, idx, n, vq[u]);
-                    store_quad_bf16(pb, idx, n, pq[u]);
+                    store_quad_lp(pb, idx, n, pq[u], fp16);
                 }
             }
         }
@@ -483,6 +555,8 @@ grad_check_kernel(const __grid_constant__ CheckArgs a)
     const uint32_t tps = a.geo.tiles_per_slot;
     const uint32_t n_entries = (uint32_t)a.n_entries;
     const GradT *grad = static_cast<const GradT *>(a.grad);
+    wait_for_prior_kernels();
+    const double unscale = a.unscale[outcome_index(a.pick, a.verdict)];
 
     // Position of the next tile to fetch, kept as (entry, tile within the slot)
     // and advanced by the grid's stride without a division.
@@ -529,9 +603,10 @@ grad_check_kernel(const __grid_constant__ CheckArgs a)
     // times a power of two (the usual loss scales); with any other scale the
     // unscaled value has a full double mantissa and keeps the two separately
     // rounded operations.
-    const bool exact_square = !kUnscale || a.unscale_is_pow2 != 0;
+    const bool exact_square = !kUnscale || (__double2loint(unscale) == 0 &&
+                                            (__double2hiint(unscale) & 0x000FFFFF) == 0);
     auto square_add = [&](float x, double &acc) {
-        const double gd = kUnscale ? __dmul_rn((double)x, a.unscale) : (double)x;
+        const double gd = kUnscale ? __dmul_rn((double)x, unscale) : (double)x;
         if (exact_square) acc = __fma_rn(gd, gd, acc);
         else acc = __dadd_rn(acc, __dmul_rn(gd, gd));
     };
@@ -577,7 +652,7 @@ grad_check_kernel(const __grid_constant__ CheckArgs a)
 }
 
 // ---------------------------------------------------------------------------
-// per-bucket fold of the tile sums (fixed order) + non-finite flag
+// per-bucket fold of the tile sums (fixed order) + non-finite flag + verdict
 // ---------------------------------------------------------------------------
 //
 // g^2 is formed in double, so it cannot overflow for a finite fp32/bf16 input,
@@ -587,27 +662,14 @@ grad_check_kernel(const __grid_constant__ CheckArgs a)
 // A bucket's tile sums are cut into segments of 4096 tiles.  One block folds
 // one segment (each thread adds up to 8 strided tile sums, then a shared-memory
 // tree); the block that finishes a bucket's last outstanding segment folds the
-// segment sums the same way and publishes the bucket's record.  Segment
-// boundaries and both fold orders are fixed, so the result does not depend on
-// which block happens to come last.  The per-bucket arrival counters start at
-// zero (bind) and are put back to zero by the publishing block.
-constexpr int kSegTiles = 4096;
-
-struct SegSum { double sum; int32_t bad; int32_t pad; };
-
-struct ReduceArgs {
-    const double *partials;        // tile sums
-    SegSum *seg;                   // n_buckets x segs_per_slot
-    uint32_t *arrivals;            // n_buckets
-    BucketStats *stats;            // device copy of the records
-    BucketStats *host_stats;       // mapped host copy, or nullptr
-    const int32_t *status;         // device status word, mirrored after the records
-    uint32_t *buckets_done;        // arrival counter over buckets (starts and ends at zero)
-    int32_t seq;                   // stamp of this reduction, written last
-    Geometry geo;
-    uint32_t segs_per_slot;
-    int32_t n_buckets;
-};
+// segment sums the same way and publishes the bucket's record; the block that
+// publishes the last bucket folds the bucket sums in index order, forms the
+// verdict (norm, clip coefficient, decision), re-points the speculated buckets
+// at their new slots if the iteration is kept, and leaves records and verdict
+// in mapped host memory.  Segment boundaries and all fold orders are fixed, so
+// the result does not depend on which block happens to come last.  The arrival
+// counters start at zero (bind) and are put back to zero by the publishing
+// blocks.
 
 // Fold `count` doubles starting at src (stride 1) in the fixed block order.
 __device__ __forceinline__ void block_fold(const double *src, uint32_t count, double *s_sum,
@@ -636,14 +698,74 @@ __device__ __forceinline__ void block_fold(const double *src, uint32_t count, do
     __syncthreads();
 }
 
+// Norm, clip coefficient and decision from the global sum and flag.  Square
+// root, addition and division are IEEE correctly rounded, so a host that does
+// the same three operations on the same sum gets the same bits.
+__device__ __forceinline__ Verdict make_verdict(double sumsq, int nonfinite, int status,
+                                                double max_grad_norm, int32_t seq)
+{
+    Verdict v;
+    v.sumsq = sumsq;
+    v.norm = __dsqrt_rn(sumsq);
+    v.coef = 1.0;
+    if (max_grad_norm > 0.0) {
+        const double c = __ddiv_rn(max_grad_norm, __dadd_rn(v.norm, 1e-6));
+        v.coef = c < 1.0 ? c : 1.0;
+    }
+    v.nonfinite = nonfinite != 0;
+    v.decision = status != 0       ? kDecisionAbandon
+                 : v.nonfinite     ? kDecisionSkip
+                 : v.coef < 1.0    ? kDecisionClip
+                                   : kDecisionCommit;
+    v.status = status;
+    v.seq = seq;
+    v.pad[0] = v.pad[1] = 0;
+    return v;
+}
+
+// Executed by one whole block of kReduceThreads threads: act on the verdict
+// (a kept iteration swaps every speculated bucket's committed and spare slot;
+// any verdict clears the speculation marks), then publish it, device copy
+// first, host copy with its stamp last.
+__device__ __forceinline__ void publish_verdict(const Verdict &v, const SlotTables &tab,
+                                                int32_t n_buckets, Verdict *host_verdict)
+{
+    const bool kept = v.decision == kDecisionCommit || v.decision == kDecisionClip;
+    for (int32_t b = threadIdx.x; b < n_buckets; b += kReduceThreads) {
+        const int32_t j = __ldcg(&tab.spec_idx[b]);
+        if (j >= 0) {
+            if (kept) {
+                const int32_t old_slot = __ldcg(&tab.slot_of[b]);
+                tab.slot_of[b] = __ldcg(&tab.free_slot[j]);
+                tab.free_slot[j] = old_slot;
+            }
+            tab.spec_idx[b] = -1;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        *const_cast<Verdict *>(tab.verdict) = v;
+        if (host_verdict) {
+            volatile Verdict *h = host_verdict;
+            h->sumsq = v.sumsq;
+            h->norm = v.norm;
+            h->coef = v.coef;
+            h->nonfinite = v.nonfinite;
+            h->decision = v.decision;
+            h->status = v.status;
+            __threadfence_system();
+            h->seq = v.seq;
+        }
+    }
+}
+
 static __global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(const ReduceArgs a)
 {
     __shared__ double s_sum[kReduceThreads];
     __shared__ int s_bad[kReduceThreads];
     __shared__ int s_last;
-    // launched as a programmatic dependent of the kernel before it: nothing of
-    // that kernel's output may be read before this returns
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    wait_for_prior_kernels();
+    allow_dependent_launch();      // the kernel after this one waits for our completion itself
     const int32_t b = (int32_t)(blockIdx.x / a.segs_per_slot);
     const uint32_t seg = blockIdx.x - (uint32_t)b * a.segs_per_slot;
     const uint32_t n = (b == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
@@ -671,8 +793,8 @@ static __global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(co
     double acc = 0.0;
     int any_bad = 0;
     for (uint32_t i = threadIdx.x; i < n_segs; i += kReduceThreads) {
-        acc = __dadd_rn(acc, segs[i].sum);
-        any_bad |= segs[i].bad;
+        acc = __dadd_rn(acc, __ldcg(&segs[i].sum));
+        any_bad |= __ldcg(&segs[i].bad);
     }
     s_sum[threadIdx.x] = acc;
     s_bad[threadIdx.x] = any_bad;
@@ -691,56 +813,104 @@ static __global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(co
         r.pad = 0;
         a.stats[b] = r;
         a.arrivals[b] = 0;
-        s_last = 0;
-        if (a.host_stats) {
-            __threadfence();
-            s_last = (atomicAdd(a.buckets_done, 1u) == (uint32_t)a.n_buckets - 1u);
-        }
+        __threadfence();
+        s_last = (atomicAdd(a.buckets_done, 1u) == (uint32_t)a.n_buckets - 1u);
     }
     __syncthreads();
     if (!s_last) return;
 
     // This block published the last bucket.  It alone writes to the mapped
-    // host copy: all records, one system-wide fence, then the stamp -- a host
-    // that sees the stamp therefore sees every record, and the kernel pays for
-    // two trips to host memory instead of one per bucket.
+    // host copy: all records, the verdict, one system-wide fence, then the
+    // stamp -- a host that sees the stamp therefore sees everything, and the
+    // kernel pays for two trips to host memory instead of one per bucket.
     __threadfence();
-    for (int32_t i = threadIdx.x; i < a.n_buckets; i += kReduceThreads) {
-        // records of other blocks: read them from L2, not from a stale L1 line
-        const int4 rec = __ldcg(reinterpret_cast<const int4 *>(a.stats + i));
-        *reinterpret_cast<int4 *>(a.host_stats + i) = rec;
+    double total = 0.0;
+    int flag = 0;
+    for (int32_t first = 0; first < a.n_buckets; first += kReduceThreads) {
+        const int32_t i = first + (int32_t)threadIdx.x;
+        __syncthreads();
+        if (i < a.n_buckets) {
+            // records of other blocks: read them from L2, not from a stale L1 line
+            const int4 rec = __ldcg(reinterpret_cast<const int4 *>(a.stats + i));
+            if (a.host_stats) *reinterpret_cast<int4 *>(a.host_stats + i) = rec;
+            s_sum[threadIdx.x] = __hiloint2double(rec.y, rec.x);
+            s_bad[threadIdx.x] = rec.z;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            // bucket sums are added one after the other in index order
+            const int32_t m = a.n_buckets - first < kReduceThreads ? a.n_buckets - first : kReduceThreads;
+            for (int32_t q = 0; q < m; ++q) {
+                total = __dadd_rn(total, s_sum[q]);
+                flag |= (s_bad[q] != 0);
+            }
+        }
     }
-    __threadfence_system();
-    __syncthreads();
+    __shared__ Verdict s_verdict;
     if (threadIdx.x == 0) {
         *a.buckets_done = 0;
-        volatile BucketStats *trailer = a.host_stats + a.n_buckets;
-        trailer->nonfinite = *a.status;
+        const int status = atomicExch(a.status, 0);
+        s_verdict = make_verdict(total, flag, status, a.max_grad_norm, a.seq);
+        if (!a.decide) s_verdict.decision = -1;
+    }
+    __syncthreads();
+    Verdict *host_verdict =
+        a.host_stats ? reinterpret_cast<Verdict *>(a.host_stats + a.n_buckets) : nullptr;
+    if (a.decide) {
+        publish_verdict(s_verdict, a.tab, a.n_buckets, host_verdict);
+    } else if (threadIdx.x == 0 && host_verdict) {
+        // a check without a decision: only the sum, the flag and the stamp travel
+        volatile Verdict *h = host_verdict;
+        h->sumsq = s_verdict.sumsq;
+        h->nonfinite = s_verdict.nonfinite;
+        h->decision = -1;
+        h->status = s_verdict.status;
         __threadfence_system();
-        trailer->pad = a.seq;
+        h->seq = s_verdict.seq;
+    }
+    if (!a.decide && threadIdx.x == 0) {
+        // the device copy that follows the records (read back when the host copy is not mapped)
+        Verdict *d = reinterpret_cast<Verdict *>(a.stats + a.n_buckets);
+        *d = s_verdict;
     }
 }
 
+// The verdict from a sum and a flag the host supplies: after so_grad_check(SO_ALL)
+// (whose reduction did not decide), or with the statistics of all ranks when the
+// optimizer states are sharded.  One block.
+static __global__ void __launch_bounds__(kReduceThreads) apply_verdict_kernel(const VerdictArgs a)
+{
+    __shared__ Verdict s_verdict;
+    wait_for_prior_kernels();
+    allow_dependent_launch();
+    if (threadIdx.x == 0)
+        s_verdict = make_verdict(a.sumsq, a.nonfinite, a.abandon, a.max_grad_norm, a.seq);
+    __syncthreads();
+    publish_verdict(s_verdict, a.tab, a.n_buckets, a.host_verdict);
+}
+
 // ---------------------------------------------------------------------------
-// stand-alone cast: fp32 master (slot src) -> bf16 copy of the bucket
+// stand-alone cast: committed fp32 master -> low-precision copy of the bucket
 // ---------------------------------------------------------------------------
 static __global__ void __launch_bounds__(kThreads) cast_params_kernel(const __grid_constant__ CastArgs a)
 {
+    wait_for_prior_kernels();
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;
     const uint32_t tps = a.geo.tiles_per_slot;
     const uint32_t total_tiles = (uint32_t)a.n_entries * tps;
+    const bool fp16 = a.param_fp16 != 0;
 
     for (uint32_t tile = warp; tile < total_tiles; tile += n_warps) {
         const uint32_t j = tile / tps;
         const uint32_t lt = tile - j * tps;
-        const BucketEntry e = a.e[j];
-        const uint32_t n = (e.bucket == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
+        const int32_t b = a.bucket[j];
+        const uint32_t n = (b == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
         const uint32_t base = lt * kTileElems;
         if (base >= n) continue;
-        const float *p = a.master + (int64_t)e.src_slot * a.geo.stride;
-        uint16_t *pb = a.param_bf16 + (int64_t)e.bucket * a.geo.stride;
+        const float *p = a.master + (int64_t)__ldcg(&a.tab.slot_of[b]) * a.geo.stride;
+        uint16_t *pb = a.param_lp + (int64_t)b * a.geo.stride;
 
         float pq[kRowsPerTile][4];
 #pragma unroll
@@ -751,7 +921,7 @@ static __global__ void __launch_bounds__(kThreads) cast_params_kernel(const __gr
 #pragma unroll
         for (int r = 0; r < kRowsPerTile; ++r) {
             const uint32_t idx = base + r * kRowElems + lane * 4;
-            if (idx < n) store_quad_bf16(pb, idx, n, pq[r]);
+            if (idx < n) store_quad_lp(pb, idx, n, pq[r], fp16);
         }
     }
 }

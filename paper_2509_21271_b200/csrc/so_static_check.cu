@@ -15,7 +15,7 @@
 #include <cmath>
 #include <mutex>
 
-#include "so_kernels.cuh"
+#include "so_types.h"
 
 using namespace so;
 
@@ -35,7 +35,7 @@ struct DeviceSetup {
     bool ready = false;
     double *tile_sums = nullptr;      // device address of g_tile_sums on this device
     int num_sms = 0;
-    int occ_check = 0;
+    int occ_check = 0, occ_check_f32 = 0;
 };
 
 DeviceSetup g_setup[kMaxDevices];
@@ -99,8 +99,9 @@ so_status setup_device(int device, DeviceSetup **out)
         if (e != cudaSuccess || ptr == nullptr) return SO_ERR_CUDA;
         e = cudaDeviceGetAttribute(&d.num_sms, cudaDevAttrMultiProcessorCount, device);
         if (e != cudaSuccess) return SO_ERR_CUDA;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.occ_check, grad_check_kernel<uint16_t>,
-                                                          kThreads, 0);
+        e = grad_check_occupancy(SO_GRAD_BF16, &d.occ_check);
+        if (e != cudaSuccess) return SO_ERR_CUDA;
+        e = grad_check_occupancy(SO_GRAD_FP32, &d.occ_check_f32);
         if (e != cudaSuccess) return SO_ERR_CUDA;
         d.tile_sums = ptr;
         d.ready = true;
@@ -137,8 +138,9 @@ extern "C" so_status so_grad_check_static(const void *grad, int64_t n_elems, int
         CheckArgs a;
         a.grad = grad;
         a.partials = d->tile_sums;
-        a.unscale = 1.0;
-        a.unscale_is_pow2 = 1;
+        a.unscale[0] = a.unscale[1] = a.unscale[2] = 1.0;
+        a.verdict = nullptr;
+        a.pick = 0;
         a.geo.stride = 0;
         a.geo.tiles_per_slot = n_tiles;
         a.geo.bucket_elems = (uint32_t)n_elems;
@@ -147,12 +149,10 @@ extern "C" so_status so_grad_check_static(const void *grad, int64_t n_elems, int
         a.n_entries = 1;
         for (int i = 0; i < kMaxBatch; ++i) a.bucket[i] = 0;
         int64_t blocks = ((int64_t)n_tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
-        const int64_t cap = (int64_t)d->num_sms * (d->occ_check > 0 ? d->occ_check : 1);
+        const int occ = grad_dtype == SO_GRAD_BF16 ? d->occ_check : d->occ_check_f32;
+        const int64_t cap = (int64_t)d->num_sms * (occ > 0 ? occ : 1);
         if (blocks > cap) blocks = cap;
-        if (grad_dtype == SO_GRAD_BF16)
-            grad_check_kernel<uint16_t><<<(unsigned)blocks, kThreads, 0, st>>>(a);
-        else
-            grad_check_kernel<float><<<(unsigned)blocks, kThreads, 0, st>>>(a);
+        if (launch_grad_check(a, grad_dtype, (unsigned)blocks, st) != cudaSuccess) return SO_ERR_CUDA;
         if (cudaGetLastError() != cudaSuccess) return SO_ERR_CUDA;
     }
     static_check_finish_kernel<<<1, kReduceThreads, 0, st>>>(d->tile_sums, n_tiles, max_grad_norm,

@@ -40,24 +40,6 @@
 
 namespace so {
 
-constexpr uint32_t kSpinLimit = 1u << 20;              // bounded mbarrier polling
-// Launches of one context that may be outstanding at a time (enqueued and not
-// yet finished, on whatever streams).  A launch takes the next pair of the ring;
-// within one stream a pair's previous user has finished and re-armed it long
-// before it comes round again, and across streams the ring is long enough that
-// one stream would have to run 4096 launches ahead of another for two running
-// kernels to meet on a pair.
-constexpr int kCounterPairs = 4096;
-
-// Control block in scratch (zeroed once at bind time): a status record and a
-// ring of {next tile, finished warps} counter pairs, one pair per launch.
-struct ControlBlock {
-    int32_t status;
-    uint32_t buckets_done;     // arrival counter of the bucket reduction
-    int32_t pad[2];
-    uint32_t counters[kCounterPairs][2];
-};
-
 // Shape of the per-warp pipeline: rows (of 128 elements) per chunk, warps per
 // block (one block per SM), chunks in flight ahead of the arithmetic, and
 // output staging buffers.
@@ -91,8 +73,11 @@ struct TmaLayout {
     static constexpr int kInStage = 3 * kF32Bytes + kGradBytes;            // p, m, v, g
     static constexpr int kOutStage = 3 * kF32Bytes + S::kChunkElems * 2;   // p, m, v, bf16
     static constexpr int kWarpBytes = S::kStagesIn * kInStage + S::kStagesOut * kOutStage;
-    // per warp and input stage: one mbarrier (8 B) and one descriptor (32 B)
-    static constexpr int kHeaderBytes = 128 * ((S::kWarps * S::kStagesIn * 40 + 127) / 128);
+    // per warp and input stage: one mbarrier (8 B) and one descriptor (32 B);
+    // then the launch's buckets with their slots resolved, and their count
+    static constexpr int kEntriesOffset = S::kWarps * S::kStagesIn * 40;
+    static constexpr int kHeaderBytes =
+        128 * ((kEntriesOffset + kMaxBatch * (int)sizeof(ResolvedEntry) + 16 + 127) / 128);
     static constexpr int kSmemBytes = kHeaderBytes + S::kWarps * kWarpBytes;
 };
 
@@ -127,10 +112,10 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok;
 }
 
-// Bounded wait; returns false if the phase did not complete in time.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+// Bounded wait; returns false if the phase did not complete within `limit` polls.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit)
 {
-    for (uint32_t it = 0; it < kSpinLimit; ++it)
+    for (uint32_t it = 0; it < limit; ++it)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -188,15 +173,48 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
     const uint32_t wib = threadIdx.x >> 5;
     const uint32_t n_warps = gridDim.x * kTmaWarps;
     const uint32_t tps = a.geo.tiles_per_slot;
-    const uint32_t total_tiles = (uint32_t)a.n_entries * tps;
 
     const uint32_t bars = smem_u32(smem) + wib * kStagesIn * 8;
     ChunkDesc *descs = reinterpret_cast<ChunkDesc *>(smem + kTmaWarps * kStagesIn * 8) +
                        wib * kStagesIn;
+    ResolvedEntry *entries = reinterpret_cast<ResolvedEntry *>(smem + L::kEntriesOffset);
+    int32_t *n_active_smem = reinterpret_cast<int32_t *>(entries + kMaxBatch);
     unsigned char *wbase = smem + L::kHeaderBytes + wib * L::kWarpBytes;
     unsigned char *out_base = wbase + kStagesIn * L::kInStage;
     uint32_t *next_tile = &ctrl->counters[pair][0];
     uint32_t *done_warps = &ctrl->counters[pair][1];
+
+    // ---- which buckets, which slots, which constants ----
+    wait_for_prior_kernels();
+    const AdamScalars &k = a.k[outcome_index(a.pick, a.tab.verdict)];
+    const bool fp16 = a.param_fp16 != 0;
+    double scale = 1.0;
+    if constexpr (kSpec) {
+        for (int i = threadIdx.x; i < a.n_entries; i += S::kThreads) {
+            entries[i] = resolve_speculative(a.tab, a.e[i]);
+            if (blockIdx.x == 0) a.tab.spec_idx[a.e[i].bucket] = a.e[i].free_idx;
+        }
+        if (threadIdx.x == 0) *n_active_smem = a.n_entries;
+    } else {
+        const FollowUp f = follow_up_of(a.tab.verdict);
+        if (f.recast) {
+            recast_speculated(a.e, a.n_entries, a.tab, a.geo, a.master, a.param_lp, fp16,
+                              blockIdx.x * kTmaWarps + wib, n_warps, lane);
+            return;
+        }
+        scale = f.scale;
+        if (threadIdx.x == 0) {
+            int32_t n = 0;
+            for (int i = 0; i < a.n_entries; ++i)
+                if (f.step_all || a.e[i].free_idx < 0) entries[n++] = resolve_after_verdict(a.tab, a.e[i]);
+            *n_active_smem = n;
+        }
+    }
+    __syncthreads();
+    // nothing to do (a commit with every bucket speculated): the same in every
+    // block, so no warp of the launch touches the tile counters
+    if (*n_active_smem == 0) return;
+    const uint32_t total_tiles = (uint32_t)*n_active_smem * tps;
 
     const uint64_t policy = l2_evict_first_policy();
     const int64_t stride = a.geo.stride;
@@ -219,7 +237,7 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
             }
             const uint32_t j = cur_tile / tps;
             const uint32_t lt = cur_tile - j * tps;
-            const BucketEntry e = a.e[j];
+            const ResolvedEntry e = entries[j];
             const uint32_t n =
                 (e.bucket == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
             if (lt * kTileElems < n) {
@@ -301,13 +319,13 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
         const uint32_t len = d.len, start = d.start;
         const bool bulk = (d.flags & kRagged) == 0;
         const int64_t dst = (int64_t)d.dst_slot * stride;
-        uint16_t *pb = a.param_bf16 + (int64_t)d.bucket * stride;
+        uint16_t *pb = a.param_lp + (int64_t)d.bucket * stride;
 
         if (bulk) {
             // every lane polls the same barrier; the verdict is made warp-wide so
             // that no lane leaves the loop while others go on to a __syncwarp
-            if (!__all_sync(0xFFFFFFFFu,
-                            mbar_wait_bounded(bars + stage * 8, (phases >> stage) & 1u))) {
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(bars + stage * 8, (phases >> stage) & 1u,
+                                                           a.spin_limit))) {
                 failed = true;
                 break;
             }
@@ -340,7 +358,7 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                     gq[0] = g4.x; gq[1] = g4.y; gq[2] = g4.z; gq[3] = g4.w;
                 }
                 adamw_quad<!kSpec, grad_traits<GradT>::kUnscale>(
-                    gq, pq, mq, vq, a.k, acc,
+                    gq, pq, mq, vq, k, scale, acc,
                     [&]() {
                         // the input stage is refilled only after this loop
                         float4 g0;
@@ -354,7 +372,8 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                         } else {
                             g0 = *reinterpret_cast<const float4 *>(in + 3 * L::kF32Bytes + off * 4);
                         }
-                        return adamw_exact_quad<!kSpec, grad_traits<GradT>::kUnscale>(g0, p0, m0, v0, a.k);
+                        return adamw_exact_quad<!kSpec, grad_traits<GradT>::kUnscale>(g0, p0, m0, v0, k,
+                                                                                      scale);
                     });
                 *reinterpret_cast<float4 *>(out + off * 4) = make_float4(pq[0], pq[1], pq[2], pq[3]);
                 *reinterpret_cast<float4 *>(out + L::kF32Bytes + off * 4) =
@@ -362,7 +381,7 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                 *reinterpret_cast<float4 *>(out + 2 * L::kF32Bytes + off * 4) =
                     make_float4(vq[0], vq[1], vq[2], vq[3]);
                 *reinterpret_cast<uint2 *>(out + 3 * L::kF32Bytes + off * 2) =
-                    make_uint2(pack_bf16x2(pq[0], pq[1]), pack_bf16x2(pq[2], pq[3]));
+                    make_uint2(pack_lp(pq[0], pq[1], fp16), pack_lp(pq[2], pq[3], fp16));
             }
             fence_async_smem();        // generic writes -> visible to the async proxy
             // every lane is done with the input stage and has filled its part
@@ -391,16 +410,16 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                 load_quad(a.mom + src, idx, d.n, mq);
                 load_quad(a.var + src, idx, d.n, vq);
                 adamw_quad<!kSpec, grad_traits<GradT>::kUnscale>(
-                    gq, pq, mq, vq, a.k, acc,
+                    gq, pq, mq, vq, k, scale, acc,
                     [&]() {                    // not stored yet: still the inputs
                         return adamw_exact_quad_at<GradT, !kSpec>(g, a.master + src, a.mom + src,
-                                                                  a.var + src, idx, d.n, a.k);
+                                                                  a.var + src, idx, d.n, k, scale);
                     });
                 if (idx < d.n) {
                     store_quad(a.master + dst, idx, d.n, pq);
                     store_quad(a.mom + dst, idx, d.n, mq);
                     store_quad(a.var + dst, idx, d.n, vq);
-                    store_quad_bf16(pb, idx, d.n, pq);
+                    store_quad_lp(pb, idx, d.n, pq, fp16);
                 }
             }
             __syncwarp();
@@ -418,14 +437,19 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
     }
 
     // this warp has no more tiles to claim: a dependent kernel may be set up
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    allow_dependent_launch();
 
     if (failed) {
-        // a copy never completed: tell the host, then give the copies that are
-        // still in flight a bounded chance to land before this block's shared
-        // memory is released
+        // a copy did not complete in time: tell the host, then wait (bounded,
+        // with the full limit) for every chunk whose loads are in flight --
+        // all stages hold a produced, unconsumed chunk at this point -- so
+        // that nothing lands in this block's shared memory after it is released
         if (lane == 0) atomicExch(&ctrl->status, 1);
-        for (int s = 0; s < kStagesIn; ++s) mbar_wait_bounded(bars + s * 8, (phases >> s) & 1u);
+        for (int s = 0; s < kStagesIn; ++s) {
+            const ChunkDesc pending = descs[s];
+            if (pending.len != 0 && (pending.flags & kRagged) == 0)
+                mbar_wait_bounded(bars + s * 8, (phases >> s) & 1u, kSpinLimit);
+        }
     }
     if (lane == 0) {
         bulk_wait_all();

@@ -1,6 +1,20 @@
 // Host side of the bucketized speculative AdamW library: layout arithmetic,
 // the slot map, the per-iteration state machine, and the kernel launches.
 // The C ABI is documented in include/superoffload.h.
+//
+// How an iteration runs without a host round trip.  The slot map (which slot
+// of the state arenas holds which bucket) lives on the device.  The bucket
+// reduction's last block forms the verdict there -- norm, clip coefficient,
+// decision -- and re-points the speculated buckets if the iteration is kept;
+// one follow-up launch, enqueued right behind it, reads that verdict and does
+// whatever it entails (nothing after a plain commit, the in-place step of
+// buckets that were only checked, the re-step of every bucket after a clip,
+// the re-cast of the speculated buckets after a skip).  The host reads the same
+// verdict from mapped memory afterwards, only for its own bookkeeping (step
+// count, loss scale, counters, its mirror of the slot map), and may enqueue the
+// next iteration's speculative steps before it has done so: those launches carry
+// the constants for every way the pending iteration can have ended and pick on
+// the device.
 #include "superoffload.h"
 
 #include <cmath>
@@ -9,17 +23,45 @@
 #include <cstring>
 #include <atomic>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "so_kernels.cuh"
 #include "so_step_tma.cuh"
+#include "so_pack.cuh"
 
 using namespace so;
 
 namespace {
 
-enum Phase { kIdle = 0, kOpen = 1, kReducing = 2, kChecked = 3 };
+enum Phase { kIdle = 0, kOpen = 1, kChecked = 2 };
 enum Cover : uint8_t { kNone = 0, kCheckedOnly = 1, kSpeculated = 2 };
+
+// One iteration as the host sees it: which buckets have been covered how.
+struct IterRec {
+    std::vector<uint8_t> cover;
+    std::vector<int32_t> free_idx;      // spare slot index of a speculated bucket
+    int32_t n_covered = 0, n_speculated = 0;
+    bool have_hp = false;
+    so_hparams hp{};
+    int phase = kIdle;
+
+    void reset()
+    {
+        std::fill(cover.begin(), cover.end(), (uint8_t)kNone);
+        std::fill(free_idx.begin(), free_idx.end(), -1);
+        n_covered = n_speculated = 0;
+        have_hp = false;
+        phase = kIdle;
+    }
+};
+
+// Step count and loss-scale state.
+struct Progress {
+    int64_t t = 0;
+    double loss_scale = 1.0;
+    int64_t good_steps = 0;
+};
 
 }  // namespace
 
@@ -28,46 +70,46 @@ struct so_ctx {
     std::vector<int64_t> numel, offsets;
     int64_t total = 0, bucket_elems = 0, stride = 0, last_elems = 0, tiles_per_slot = 0;
     int32_t n_buckets = 0, undo_slots = 0, n_slots = 0, grad_dtype = SO_GRAD_BF16;
+    int32_t param_dtype = SO_PARAM_BF16;
     // ---- binding ----
     bool bound = false;
     int device = -1, num_sms = 0;
     float *master = nullptr, *mom = nullptr, *var = nullptr;
     void *grad = nullptr;
-    uint16_t *param_bf16 = nullptr;
+    uint16_t *param_lp = nullptr;
     double *d_partials = nullptr;
-    BucketStats *d_stats = nullptr;     // n_buckets results, then one record whose first
-                                        // word is the device status (0 = fine)
-    ControlBlock *d_ctrl = nullptr;     // status word + tile counters, right after d_stats
-    uint32_t launch_seq = 0;            // picks the counter pair of each pipeline launch
-    int step_variant = 0;               // 0: bulk-copy pipeline, 1: register path
-    BucketStats *h_stats = nullptr;
-    BucketStats *h_stats_dev = nullptr; // device view of h_stats when it is mapped pinned memory
-    bool h_stats_pinned = false;
+    BucketStats *d_stats = nullptr;     // n_buckets records, then the device Verdict
+    Verdict *d_verdict = nullptr;
+    ControlBlock *d_ctrl = nullptr;
     SegSum *d_seg = nullptr;            // per-bucket segment sums of the reduction
     uint32_t *d_arrivals = nullptr;     // per-bucket arrival counters of the reduction
+    int32_t *d_slot_of = nullptr, *d_free_slot = nullptr, *d_spec_idx = nullptr;
+    PackTensor *d_tensors = nullptr;    // per-tensor (pointer, flat offset, numel) for pack / unpack
+    uint64_t *h_ptr_stage = nullptr;    // pinned staging of a tensor pointer list
     int64_t segs_per_slot = 1;
+    uint32_t launch_seq = 0;            // picks the counter pair of each pipeline launch
+    int step_variant = 0;               // 0: bulk-copy pipeline, 1: register path
+    uint32_t spin_limit = kSpinLimit;   // polls a step kernel waits for a chunk (debug hook)
+    BucketStats *h_stats = nullptr;     // host copy: n_buckets records, then a Verdict
+    BucketStats *h_stats_dev = nullptr; // device view of h_stats when it is mapped pinned memory
+    bool h_stats_pinned = false;
     int32_t reduce_seq = 0;             // stamp of the latest reduction (never 0)
-    cudaStream_t reduce_stream = nullptr;   // stream the reduction in flight was launched on
     cudaEvent_t reduce_done = nullptr;  // completion of the copy-back when h_stats is not mapped
     int occ_step = 0, occ_check = 0, occ_cast = 0;
-    // ---- slot map ----
+    // ---- slot map (host mirror of the device tables) ----
     std::vector<int32_t> slot_of;       // committed slot of each bucket
-    std::vector<int32_t> spec_slot;     // slot holding the speculative result, or -1
-    std::vector<int32_t> free_slots;
-    // ---- iteration state ----
-    int phase = kIdle;
-    std::vector<uint8_t> cover;
-    int32_t n_covered = 0, n_speculated = 0;
-    bool have_hp = false;
-    so_hparams hp_iter{};
-    so_grad_stats stats{};
-    int64_t t = 0;
-    // ---- loss scaling (fp16 gradients) ----
-    double loss_scale = 1.0;            // stored gradient = loss_scale * gradient
+    std::vector<int32_t> free_slot;     // the spare slots, by index
+    // ---- iterations ----
+    IterRec cur;                        // the iteration being assembled
+    IterRec pend;                       // an iteration whose validation has been enqueued
+    bool pending = false;               //   ... and whose verdict the host has not applied yet
+    bool pend_known = false;            // its verdict was formed from host-supplied statistics
+    Verdict pend_verdict{};             //   (then this is it)
+    cudaStream_t pend_stream = nullptr;
+    so_grad_stats stats{};              // result of the last completed check
+    Progress prog;
     double ls_growth = 2.0, ls_backoff = 0.5;
     int64_t ls_interval = 0;            // clean iterations before growth; 0 = static scale
-    int64_t ls_good_steps = 0;
-    double iter_unscale = 1.0;          // 1 / loss_scale, fixed for the iteration in flight
     // ---- bookkeeping ----
     so_counters counters{};
     int32_t last_cuda_error = 0;
@@ -90,6 +132,21 @@ Geometry geometry_of(const so_ctx *c)
     g.last_elems = (uint32_t)c->last_elems;
     g.last_bucket = c->n_buckets - 1;
     return g;
+}
+
+SlotTables tables_of(const so_ctx *c)
+{
+    SlotTables t;
+    t.slot_of = c->d_slot_of;
+    t.free_slot = c->d_free_slot;
+    t.spec_idx = c->d_spec_idx;
+    t.verdict = c->d_verdict;
+    return t;
+}
+
+Verdict *host_verdict_of(const so_ctx *c)
+{
+    return reinterpret_cast<Verdict *>(c->h_stats + c->n_buckets);
 }
 
 int64_t elems_of(const so_ctx *c, int32_t b)
@@ -119,7 +176,7 @@ bool hparams_equal(const so_hparams &a, const so_hparams &b)
     return std::memcmp(&a, &b, sizeof(so_hparams)) == 0;
 }
 
-AdamScalars scalars_for(const so_hparams &hp, int64_t step_index, double scale, double unscale)
+AdamScalars scalars_for(const so_hparams &hp, int64_t step_index, double unscale)
 {
     const double bc1 = 1.0 - std::pow(hp.beta1, (double)step_index);
     const double bc2 = 1.0 - std::pow(hp.beta2, (double)step_index);
@@ -135,7 +192,6 @@ AdamScalars scalars_for(const so_hparams &hp, int64_t step_index, double scale, 
     k.lr = hp.lr;
     k.bc1 = bc1;
     k.bc2 = bc2;
-    k.scale = scale;
     k.unscale = unscale;
     return k;
 }
@@ -145,6 +201,47 @@ double clip_coef_of(double norm, double max_norm)
     if (!(max_norm > 0.0)) return 1.0;
     const double c = max_norm / (norm + 1e-6);
     return c < 1.0 ? c : 1.0;
+}
+
+// The verdict as the device forms it (make_verdict), restated for the host:
+// used where no device takes part (dry run) and where the host already holds
+// the global sum and flag.  Same three IEEE operations, same bits.
+Verdict verdict_of(double sumsq, int nonfinite, int status, double max_grad_norm, int32_t seq)
+{
+    Verdict v;
+    std::memset(&v, 0, sizeof(v));
+    v.sumsq = sumsq;
+    v.norm = std::sqrt(sumsq);
+    v.coef = clip_coef_of(v.norm, max_grad_norm);
+    v.nonfinite = nonfinite != 0;
+    v.decision = status != 0 ? kDecisionAbandon
+                 : v.nonfinite ? kDecisionSkip
+                 : v.coef < 1.0 ? kDecisionClip
+                                : kDecisionCommit;
+    v.status = status;
+    v.seq = seq;
+    return v;
+}
+
+// Step count and loss scale after an iteration that ended in `outcome`
+// (kAfterKept / kAfterSkipped / kAfterAbandoned).  Dynamic loss scaling: back
+// off after an overflow, grow after a run of clean iterations.
+Progress progress_after(const so_ctx *c, int outcome)
+{
+    Progress p = c->prog;
+    if (outcome == kAfterKept) {
+        p.t += 1;
+        if (c->ls_interval > 0 && ++p.good_steps == c->ls_interval) {
+            p.loss_scale *= c->ls_growth;
+            p.good_steps = 0;
+        }
+    } else if (outcome == kAfterSkipped) {
+        if (c->ls_interval > 0) {
+            p.loss_scale *= c->ls_backoff;
+            p.good_steps = 0;
+        }
+    }
+    return p;
 }
 
 // Persistent grid: enough blocks to fill every SM at the kernel's occupancy,
@@ -158,29 +255,48 @@ unsigned grid_for(const so_ctx *c, int64_t total_tiles, int blocks_per_sm)
     return (unsigned)want;
 }
 
-so_status after_launch(so_ctx *c)
+so_status after_launch(so_ctx *c, cudaError_t launch_error = cudaSuccess)
 {
     c->counters.kernel_launches += 1;
     if (c->dry_run) return SO_OK;
+    if (launch_error != cudaSuccess) return cuda_fail(c, launch_error);
     const cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? SO_OK : cuda_fail(c, e);
 }
 
 // ---- launches --------------------------------------------------------------
 
+// Every kernel is launched as a programmatic dependent of whatever precedes it
+// in the stream: its blocks may be set up while that kernel drains, and each of
+// them waits (griddepcontrol.wait, first thing) for its completion and memory
+// flush before reading anything.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem,
+                             cudaStream_t stream, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 // Shapes of the bulk-copy pipeline: rows per chunk, warps per block (one block
-// per SM), input stages, output stages.  The defaults came out of a sweep on
-// B200: 512-element chunks halve the per-chunk bookkeeping, two input stages of
-// 7 KB per warp keep ~140 KB of loads in flight per SM, and ten warps are the
-// most that fit in shared memory (nine with fp32 gradients).  The alternates
-// stay selectable for measurements (so_debug_set_step_variant 10 / 11).
+// per SM), input stages, output stages.  They came out of a sweep on B200:
+// 512-element chunks halve the per-chunk bookkeeping, two input stages of 7 KB
+// per warp keep ~140 KB of loads in flight per SM, and ten warps are the most
+// that fit in shared memory (nine with fp32 gradients).
 using ShapeBf16 = PipeShape<4, 10, 2, 1>;
 using ShapeFp32 = PipeShape<4, 9, 2, 1>;
-using ShapeAlt16 = PipeShape<2, 16, 3, 1>;      // bf16 gradients only
-using ShapeAlt12 = PipeShape<2, 12, 3, 1>;
 
 template <typename GradT, typename S>
-void launch_tma(so_ctx *c, const StepArgs &a, int n, bool speculative, cudaStream_t stream)
+cudaError_t launch_tma(so_ctx *c, const StepArgs &a, int n, bool speculative, cudaStream_t stream)
 {
     int64_t blocks = ((int64_t)n * a.geo.tiles_per_slot + S::kWarps - 1) / S::kWarps;
     if (blocks > c->num_sms) blocks = c->num_sms;
@@ -189,24 +305,18 @@ void launch_tma(so_ctx *c, const StepArgs &a, int n, bool speculative, cudaStrea
     const int pair = (int)(c->launch_seq++ % kCounterPairs);
     const size_t sm = TmaLayout<GradT, S>::kSmemBytes;
     if (speculative)
-        adamw_step_tma_kernel<GradT, true, S><<<grid, S::kThreads, sm, stream>>>(a, c->d_ctrl, pair);
-    else
-        adamw_step_tma_kernel<GradT, false, S><<<grid, S::kThreads, sm, stream>>>(a, c->d_ctrl, pair);
+        return launch_dependent(adamw_step_tma_kernel<GradT, true, S>, grid, S::kThreads, sm, stream,
+                                a, c->d_ctrl, pair);
+    return launch_dependent(adamw_step_tma_kernel<GradT, false, S>, grid, S::kThreads, sm, stream, a,
+                            c->d_ctrl, pair);
 }
 
-void launch_tma_variant(so_ctx *c, const StepArgs &a, int n, bool speculative, cudaStream_t stream)
+template <typename GradT>
+cudaError_t launch_registers(const StepArgs &a, unsigned grid, bool speculative, cudaStream_t stream)
 {
-    const int dt = c->grad_dtype;
-    if (c->step_variant == 10 && dt == SO_GRAD_BF16) {
-        launch_tma<uint16_t, ShapeAlt16>(c, a, n, speculative, stream);
-    } else if (c->step_variant == 11 && dt != SO_GRAD_FP16) {
-        if (dt == SO_GRAD_BF16) launch_tma<uint16_t, ShapeAlt12>(c, a, n, speculative, stream);
-        else launch_tma<float, ShapeAlt12>(c, a, n, speculative, stream);
-    } else {
-        if (dt == SO_GRAD_BF16) launch_tma<uint16_t, ShapeBf16>(c, a, n, speculative, stream);
-        else if (dt == SO_GRAD_FP16) launch_tma<half_t, ShapeBf16>(c, a, n, speculative, stream);
-        else launch_tma<float, ShapeFp32>(c, a, n, speculative, stream);
-    }
+    if (speculative)
+        return launch_dependent(adamw_step_kernel<GradT, true, 2>, grid, kThreads, 0, stream, a);
+    return launch_dependent(adamw_step_kernel<GradT, false, 2>, grid, kThreads, 0, stream, a);
 }
 
 // The bulk-copy kernels stage through more than 48 KB of shared memory.
@@ -223,10 +333,13 @@ cudaError_t allow_smem()
     return e;
 }
 
-// Step the listed buckets (src slot -> dst slot).  speculative: scale 1 and
-// tile sums written; otherwise the given scale and no sums.
+// Step the listed buckets.  speculative: scale 1, new state into the spare
+// slot, tile sums written.  Otherwise the launch follows a verdict and does
+// what the verdict on the device says (see adamw_step_kernel).
+// A speculative launch enqueued while a validation is pending carries the
+// constants for each way that validation can end.
 so_status launch_steps(so_ctx *c, const std::vector<BucketEntry> &entries, const so_hparams &hp,
-                       bool speculative, double scale, cudaStream_t stream)
+                       bool speculative, cudaStream_t stream)
 {
     const Geometry geo = geometry_of(c);
     for (size_t first = 0; first < entries.size(); first += kMaxBatch) {
@@ -236,32 +349,35 @@ so_status launch_steps(so_ctx *c, const std::vector<BucketEntry> &entries, const
         a.master = c->master;
         a.mom = c->mom;
         a.var = c->var;
-        a.param_bf16 = c->param_bf16;
+        a.param_lp = c->param_lp;
         a.partials = c->d_partials;
         a.geo = geo;
-        a.k = scalars_for(hp, c->t + 1, scale, c->iter_unscale);
-        a.n_entries = n;
-        for (int i = 0; i < n; ++i) {
-            a.e[i] = entries[first + i];
-            c->counters.elems_stepped += elems_of(c, a.e[i].bucket);
+        a.tab = tables_of(c);
+        a.pick = c->pending ? 1 : 0;
+        for (int o = 0; o < 3; ++o) {
+            const Progress p = c->pending ? progress_after(c, o) : c->prog;
+            a.k[o] = scalars_for(hp, p.t + 1, 1.0 / p.loss_scale);
         }
-        for (int i = n; i < kMaxBatch; ++i) a.e[i] = BucketEntry{0, 0, 0};
+        a.param_fp16 = c->param_dtype == SO_PARAM_FP16;
+        a.spin_limit = c->spin_limit;
+        a.n_entries = n;
+        for (int i = 0; i < n; ++i) a.e[i] = entries[first + i];
+        for (int i = n; i < kMaxBatch; ++i) a.e[i] = BucketEntry{0, -1};
+        cudaError_t e = cudaSuccess;
         if (!c->dry_run) {
             const int dt = c->grad_dtype;
             const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_step);
             if (c->step_variant != 1) {
-                launch_tma_variant(c, a, n, speculative, stream);
-            } else if (speculative) {
-                if (dt == SO_GRAD_BF16) adamw_step_kernel<uint16_t, true, 2><<<grid, kThreads, 0, stream>>>(a);
-                else if (dt == SO_GRAD_FP16) adamw_step_kernel<half_t, true, 2><<<grid, kThreads, 0, stream>>>(a);
-                else adamw_step_kernel<float, true, 2><<<grid, kThreads, 0, stream>>>(a);
+                if (dt == SO_GRAD_BF16) e = launch_tma<uint16_t, ShapeBf16>(c, a, n, speculative, stream);
+                else if (dt == SO_GRAD_FP16) e = launch_tma<half_t, ShapeBf16>(c, a, n, speculative, stream);
+                else e = launch_tma<float, ShapeFp32>(c, a, n, speculative, stream);
             } else {
-                if (dt == SO_GRAD_BF16) adamw_step_kernel<uint16_t, false, 2><<<grid, kThreads, 0, stream>>>(a);
-                else if (dt == SO_GRAD_FP16) adamw_step_kernel<half_t, false, 2><<<grid, kThreads, 0, stream>>>(a);
-                else adamw_step_kernel<float, false, 2><<<grid, kThreads, 0, stream>>>(a);
+                if (dt == SO_GRAD_BF16) e = launch_registers<uint16_t>(a, grid, speculative, stream);
+                else if (dt == SO_GRAD_FP16) e = launch_registers<half_t>(a, grid, speculative, stream);
+                else e = launch_registers<float>(a, grid, speculative, stream);
             }
         }
-        const so_status s = after_launch(c);
+        const so_status s = after_launch(c, e);
         if (s != SO_OK) return s;
     }
     return SO_OK;
@@ -275,9 +391,10 @@ so_status launch_checks(so_ctx *c, const std::vector<int32_t> &buckets, cudaStre
         CheckArgs a;
         a.grad = c->grad;
         a.partials = c->d_partials;
-        a.unscale = c->iter_unscale;
-        int exponent = 0;
-        a.unscale_is_pow2 = std::frexp(a.unscale, &exponent) == 0.5 ? 1 : 0;
+        for (int o = 0; o < 3; ++o)
+            a.unscale[o] = 1.0 / (c->pending ? progress_after(c, o) : c->prog).loss_scale;
+        a.verdict = c->d_verdict;
+        a.pick = c->pending ? 1 : 0;
         a.geo = geo;
         a.n_entries = n;
         for (int i = 0; i < n; ++i) {
@@ -285,236 +402,344 @@ so_status launch_checks(so_ctx *c, const std::vector<int32_t> &buckets, cudaStre
             c->counters.elems_checked += elems_of(c, a.bucket[i]);
         }
         for (int i = n; i < kMaxBatch; ++i) a.bucket[i] = 0;
+        cudaError_t e = cudaSuccess;
         if (!c->dry_run) {
             const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_check);
-            if (c->grad_dtype == SO_GRAD_BF16)
-                grad_check_kernel<uint16_t><<<grid, kThreads, 0, stream>>>(a);
-            else if (c->grad_dtype == SO_GRAD_FP16)
-                grad_check_kernel<half_t><<<grid, kThreads, 0, stream>>>(a);
-            else
-                grad_check_kernel<float><<<grid, kThreads, 0, stream>>>(a);
+            e = launch_grad_check(a, c->grad_dtype, grid, stream);
         }
-        const so_status s = after_launch(c);
+        const so_status s = after_launch(c, e);
         if (s != SO_OK) return s;
     }
     return SO_OK;
 }
 
-so_status launch_casts(so_ctx *c, const std::vector<BucketEntry> &entries, cudaStream_t stream)
+so_status launch_casts(so_ctx *c, const std::vector<int32_t> &buckets, cudaStream_t stream)
 {
     const Geometry geo = geometry_of(c);
-    for (size_t first = 0; first < entries.size(); first += kMaxBatch) {
-        const int n = (int)std::min<size_t>(kMaxBatch, entries.size() - first);
+    for (size_t first = 0; first < buckets.size(); first += kMaxBatch) {
+        const int n = (int)std::min<size_t>(kMaxBatch, buckets.size() - first);
         CastArgs a;
         a.master = c->master;
-        a.param_bf16 = c->param_bf16;
+        a.param_lp = c->param_lp;
         a.geo = geo;
+        a.tab = tables_of(c);
+        a.param_fp16 = c->param_dtype == SO_PARAM_FP16;
         a.n_entries = n;
         for (int i = 0; i < n; ++i) {
-            a.e[i] = entries[first + i];
-            c->counters.elems_cast += elems_of(c, a.e[i].bucket);
+            a.bucket[i] = buckets[first + i];
+            c->counters.elems_cast += elems_of(c, a.bucket[i]);
         }
-        for (int i = n; i < kMaxBatch; ++i) a.e[i] = BucketEntry{0, 0, 0};
+        for (int i = n; i < kMaxBatch; ++i) a.bucket[i] = 0;
+        cudaError_t e = cudaSuccess;
         if (!c->dry_run) {
             const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_cast);
-            cast_params_kernel<<<grid, kThreads, 0, stream>>>(a);
+            e = launch_dependent(cast_params_kernel, grid, kThreads, 0, stream, a);
         }
-        const so_status s = after_launch(c);
+        const so_status s = after_launch(c, e);
         if (s != SO_OK) return s;
     }
     return SO_OK;
 }
 
-// First half of finishing the gradient check: scan what is still uncovered and
-// launch the per-bucket reduction, whose records travel to the host on their
-// own.  Nothing here waits.
-so_status begin_check(so_ctx *c, cudaStream_t stream)
+// Scan whatever the open iteration has not covered yet.
+so_status scan_uncovered(so_ctx *c, cudaStream_t stream)
 {
     std::vector<int32_t> todo;
     for (int32_t b = 0; b < c->n_buckets; ++b)
-        if (c->cover[b] == kNone) todo.push_back(b);
-    if (!todo.empty()) {
-        const so_status s = launch_checks(c, todo, stream);
-        if (s != SO_OK) return s;
-        for (int32_t b : todo) c->cover[b] = kCheckedOnly;
-        c->n_covered = c->n_buckets;
-    }
-    c->reduce_stream = stream;
-    if (c->n_buckets > 0) {
-        if (!c->dry_run) {
-            ReduceArgs r;
-            r.partials = c->d_partials;
-            r.seg = c->d_seg;
-            r.arrivals = c->d_arrivals;
-            r.stats = c->d_stats;
-            r.host_stats = c->h_stats_dev;     // records land in host memory directly
-            r.status = &c->d_ctrl->status;
-            r.buckets_done = &c->d_ctrl->buckets_done;
-            c->reduce_seq = c->reduce_seq == 0x7FFFFFFF ? 1 : c->reduce_seq + 1;
-            r.seq = c->reduce_seq;
-            r.geo = geometry_of(c);
-            r.segs_per_slot = (uint32_t)c->segs_per_slot;
-            r.n_buckets = c->n_buckets;
-            const int64_t blocks = (int64_t)c->n_buckets * c->segs_per_slot;
-            // Programmatic dependent launch: the reduction's blocks may be set up
-            // while the step (or scan) kernel before it in the stream drains; they
-            // wait for its completion and memory flush before reading anything.
-            cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3((unsigned)blocks);
-            cfg.blockDim = dim3(kReduceThreads);
-            cfg.dynamicSmemBytes = 0;
-            cfg.stream = stream;
-            cudaLaunchAttribute attr[1];
-            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-            attr[0].val.programmaticStreamSerializationAllowed = 1;
-            cfg.attrs = attr;
-            cfg.numAttrs = 1;
-            cudaLaunchKernelEx(&cfg, bucket_reduce_kernel, r);
-        }
-        const so_status s = after_launch(c);
-        if (s != SO_OK) return s;
-        if (!c->dry_run && !c->h_stats_dev) {
-            cudaError_t e = cudaMemcpyAsync(c->h_stats, c->d_stats,
-                                            sizeof(BucketStats) * (size_t)(c->n_buckets + 1),
-                                            cudaMemcpyDeviceToHost, stream);
-            if (e == cudaSuccess && !c->reduce_done)
-                e = cudaEventCreateWithFlags(&c->reduce_done, cudaEventDisableTiming);
-            if (e == cudaSuccess) e = cudaEventRecord(c->reduce_done, stream);
-            if (e != cudaSuccess) return cuda_fail(c, e);
-        }
-    }
-    c->phase = kReducing;
+        if (c->cur.cover[b] == kNone) todo.push_back(b);
+    if (todo.empty()) return SO_OK;
+    const so_status s = launch_checks(c, todo, stream);
+    if (s != SO_OK) return s;
+    for (int32_t b : todo) c->cur.cover[b] = kCheckedOnly;
+    c->cur.n_covered = c->n_buckets;
     return SO_OK;
 }
 
-// Have the records of the reduction in flight reached the host?  Never blocks.
-bool check_arrived(so_ctx *c)
+// The per-bucket reduction; with `decide` its last block also forms the verdict
+// and re-points the slots.  Its records travel to the host on their own.
+so_status launch_reduce(so_ctx *c, double max_grad_norm, bool decide, cudaStream_t stream)
+{
+    c->reduce_seq = c->reduce_seq == 0x7FFFFFFF ? 1 : c->reduce_seq + 1;
+    if (c->n_buckets == 0) return SO_OK;
+    cudaError_t e = cudaSuccess;
+    if (!c->dry_run) {
+        ReduceArgs r;
+        r.partials = c->d_partials;
+        r.seg = c->d_seg;
+        r.arrivals = c->d_arrivals;
+        r.stats = c->d_stats;
+        r.host_stats = c->h_stats_dev;     // records land in host memory directly
+        r.status = &c->d_ctrl->status;
+        r.buckets_done = &c->d_ctrl->buckets_done;
+        r.tab = tables_of(c);
+        r.max_grad_norm = max_grad_norm;
+        r.decide = decide ? 1 : 0;
+        r.seq = c->reduce_seq;
+        r.geo = geometry_of(c);
+        r.segs_per_slot = (uint32_t)c->segs_per_slot;
+        r.n_buckets = c->n_buckets;
+        const int64_t blocks = (int64_t)c->n_buckets * c->segs_per_slot;
+        e = launch_dependent(bucket_reduce_kernel, (unsigned)blocks, kReduceThreads, 0, stream, r);
+    }
+    so_status s = after_launch(c, e);
+    if (s != SO_OK) return s;
+    if (!c->dry_run && !c->h_stats_dev) {
+        e = cudaMemcpyAsync(c->h_stats, c->d_stats,
+                            sizeof(BucketStats) * (size_t)c->n_buckets + sizeof(Verdict),
+                            cudaMemcpyDeviceToHost, stream);
+        if (e == cudaSuccess && !c->reduce_done)
+            e = cudaEventCreateWithFlags(&c->reduce_done, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventRecord(c->reduce_done, stream);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+    }
+    return SO_OK;
+}
+
+// The verdict from statistics the host holds (after so_grad_check(SO_ALL), or
+// global ones from so_set_global_grad_stats), applied on the device.
+so_status launch_verdict(so_ctx *c, const Verdict &v, double max_grad_norm, cudaStream_t stream)
+{
+    if (c->n_buckets == 0) return SO_OK;
+    cudaError_t e = cudaSuccess;
+    if (!c->dry_run) {
+        VerdictArgs a;
+        a.tab = tables_of(c);
+        a.host_verdict = nullptr;
+        a.sumsq = v.sumsq;
+        a.max_grad_norm = max_grad_norm;
+        a.nonfinite = v.nonfinite;
+        a.abandon = v.decision == kDecisionAbandon ? 1 : 0;
+        a.seq = v.seq;
+        a.n_buckets = c->n_buckets;
+        e = launch_dependent(apply_verdict_kernel, 1u, kReduceThreads, 0, stream, a);
+    }
+    return after_launch(c, e);
+}
+
+// The launch that follows a verdict: every bucket of the open iteration, with
+// the spare slot index of the speculated ones; the kernels read on the device
+// what there is to do.
+so_status launch_follow_up(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
+{
+    std::vector<BucketEntry> all;
+    all.reserve((size_t)c->n_buckets);
+    for (int32_t b = 0; b < c->n_buckets; ++b)
+        all.push_back(BucketEntry{b, c->cur.cover[b] == kSpeculated ? c->cur.free_idx[b] : -1});
+    if (all.empty()) return SO_OK;
+    return launch_steps(c, all, hp, /*speculative=*/false, stream);
+}
+
+// ---- validation ------------------------------------------------------------
+
+// Have the records of the latest reduction reached the host?  Never blocks.
+bool reduction_arrived(so_ctx *c)
 {
     if (c->dry_run || c->n_buckets == 0) return true;
     if (c->h_stats_dev) {
-        const volatile int32_t *stamp = &c->h_stats[c->n_buckets].pad;
+        const volatile int32_t *stamp = &host_verdict_of(c)->seq;
         return *stamp == c->reduce_seq;
     }
     return cudaEventQuery(c->reduce_done) == cudaSuccess;
 }
 
-void end_iteration(so_ctx *c);
-
-// A kernel of this iteration gave up waiting for one of its own copies: give
-// the iteration up.  Speculative slots go back to the free list (the committed
-// slots were never written), the bf16 copy of the speculated buckets - partly
-// overwritten - is derived again from the committed master, and the context is
-// idle again with step count and loss scale as they were.
-so_status abandon_iteration(so_ctx *c)
+// Wait (bounded spinning on the stamp, then a stream synchronisation that also
+// surfaces any error) until the latest reduction's records are in host memory.
+so_status wait_for_reduction(so_ctx *c, cudaStream_t stream)
 {
-    std::vector<BucketEntry> recast;
-    for (int32_t b = 0; b < c->n_buckets; ++b)
-        if (c->cover[b] == kSpeculated) {
-            recast.push_back(BucketEntry{b, c->slot_of[b], 0});
-            c->free_slots.push_back(c->spec_slot[b]);
+    if (c->dry_run || c->n_buckets == 0) return SO_OK;
+    cudaError_t e = cudaSuccess;
+    if (c->h_stats_dev) {
+        // The records arrive in mapped host memory; watching for the stamp
+        // that follows them is several microseconds quicker than waiting for
+        // the stream's completion to be signalled.
+        const auto t0 = std::chrono::steady_clock::now();
+        bool arrived = false;
+        for (uint32_t spins = 0;; ++spins) {
+            if (reduction_arrived(c)) { arrived = true; break; }
+            if ((spins & 0xFFFu) == 0xFFFu &&
+                std::chrono::steady_clock::now() - t0 > std::chrono::seconds(2))
+                break;
         }
-    if (!recast.empty()) launch_casts(c, recast, c->reduce_stream);   // best effort
-    c->counters.timeouts += 1;
-    end_iteration(c);
-    return SO_ERR_TIMEOUT;
-}
-
-// Second half: wait for the per-bucket records to reach the host, fold over
-// buckets in index order, derive norm and clip coefficient.
-so_status finish_check(so_ctx *c, const so_hparams &hp)
-{
-    if (c->n_buckets > 0) {
-        if (!c->dry_run) {
-            cudaError_t e = cudaSuccess;
-            if (c->h_stats_dev) {
-                // The records arrive in mapped host memory; watching for the
-                // stamp that follows them is several microseconds quicker than
-                // waiting for the stream's completion to be signalled.  Bounded:
-                // after two seconds fall back to a stream synchronisation, which
-                // also surfaces any launch or execution error.
-                const auto t0 = std::chrono::steady_clock::now();
-                bool arrived = false;
-                for (uint32_t spins = 0;; ++spins) {
-                    if (check_arrived(c)) { arrived = true; break; }
-                    if ((spins & 0xFFFu) == 0xFFFu &&
-                        std::chrono::steady_clock::now() - t0 > std::chrono::seconds(2))
-                        break;
-                }
-                std::atomic_thread_fence(std::memory_order_acquire);
-                if (!arrived) {
-                    e = cudaStreamSynchronize(c->reduce_stream);
-                    if (e != cudaSuccess) return cuda_fail(c, e);
-                    if (!check_arrived(c)) return cuda_fail(c, cudaErrorUnknown);
-                }
-            } else {
-                e = cudaStreamSynchronize(c->reduce_stream);
-                if (e != cudaSuccess) return cuda_fail(c, e);
-            }
-            int32_t device_status = c->h_stats[c->n_buckets].nonfinite;
-            if (!c->h_stats_dev)
-                std::memcpy(&device_status, &c->h_stats[c->n_buckets], sizeof(device_status));
-            if (device_status != 0) {
-                // a kernel gave up waiting for one of its own copies; its tile
-                // counters may be left mid-way, so re-arm the whole control block
-                cudaMemsetAsync(c->d_ctrl, 0, sizeof(ControlBlock), c->reduce_stream);
-                if (c->h_stats_dev) std::memset(&c->h_stats[c->n_buckets], 0, sizeof(BucketStats));
-                return abandon_iteration(c);
-            }
-        } else {
-            for (int32_t b = 0; b < c->n_buckets; ++b) c->h_stats[b] = c->injected[b];
-            if (c->injected_status != 0) {
-                c->injected_status = 0;
-                return abandon_iteration(c);
-            }
+        std::atomic_thread_fence(std::memory_order_acquire);
+        if (!arrived) {
+            e = cudaStreamSynchronize(stream);
+            if (e != cudaSuccess) return cuda_fail(c, e);
+            if (!reduction_arrived(c)) return cuda_fail(c, cudaErrorUnknown);
         }
+    } else {
+        e = cudaStreamSynchronize(stream);
+        if (e != cudaSuccess) return cuda_fail(c, e);
     }
-    double sumsq = 0.0;
-    int32_t nonfinite = 0;
-    for (int32_t b = 0; b < c->n_buckets; ++b) {
-        sumsq += c->h_stats[b].sumsq;
-        nonfinite |= (c->h_stats[b].nonfinite != 0);
-    }
-    c->stats.sumsq = sumsq;
-    c->stats.norm = std::sqrt(sumsq);
-    c->stats.clip_coef = clip_coef_of(c->stats.norm, hp.max_grad_norm);
-    c->stats.nonfinite = nonfinite;
-    c->stats.reserved = 0;
-    c->phase = kChecked;
     return SO_OK;
 }
 
-so_status finalize_check(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
+// Dry run: the records a device would have produced, from the injected values.
+// `consume_status` false leaves the injected status word for a later call.
+void inject_records(so_ctx *c, double max_grad_norm, bool decide, bool consume_status)
 {
-    if (c->phase != kReducing) {
-        const so_status s = begin_check(c, stream);
-        if (s != SO_OK) return s;
+    double sumsq = 0.0;
+    int flag = 0;
+    for (int32_t b = 0; b < c->n_buckets; ++b) {
+        c->h_stats[b] = c->injected[b];
+        sumsq += c->injected[b].sumsq;
+        flag |= c->injected[b].nonfinite != 0;
     }
-    return finish_check(c, hp);
+    Verdict v = verdict_of(sumsq, flag, c->injected_status, max_grad_norm, c->reduce_seq);
+    if (!decide) v.decision = -1;
+    if (consume_status) c->injected_status = 0;
+    *host_verdict_of(c) = v;
 }
 
-void end_iteration(so_ctx *c)
-{
-    c->iter_unscale = 1.0 / c->loss_scale;
-    std::fill(c->cover.begin(), c->cover.end(), (uint8_t)kNone);
-    std::fill(c->spec_slot.begin(), c->spec_slot.end(), -1);
-    c->n_covered = 0;
-    c->n_speculated = 0;
-    c->have_hp = false;
-    c->phase = kIdle;
-}
-
-so_status note_hparams(so_ctx *c, const so_hparams *hp)
+so_status note_hparams(const IterRec &it, const so_hparams *hp)
 {
     if (!hparams_ok(hp)) return SO_ERR_INVALID_ARG;
-    if (c->have_hp && !hparams_equal(c->hp_iter, *hp)) return SO_ERR_INVALID_ARG;
+    if (it.have_hp && !hparams_equal(it.hp, *hp)) return SO_ERR_INVALID_ARG;
     return SO_OK;
+}
+
+void make_pending(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
+{
+    if (!c->cur.have_hp) { c->cur.hp = hp; c->cur.have_hp = true; }
+    std::swap(c->cur, c->pend);
+    c->cur.reset();
+    c->pending = true;
+    c->pend_stream = stream;
+}
+
+// Enqueue the end of the open iteration: scan what is uncovered, reduce and
+// decide on the device, follow up.  The iteration becomes the pending one.
+so_status begin_validation(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
+{
+    so_status s = scan_uncovered(c, stream);
+    if (s != SO_OK) return s;
+    s = launch_reduce(c, hp.max_grad_norm, /*decide=*/true, stream);
+    if (s != SO_OK) return s;
+    s = launch_follow_up(c, hp, stream);
+    if (s != SO_OK) return s;
+    make_pending(c, hp, stream);
+    c->pend_known = false;
+    return SO_OK;
+}
+
+// The same with a verdict the host already holds (the check has completed,
+// possibly with global statistics handed in): the device applies it, nothing
+// is waited for.
+so_status begin_validation_known(so_ctx *c, const so_hparams &hp, const Verdict &v,
+                                 cudaStream_t stream)
+{
+    so_status s = launch_verdict(c, v, hp.max_grad_norm, stream);
+    if (s != SO_OK) return s;
+    s = launch_follow_up(c, hp, stream);
+    if (s != SO_OK) return s;
+    make_pending(c, hp, stream);
+    c->pend_known = true;
+    c->pend_verdict = v;
+    return SO_OK;
+}
+
+// The pending iteration's verdict, waiting for it if it is still on its way.
+so_status pending_verdict(so_ctx *c, Verdict *v, bool consume_status)
+{
+    if (c->pend_known) {
+        *v = c->pend_verdict;
+        return SO_OK;
+    }
+    if (c->dry_run) {
+        inject_records(c, c->pend.hp.max_grad_norm, /*decide=*/true, consume_status);
+    } else {
+        const so_status s = wait_for_reduction(c, c->pend_stream);
+        if (s != SO_OK) return s;
+    }
+    if (c->n_buckets > 0) std::memcpy(v, host_verdict_of(c), sizeof(*v));
+    else *v = verdict_of(0.0, 0, 0, c->pend.hp.max_grad_norm, c->reduce_seq);
+    return SO_OK;
+}
+
+// Learn the pending iteration's verdict and bring the host's books in line
+// with what the device has done.
+so_status collect_validation(so_ctx *c, so_step_result *out)
+{
+    Verdict v;
+    const so_status got = pending_verdict(c, &v, /*consume_status=*/true);
+    if (got != SO_OK) return got;
+    const IterRec &it = c->pend;
+    const int outcome = v.decision == kDecisionAbandon ? kAfterAbandoned
+                        : v.decision == kDecisionSkip  ? kAfterSkipped
+                                                       : kAfterKept;
+    const bool clip = v.decision == kDecisionClip;
+    for (int32_t b = 0; b < c->n_buckets; ++b) {
+        const int64_t n = elems_of(c, b);
+        if (it.cover[b] == kSpeculated) {
+            if (outcome == kAfterKept) {
+                std::swap(c->slot_of[b], c->free_slot[it.free_idx[b]]);
+                if (clip) c->counters.elems_stepped += n;
+            } else {
+                c->counters.elems_cast += n;     // low-precision copy derived again from the old master
+            }
+        } else if (outcome == kAfterKept) {
+            c->counters.elems_stepped += n;       // stepped in place with the validated scale
+        }
+    }
+    c->prog = progress_after(c, outcome);
+    if (outcome == kAfterKept) {
+        if (clip) c->counters.clip_resteps += 1; else c->counters.commits += 1;
+    } else if (outcome == kAfterSkipped) {
+        c->counters.skips += 1;
+    } else {
+        c->counters.timeouts += 1;
+    }
+    c->stats.sumsq = v.sumsq;
+    c->stats.norm = v.norm;
+    c->stats.clip_coef = v.coef;
+    c->stats.nonfinite = v.nonfinite;
+    c->stats.reserved = 0;
+    if (out && outcome != kAfterAbandoned) {
+        out->decision = v.decision;
+        out->buckets_speculated = it.n_speculated;
+        out->step_after = c->prog.t;
+        out->stats = c->stats;
+        out->loss_scale = c->prog.loss_scale;
+    }
+    c->pending = false;
+    c->pend_known = false;
+    c->pend.reset();
+    return outcome == kAfterAbandoned ? SO_ERR_TIMEOUT : SO_OK;
 }
 
 }  // namespace
 
+namespace so {
+
+cudaError_t launch_grad_check(const CheckArgs &a, int grad_dtype, unsigned grid, cudaStream_t stream)
+{
+    if (grad_dtype == SO_GRAD_BF16)
+        return launch_dependent(grad_check_kernel<uint16_t>, grid, kThreads, 0, stream, a);
+    if (grad_dtype == SO_GRAD_FP16)
+        return launch_dependent(grad_check_kernel<half_t>, grid, kThreads, 0, stream, a);
+    return launch_dependent(grad_check_kernel<float>, grid, kThreads, 0, stream, a);
+}
+
+cudaError_t grad_check_occupancy(int grad_dtype, int *blocks_per_sm)
+{
+    if (grad_dtype == SO_GRAD_BF16)
+        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, grad_check_kernel<uint16_t>,
+                                                             kThreads, 0);
+    if (grad_dtype == SO_GRAD_FP16)
+        return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, grad_check_kernel<half_t>,
+                                                             kThreads, 0);
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(blocks_per_sm, grad_check_kernel<float>,
+                                                         kThreads, 0);
+}
+
+}  // namespace so
+
 // ============================================================================
 // C ABI
 // ============================================================================
+
+// Scratch: tile sums | per-bucket records + verdict | control block | segment
+// sums | arrival counters | slot tables | tensor table of pack / unpack.
+static uint64_t round256(uint64_t x) { return (x + 255u) / 256u * 256u; }
 
 extern "C" {
 
@@ -556,9 +781,12 @@ so_status so_layout_init(so_ctx **out, int32_t n_tensors, const int64_t *numel,
         c->grad_dtype = grad_dtype;
         c->slot_of.resize(nb);
         for (int32_t b = 0; b < nb; ++b) c->slot_of[b] = b;
-        c->spec_slot.assign(nb, -1);
-        for (int32_t s = c->n_slots - 1; s >= nb; --s) c->free_slots.push_back(s);
-        c->cover.assign(nb, (uint8_t)kNone);
+        c->free_slot.resize(undo_slots);
+        for (int32_t j = 0; j < undo_slots; ++j) c->free_slot[j] = nb + j;
+        for (IterRec *it : {&c->cur, &c->pend}) {
+            it->cover.assign(nb, (uint8_t)kNone);
+            it->free_idx.assign(nb, -1);
+        }
         c->injected.assign(nb, BucketStats{0.0, 0, 0});
     } catch (...) {
         delete c;
@@ -589,11 +817,16 @@ so_status so_layout_get_info(const so_ctx *c, so_layout_info *info)
     info->bytes_grad = (uint64_t)c->n_buckets * (uint64_t)c->stride *
                        (c->grad_dtype == SO_GRAD_FP32 ? 4u : 2u);
     info->bytes_param_bf16 = (uint64_t)c->n_buckets * (uint64_t)c->stride * 2u;
-    const uint64_t partial_bytes = (uint64_t)c->n_buckets * (uint64_t)c->tiles_per_slot * 8u;
-    const uint64_t stats_bytes = (uint64_t)c->n_buckets * sizeof(BucketStats) + sizeof(ControlBlock);
-    const uint64_t segs = (uint64_t)((c->tiles_per_slot + kSegTiles - 1) / kSegTiles);
-    const uint64_t reduce_bytes = (uint64_t)c->n_buckets * (segs * sizeof(SegSum) + 4u);
-    info->bytes_scratch = (partial_bytes + 255u) / 256u * 256u + stats_bytes + reduce_bytes + 512u;
+    const uint64_t nb = (uint64_t)c->n_buckets;
+    uint64_t segs = (uint64_t)((c->tiles_per_slot + kSegTiles - 1) / kSegTiles);
+    if (segs < 1) segs = 1;
+    info->bytes_scratch = round256(nb * (uint64_t)c->tiles_per_slot * 8u) +
+                          round256(nb * sizeof(BucketStats) + sizeof(Verdict)) +
+                          round256(sizeof(ControlBlock)) +
+                          round256(nb * segs * sizeof(SegSum)) +
+                          round256(nb * 4u) +
+                          round256((2u * nb + (uint64_t)c->undo_slots) * 4u) +
+                          round256((uint64_t)c->numel.size() * sizeof(PackTensor)) + 256u;
     return SO_OK;
 }
 
@@ -614,7 +847,7 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
                          void *param_bf16, void *scratch)
 {
     if (!c) return SO_ERR_INVALID_ARG;
-    if (c->phase != kIdle) return SO_ERR_STATE;
+    if (c->cur.phase != kIdle || c->pending) return SO_ERR_STATE;
     void *ptrs[] = {master, m, v, grad, param_bf16, scratch};
     for (void *p : ptrs) {
         if (c->n_buckets > 0 && !p) return SO_ERR_INVALID_ARG;
@@ -635,14 +868,7 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
                 : cudaOccupancyMaxActiveBlocksPerMultiprocessor(
                       &c->occ_step, adamw_step_kernel<float, true, 2>, kThreads, 0);
         if (e != cudaSuccess) return cuda_fail(c, e);
-        e = dt == SO_GRAD_BF16
-                ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                      &c->occ_check, grad_check_kernel<uint16_t>, kThreads, 0)
-            : dt == SO_GRAD_FP16
-                ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                      &c->occ_check, grad_check_kernel<half_t>, kThreads, 0)
-                : cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-                      &c->occ_check, grad_check_kernel<float>, kThreads, 0);
+        e = grad_check_occupancy(dt, &c->occ_check);
         if (e != cudaSuccess) return cuda_fail(c, e);
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_cast, cast_params_kernel,
                                                           kThreads, 0);
@@ -650,16 +876,13 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
         e = allow_smem<uint16_t, ShapeBf16>();
         if (e == cudaSuccess) e = allow_smem<half_t, ShapeBf16>();
         if (e == cudaSuccess) e = allow_smem<float, ShapeFp32>();
-        if (e == cudaSuccess) e = allow_smem<uint16_t, ShapeAlt16>();
-        if (e == cudaSuccess) e = allow_smem<uint16_t, ShapeAlt12>();
-        if (e == cudaSuccess) e = allow_smem<float, ShapeAlt12>();
         if (e != cudaSuccess) return cuda_fail(c, e);
     } else {
         c->num_sms = 148;
         c->occ_step = c->occ_check = c->occ_cast = 2;
     }
     if (!c->h_stats) {
-        const size_t bytes = sizeof(BucketStats) * (size_t)(c->n_buckets + 1);
+        const size_t bytes = sizeof(BucketStats) * (size_t)c->n_buckets + sizeof(Verdict);
         if (!c->dry_run && cudaHostAlloc(reinterpret_cast<void **>(&c->h_stats), bytes,
                                          cudaHostAllocMapped) == cudaSuccess) {
             c->h_stats_pinned = true;
@@ -671,7 +894,7 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
                 cudaGetLastError();                   // fall back to an explicit copy
         } else {
             if (!c->dry_run) cudaGetLastError();      // clear the failed pinned allocation
-            c->h_stats = static_cast<BucketStats *>(std::malloc(bytes));
+            c->h_stats = static_cast<BucketStats *>(std::calloc(1, bytes));
             if (!c->h_stats) return SO_ERR_NOMEM;
         }
     }
@@ -679,25 +902,60 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
     c->mom = static_cast<float *>(m);
     c->var = static_cast<float *>(v);
     c->grad = grad;
-    c->param_bf16 = static_cast<uint16_t *>(param_bf16);
-    c->d_partials = static_cast<double *>(scratch);
-    const uint64_t partial_bytes = (uint64_t)c->n_buckets * (uint64_t)c->tiles_per_slot * 8u;
-    c->d_stats = reinterpret_cast<BucketStats *>(static_cast<char *>(scratch) +
-                                                 (partial_bytes + 255u) / 256u * 256u);
-    c->d_ctrl = reinterpret_cast<ControlBlock *>(c->d_stats + c->n_buckets);
+    c->param_lp = static_cast<uint16_t *>(param_bf16);
+    // carve scratch up (the same arithmetic as so_layout_get_info)
+    const uint64_t nb = (uint64_t)c->n_buckets;
     c->segs_per_slot = (c->tiles_per_slot + kSegTiles - 1) / kSegTiles;
     if (c->segs_per_slot < 1) c->segs_per_slot = 1;
-    c->d_seg = reinterpret_cast<SegSum *>(c->d_ctrl + 1);
-    c->d_arrivals = reinterpret_cast<uint32_t *>(c->d_seg + (int64_t)c->n_buckets * c->segs_per_slot);
-    if (!c->dry_run) {
-        // the control block and the arrival counters must start at zero; the
-        // rest of scratch is written before it is read
+    char *at = static_cast<char *>(scratch);
+    c->d_partials = reinterpret_cast<double *>(at);
+    at += round256(nb * (uint64_t)c->tiles_per_slot * 8u);
+    c->d_stats = reinterpret_cast<BucketStats *>(at);
+    c->d_verdict = reinterpret_cast<Verdict *>(c->d_stats + nb);
+    at += round256(nb * sizeof(BucketStats) + sizeof(Verdict));
+    c->d_ctrl = reinterpret_cast<ControlBlock *>(at);
+    at += round256(sizeof(ControlBlock));
+    c->d_seg = reinterpret_cast<SegSum *>(at);
+    at += round256(nb * (uint64_t)c->segs_per_slot * sizeof(SegSum));
+    c->d_arrivals = reinterpret_cast<uint32_t *>(at);
+    at += round256(nb * 4u);
+    c->d_slot_of = reinterpret_cast<int32_t *>(at);
+    c->d_spec_idx = c->d_slot_of + nb;
+    c->d_free_slot = c->d_spec_idx + nb;
+    at += round256((2u * nb + (uint64_t)c->undo_slots) * 4u);
+    c->d_tensors = reinterpret_cast<PackTensor *>(at);
+    if (!c->dry_run && c->n_buckets > 0) {
+        // the control block, the verdict and the arrival counters start at zero,
+        // the slot tables at the host's current map; the rest of scratch is
+        // written before it is read.  (An empty model binds nothing and touches
+        // no device memory.)
         cudaError_t e = cudaMemset(c->d_ctrl, 0, sizeof(ControlBlock));
-        if (e == cudaSuccess && c->n_buckets > 0)
-            e = cudaMemset(c->d_arrivals, 0, sizeof(uint32_t) * (size_t)c->n_buckets);
+        if (e == cudaSuccess) e = cudaMemset(c->d_verdict, 0, sizeof(Verdict));
+        if (e == cudaSuccess) e = cudaMemset(c->d_arrivals, 0, sizeof(uint32_t) * nb);
+        if (e == cudaSuccess) e = cudaMemset(c->d_spec_idx, 0xFF, sizeof(int32_t) * nb);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(c->d_slot_of, c->slot_of.data(), sizeof(int32_t) * nb, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess && c->undo_slots > 0)
+            e = cudaMemcpy(c->d_free_slot, c->free_slot.data(), sizeof(int32_t) * (size_t)c->undo_slots,
+                           cudaMemcpyHostToDevice);
+        if (e == cudaSuccess && !c->numel.empty()) {
+            std::vector<PackTensor> table(c->numel.size());
+            for (size_t i = 0; i < table.size(); ++i)
+                table[i] = PackTensor{nullptr, c->offsets[i], c->numel[i]};
+            e = cudaMemcpy(c->d_tensors, table.data(), sizeof(PackTensor) * table.size(),
+                           cudaMemcpyHostToDevice);
+        }
         if (e != cudaSuccess) return cuda_fail(c, e);
     }
     c->bound = true;
+    return SO_OK;
+}
+
+so_status so_param_dtype_config(so_ctx *c, int32_t param_dtype)
+{
+    if (!c || (param_dtype != SO_PARAM_BF16 && param_dtype != SO_PARAM_FP16)) return SO_ERR_INVALID_ARG;
+    if (c->cur.phase != kIdle || c->pending) return SO_ERR_STATE;
+    c->param_dtype = param_dtype;
     return SO_OK;
 }
 
@@ -706,25 +964,63 @@ so_status so_grad_check(so_ctx *c, const so_hparams *hp, int32_t bucket, void *s
 {
     if (!c) return SO_ERR_INVALID_ARG;
     if (!c->bound) return SO_ERR_STATE;
-    if (c->phase == kChecked) return SO_ERR_STATE;
-    if (c->phase == kReducing && bucket != SO_ALL) return SO_ERR_STATE;
+    if (c->cur.phase == kChecked) return SO_ERR_STATE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (bucket == SO_ALL) {
-        so_status s = note_hparams(c, hp);
+        if (c->pending) {
+            // a validation has been enqueued: its statistics, as soon as they are in
+            if (c->cur.phase != kIdle) return SO_ERR_STATE;
+            so_status s = note_hparams(c->pend, hp);
+            if (s != SO_OK) return s;
+            Verdict v;
+            s = pending_verdict(c, &v, /*consume_status=*/false);
+            if (s != SO_OK) return s;
+            if (out) {
+                out->sumsq = v.sumsq;
+                out->norm = v.norm;
+                out->clip_coef = v.coef;
+                out->nonfinite = v.nonfinite;
+                out->reserved = 0;
+            }
+            return SO_OK;
+        }
+        so_status s = note_hparams(c->cur, hp);
         if (s != SO_OK) return s;
-        s = finalize_check(c, *hp, st);
+        s = scan_uncovered(c, st);
         if (s != SO_OK) return s;
-        if (!c->have_hp) { c->hp_iter = *hp; c->have_hp = true; }
+        s = launch_reduce(c, hp->max_grad_norm, /*decide=*/false, st);
+        if (s != SO_OK) return s;
+        if (c->dry_run) inject_records(c, hp->max_grad_norm, false, true);
+        else if ((s = wait_for_reduction(c, st)) != SO_OK) return s;
+        Verdict v;
+        if (c->n_buckets > 0) std::memcpy(&v, host_verdict_of(c), sizeof(v));
+        else v = verdict_of(0.0, 0, 0, hp->max_grad_norm, 0);
+        if (!c->cur.have_hp) { c->cur.hp = *hp; c->cur.have_hp = true; }
+        if (v.status != 0) {
+            // a kernel gave up waiting for one of its own copies: give the
+            // iteration up (the device drops the speculative slots and derives
+            // the low-precision copy of those buckets again)
+            const Verdict gave_up = verdict_of(v.sumsq, v.nonfinite, v.status, hp->max_grad_norm, 0);
+            s = begin_validation_known(c, *hp, gave_up, st);
+            if (s != SO_OK) return s;
+            return collect_validation(c, nullptr);
+        }
+        c->stats.sumsq = v.sumsq;
+        c->stats.norm = std::sqrt(v.sumsq);
+        c->stats.clip_coef = clip_coef_of(c->stats.norm, hp->max_grad_norm);
+        c->stats.nonfinite = v.nonfinite;
+        c->stats.reserved = 0;
+        c->cur.phase = kChecked;
         if (out) *out = c->stats;
         return SO_OK;
     }
     if (bucket < 0 || bucket >= c->n_buckets) return SO_ERR_INVALID_ARG;
-    if (c->cover[bucket] != kNone) return SO_ERR_STATE;
+    if (c->cur.cover[bucket] != kNone) return SO_ERR_STATE;
     const so_status s = launch_checks(c, std::vector<int32_t>{bucket}, st);
     if (s != SO_OK) return s;
-    c->cover[bucket] = kCheckedOnly;
-    c->n_covered += 1;
-    c->phase = kOpen;
+    c->cur.cover[bucket] = kCheckedOnly;
+    c->cur.n_covered += 1;
+    c->cur.phase = kOpen;
     return SO_OK;
 }
 
@@ -732,36 +1028,34 @@ so_status so_adam_step_speculative(so_ctx *c, const so_hparams *hp, int32_t buck
 {
     if (!c) return SO_ERR_INVALID_ARG;
     if (!c->bound) return SO_ERR_STATE;
-    if (c->phase == kChecked || c->phase == kReducing) return SO_ERR_STATE;
-    so_status s = note_hparams(c, hp);
+    if (c->cur.phase == kChecked) return SO_ERR_STATE;
+    so_status s = note_hparams(c->cur, hp);
     if (s != SO_OK) return s;
     if (bucket != SO_ALL && (bucket < 0 || bucket >= c->n_buckets)) return SO_ERR_INVALID_ARG;
 
+    IterRec &it = c->cur;
     std::vector<BucketEntry> entries;
+    int32_t next_free = it.n_speculated;
     if (bucket == SO_ALL) {
-        size_t free_left = c->free_slots.size();
-        for (int32_t b = 0; b < c->n_buckets && free_left > 0; ++b)
-            if (c->cover[b] == kNone) {
-                entries.push_back(BucketEntry{b, c->slot_of[b], c->free_slots[free_left - 1]});
-                --free_left;
-            }
+        for (int32_t b = 0; b < c->n_buckets && next_free < c->undo_slots; ++b)
+            if (it.cover[b] == kNone) entries.push_back(BucketEntry{b, next_free++});
     } else {
-        if (c->cover[bucket] != kNone) return SO_ERR_STATE;
-        if (c->free_slots.empty()) return SO_ERR_UNDO_EXHAUSTED;
-        entries.push_back(BucketEntry{bucket, c->slot_of[bucket], c->free_slots.back()});
+        if (it.cover[bucket] != kNone) return SO_ERR_STATE;
+        if (next_free >= c->undo_slots) return SO_ERR_UNDO_EXHAUSTED;
+        entries.push_back(BucketEntry{bucket, next_free});
     }
     if (entries.empty()) return SO_OK;
-    s = launch_steps(c, entries, *hp, /*speculative=*/true, 1.0, static_cast<cudaStream_t>(stream));
+    s = launch_steps(c, entries, *hp, /*speculative=*/true, static_cast<cudaStream_t>(stream));
     if (s != SO_OK) return s;
     for (const BucketEntry &e : entries) {
-        c->free_slots.pop_back();
-        c->spec_slot[e.bucket] = e.dst_slot;
-        c->cover[e.bucket] = kSpeculated;
+        it.free_idx[e.bucket] = e.free_idx;
+        it.cover[e.bucket] = kSpeculated;
+        c->counters.elems_stepped += elems_of(c, e.bucket);
     }
-    c->n_covered += (int32_t)entries.size();
-    c->n_speculated += (int32_t)entries.size();
-    if (!c->have_hp) { c->hp_iter = *hp; c->have_hp = true; }
-    c->phase = kOpen;
+    it.n_covered += (int32_t)entries.size();
+    it.n_speculated += (int32_t)entries.size();
+    if (!it.have_hp) { it.hp = *hp; it.have_hp = true; }
+    it.phase = kOpen;
     return SO_OK;
 }
 
@@ -770,130 +1064,73 @@ so_status so_validate_commit_or_rollback(so_ctx *c, const so_hparams *hp, void *
 {
     if (!c) return SO_ERR_INVALID_ARG;
     if (!c->bound) return SO_ERR_STATE;
-    so_status s = note_hparams(c, hp);
-    if (s != SO_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (c->phase != kChecked) {
-        s = finalize_check(c, *hp, st);
+    if (c->pending) {
+        // a validation enqueued earlier (so_validate_begin): collect it; the
+        // iteration that may have been opened since is not touched
+        const so_status s = note_hparams(c->pend, hp);
         if (s != SO_OK) return s;
+        return collect_validation(c, out);
     }
-    // the coefficient always follows the hyper-parameters given here
-    c->stats.clip_coef = clip_coef_of(c->stats.norm, hp->max_grad_norm);
-
-    int32_t decision;
-    if (c->stats.nonfinite) decision = SO_DECISION_SKIP;
-    else if (c->stats.clip_coef < 1.0) decision = SO_DECISION_CLIP_RESTEP;
-    else decision = SO_DECISION_COMMIT;
-
-    const int32_t n_spec = c->n_speculated;
-    if (decision == SO_DECISION_SKIP) {
-        // drop the speculative slots; the bf16 copy of those buckets was
-        // overwritten by the speculative step and is re-derived from the old master
-        std::vector<BucketEntry> recast;
-        for (int32_t b = 0; b < c->n_buckets; ++b)
-            if (c->cover[b] == kSpeculated) recast.push_back(BucketEntry{b, c->slot_of[b], 0});
-        if (!recast.empty()) {
-            s = launch_casts(c, recast, st);
-            if (s != SO_OK) return s;
-        }
-        for (int32_t b = 0; b < c->n_buckets; ++b)
-            if (c->cover[b] == kSpeculated) c->free_slots.push_back(c->spec_slot[b]);
-        c->counters.skips += 1;
+    so_status s = note_hparams(c->cur, hp);
+    if (s != SO_OK) return s;
+    if (c->cur.phase == kChecked) {
+        // the check has completed on the host (possibly with global statistics)
+        const Verdict v = verdict_of(c->stats.sumsq, c->stats.nonfinite, 0, hp->max_grad_norm, 0);
+        s = begin_validation_known(c, *hp, v, st);
     } else {
-        const bool clip = decision == SO_DECISION_CLIP_RESTEP;
-        // buckets to (re-)step with the validated scale: all of them after a
-        // clip, only the never-speculated ones after a commit
-        std::vector<BucketEntry> work;
-        for (int32_t b = 0; b < c->n_buckets; ++b) {
-            if (c->cover[b] == kSpeculated) {
-                if (clip) work.push_back(BucketEntry{b, c->slot_of[b], c->spec_slot[b]});
-            } else {
-                work.push_back(BucketEntry{b, c->slot_of[b], c->slot_of[b]});
-            }
-        }
-        if (!work.empty()) {
-            s = launch_steps(c, work, *hp, /*speculative=*/false,
-                             clip ? c->stats.clip_coef : 1.0, st);
-            if (s != SO_OK) return s;
-        }
-        for (int32_t b = 0; b < c->n_buckets; ++b)
-            if (c->cover[b] == kSpeculated) {
-                c->free_slots.push_back(c->slot_of[b]);
-                c->slot_of[b] = c->spec_slot[b];
-            }
-        c->t += 1;
-        if (clip) c->counters.clip_resteps += 1; else c->counters.commits += 1;
+        s = begin_validation(c, *hp, st);
     }
-    // dynamic loss scaling: back off after an overflow, grow after a run of
-    // clean iterations (takes effect from the next iteration on)
-    if (c->ls_interval > 0) {
-        if (decision == SO_DECISION_SKIP) {
-            c->loss_scale *= c->ls_backoff;
-            c->ls_good_steps = 0;
-        } else if (++c->ls_good_steps == c->ls_interval) {
-            c->loss_scale *= c->ls_growth;
-            c->ls_good_steps = 0;
-        }
-    }
-    if (out) {
-        out->decision = decision;
-        out->buckets_speculated = n_spec;
-        out->step_after = c->t;
-        out->stats = c->stats;
-        out->loss_scale = c->loss_scale;
-    }
-    end_iteration(c);
-    return SO_OK;
+    if (s != SO_OK) return s;
+    return collect_validation(c, out);
 }
 
 so_status so_validate_begin(so_ctx *c, const so_hparams *hp, void *stream)
 {
     if (!c) return SO_ERR_INVALID_ARG;
     if (!c->bound) return SO_ERR_STATE;
-    if (c->phase == kChecked || c->phase == kReducing) return SO_ERR_STATE;
-    so_status s = note_hparams(c, hp);
+    if (c->pending || c->cur.phase == kChecked) return SO_ERR_STATE;
+    const so_status s = note_hparams(c->cur, hp);
     if (s != SO_OK) return s;
-    s = begin_check(c, static_cast<cudaStream_t>(stream));
-    if (s != SO_OK) return s;
-    if (!c->have_hp) { c->hp_iter = *hp; c->have_hp = true; }
-    return SO_OK;
+    return begin_validation(c, *hp, static_cast<cudaStream_t>(stream));
 }
 
 so_status so_set_global_grad_stats(so_ctx *c, double global_sumsq, int32_t global_nonfinite)
 {
     if (!c) return SO_ERR_INVALID_ARG;
-    if (c->phase != kChecked) return SO_ERR_STATE;
+    if (c->cur.phase != kChecked) return SO_ERR_STATE;
     if (std::isnan(global_sumsq) ? false : global_sumsq < 0.0) return SO_ERR_INVALID_ARG;
     c->stats.sumsq = global_sumsq;
     c->stats.norm = std::sqrt(global_sumsq);
     c->stats.nonfinite = (global_nonfinite != 0 || !std::isfinite(global_sumsq)) ? 1 : 0;
-    c->stats.clip_coef = clip_coef_of(c->stats.norm, c->hp_iter.max_grad_norm);
+    c->stats.clip_coef = clip_coef_of(c->stats.norm, c->cur.hp.max_grad_norm);
     return SO_OK;
 }
 
 so_status so_validate_poll(so_ctx *c, int32_t *ready)
 {
     if (!c || !ready) return SO_ERR_INVALID_ARG;
-    if (c->phase == kChecked) { *ready = 1; return SO_OK; }
-    if (c->phase != kReducing) return SO_ERR_STATE;
-    *ready = check_arrived(c) ? 1 : 0;
-    return SO_OK;
+    if (c->pending) {
+        *ready = (c->pend_known || reduction_arrived(c)) ? 1 : 0;
+        return SO_OK;
+    }
+    if (c->cur.phase == kChecked) { *ready = 1; return SO_OK; }
+    return SO_ERR_STATE;
 }
 
 so_status so_cast_params(so_ctx *c, int32_t bucket, void *stream)
 {
     if (!c) return SO_ERR_INVALID_ARG;
-    if (!c->bound || c->phase != kIdle) return SO_ERR_STATE;
+    if (!c->bound || c->cur.phase != kIdle || c->pending) return SO_ERR_STATE;
     if (bucket != SO_ALL && (bucket < 0 || bucket >= c->n_buckets)) return SO_ERR_INVALID_ARG;
-    std::vector<BucketEntry> entries;
+    std::vector<int32_t> buckets;
     if (bucket == SO_ALL) {
-        for (int32_t b = 0; b < c->n_buckets; ++b)
-            entries.push_back(BucketEntry{b, c->slot_of[b], 0});
+        for (int32_t b = 0; b < c->n_buckets; ++b) buckets.push_back(b);
     } else {
-        entries.push_back(BucketEntry{bucket, c->slot_of[bucket], 0});
+        buckets.push_back(bucket);
     }
-    if (entries.empty()) return SO_OK;
-    return launch_casts(c, entries, static_cast<cudaStream_t>(stream));
+    if (buckets.empty()) return SO_OK;
+    return launch_casts(c, buckets, static_cast<cudaStream_t>(stream));
 }
 
 static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void *host_grad,
@@ -903,7 +1140,7 @@ so_status so_iteration_host(so_ctx *c, const so_hparams *hp, const void *host_gr
                             void *host_param_bf16, void *stream, so_step_result *out)
 {
     if (!c) return SO_ERR_INVALID_ARG;
-    if (!c->bound || c->phase != kIdle) return SO_ERR_STATE;
+    if (!c->bound || c->cur.phase != kIdle || c->pending) return SO_ERR_STATE;
     if (!hparams_ok(hp) || (c->n_buckets > 0 && !host_grad)) return SO_ERR_INVALID_ARG;
     if (c->dry_run) return SO_ERR_UNSUPPORTED;
     const so_status s = iteration_host_body(c, hp, host_grad, host_param_bf16, stream, out);
@@ -955,7 +1192,7 @@ static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void
         if ((e = cudaStreamWaitEvent(main, c->events[2 * b], 0)) != cudaSuccess) return cuda_fail(c, e);
         so_status s;
         bool speculated = false;
-        if (!c->free_slots.empty()) {
+        if (c->cur.n_speculated < c->undo_slots) {
             s = so_adam_step_speculative(c, hp, b, stream);
             speculated = true;
         } else {
@@ -966,12 +1203,12 @@ static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void
             if ((e = cudaEventRecord(c->events[2 * b + 1], main)) != cudaSuccess) return cuda_fail(c, e);
             if ((e = cudaStreamWaitEvent(c->copy_out, c->events[2 * b + 1], 0)) != cudaSuccess) return cuda_fail(c, e);
             e = cudaMemcpyAsync(hp_out + (size_t)b * (size_t)c->bucket_elems * 2,
-                                c->param_bf16 + (size_t)b * (size_t)c->stride, n * 2,
+                                c->param_lp + (size_t)b * (size_t)c->stride, n * 2,
                                 cudaMemcpyDeviceToHost, c->copy_out);
             if (e != cudaSuccess) return cuda_fail(c, e);
         }
     }
-    std::vector<uint8_t> was_speculated(c->cover.begin(), c->cover.end());
+    std::vector<uint8_t> was_speculated(c->cur.cover.begin(), c->cur.cover.end());
     so_step_result res;
     so_status s = so_validate_commit_or_rollback(c, hp, stream, &res);
     if (s != SO_OK) return s;
@@ -985,7 +1222,7 @@ static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void
             if (!sent && res.decision == SO_DECISION_SKIP) continue;   // never changed
             const size_t n = (size_t)elems_of(c, b);
             e = cudaMemcpyAsync(hp_out + (size_t)b * (size_t)c->bucket_elems * 2,
-                                c->param_bf16 + (size_t)b * (size_t)c->stride, n * 2,
+                                c->param_lp + (size_t)b * (size_t)c->stride, n * 2,
                                 cudaMemcpyDeviceToHost, c->copy_out);
             if (e != cudaSuccess) return cuda_fail(c, e);
         }
@@ -1002,27 +1239,28 @@ so_status so_loss_scale_config(so_ctx *c, double init_scale, double growth, doub
                                int64_t interval)
 {
     if (!c) return SO_ERR_INVALID_ARG;
-    if (c->phase != kIdle) return SO_ERR_STATE;
+    if (c->cur.phase != kIdle || c->pending) return SO_ERR_STATE;
     if (c->grad_dtype != SO_GRAD_FP16) return SO_ERR_UNSUPPORTED;
     if (!(init_scale > 0.0) || !std::isfinite(init_scale) || interval < 0) return SO_ERR_INVALID_ARG;
     if (interval > 0 && (!(growth >= 1.0) || !std::isfinite(growth) || !(backoff > 0.0) ||
                          !(backoff <= 1.0)))
         return SO_ERR_INVALID_ARG;
-    c->loss_scale = init_scale;
+    c->prog.loss_scale = init_scale;
     c->ls_growth = growth;
     c->ls_backoff = backoff;
     c->ls_interval = interval;
-    c->ls_good_steps = 0;
-    c->iter_unscale = 1.0 / init_scale;
+    c->prog.good_steps = 0;
     return SO_OK;
 }
 
 so_status so_get_loss_scale(const so_ctx *c, double *scale)
 {
     if (!c || !scale) return SO_ERR_INVALID_ARG;
-    *scale = c->loss_scale;
+    *scale = c->prog.loss_scale;
     return SO_OK;
 }
+
+}  // extern "C"
 
 namespace {
 
@@ -1048,12 +1286,81 @@ so_status copy_state(so_ctx *c, void *flat[3], bool to_flat, cudaStream_t stream
     return SO_OK;
 }
 
+// One launch that moves every tensor of the list between its own buffer and
+// the bucket arena (see so_pack.cuh).  The pointer list goes through a pinned
+// staging buffer so that the upload is asynchronous.
+so_status pack_or_unpack(so_ctx *c, const void *const *tensor_ptrs, bool pack, cudaStream_t stream)
+{
+    const size_t nt = c->numel.size();
+    if (nt == 0 || c->total == 0) return SO_OK;
+    if (!tensor_ptrs) return SO_ERR_INVALID_ARG;
+    const size_t esz = pack ? (c->grad_dtype == SO_GRAD_FP32 ? 4u : 2u) : 2u;
+    for (size_t i = 0; i < nt; ++i) {
+        if (c->numel[i] > 0 && !tensor_ptrs[i]) return SO_ERR_INVALID_ARG;
+        if ((reinterpret_cast<uintptr_t>(tensor_ptrs[i]) & (esz - 1)) != 0) return SO_ERR_INVALID_ARG;
+    }
+    cudaError_t e = cudaSuccess;
+    if (!c->dry_run) {
+        if (!c->h_ptr_stage) {
+            e = cudaHostAlloc(reinterpret_cast<void **>(&c->h_ptr_stage), nt * sizeof(uint64_t),
+                              cudaHostAllocDefault);
+            if (e != cudaSuccess) return cuda_fail(c, e);
+        } else {
+            // the staging buffer may still feed the previous call's upload
+            e = cudaStreamSynchronize(stream);
+            if (e != cudaSuccess) return cuda_fail(c, e);
+        }
+        for (size_t i = 0; i < nt; ++i) c->h_ptr_stage[i] = reinterpret_cast<uint64_t>(tensor_ptrs[i]);
+        // the pointer is the first member of each table entry
+        e = cudaMemcpy2DAsync(c->d_tensors, sizeof(PackTensor), c->h_ptr_stage, sizeof(uint64_t),
+                              sizeof(uint64_t), nt, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        PackArgs a;
+        a.tensors = c->d_tensors;
+        a.n_tensors = (int32_t)nt;
+        a.arena = pack ? c->grad : static_cast<void *>(c->param_lp);
+        a.total = c->total;
+        a.bucket_elems = c->bucket_elems;
+        a.stride = c->stride;
+        const int64_t tiles = (c->total + kPackTileElems - 1) / kPackTileElems;
+        int64_t blocks = (tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
+        const int64_t cap = (int64_t)c->num_sms * 8;
+        if (blocks > cap) blocks = cap;
+        const unsigned grid = (unsigned)blocks;
+        if (esz == 4) {
+            if (pack) e = launch_dependent(pack_kernel<uint32_t, true>, grid, kThreads, 0, stream, a);
+            else e = launch_dependent(pack_kernel<uint32_t, false>, grid, kThreads, 0, stream, a);
+        } else {
+            if (pack) e = launch_dependent(pack_kernel<uint16_t, true>, grid, kThreads, 0, stream, a);
+            else e = launch_dependent(pack_kernel<uint16_t, false>, grid, kThreads, 0, stream, a);
+        }
+    }
+    return after_launch(c, e);
+}
+
 }  // namespace
+
+extern "C" {
+
+so_status so_layout_pack_grads(so_ctx *c, const void *const *tensor_grads, void *stream)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (!c->bound) return SO_ERR_STATE;
+    if (c->cur.phase != kIdle) return SO_ERR_STATE;         // its gradients are in use
+    return pack_or_unpack(c, tensor_grads, /*pack=*/true, static_cast<cudaStream_t>(stream));
+}
+
+so_status so_layout_unpack_params(so_ctx *c, void *const *tensor_params, void *stream)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (!c->bound) return SO_ERR_STATE;
+    return pack_or_unpack(c, tensor_params, /*pack=*/false, static_cast<cudaStream_t>(stream));
+}
 
 so_status so_state_export(so_ctx *c, void *master, void *m, void *v, void *stream)
 {
     if (!c) return SO_ERR_INVALID_ARG;
-    if (!c->bound || c->phase != kIdle) return SO_ERR_STATE;
+    if (!c->bound || c->cur.phase != kIdle || c->pending) return SO_ERR_STATE;
     if (c->dry_run) return SO_ERR_UNSUPPORTED;
     void *flat[3] = {master, m, v};
     return copy_state(c, flat, /*to_flat=*/true, static_cast<cudaStream_t>(stream));
@@ -1063,7 +1370,7 @@ so_status so_state_import(so_ctx *c, const void *master, const void *m, const vo
                           void *stream)
 {
     if (!c) return SO_ERR_INVALID_ARG;
-    if (!c->bound || c->phase != kIdle) return SO_ERR_STATE;
+    if (!c->bound || c->cur.phase != kIdle || c->pending) return SO_ERR_STATE;
     if (c->dry_run) return SO_ERR_UNSUPPORTED;
     void *flat[3] = {const_cast<void *>(master), const_cast<void *>(m), const_cast<void *>(v)};
     return copy_state(c, flat, /*to_flat=*/false, static_cast<cudaStream_t>(stream));
@@ -1079,22 +1386,22 @@ so_status so_bucket_slot(const so_ctx *c, int32_t bucket, int32_t *slot)
 so_status so_get_step(const so_ctx *c, int64_t *t)
 {
     if (!c || !t) return SO_ERR_INVALID_ARG;
-    *t = c->t;
+    *t = c->prog.t;
     return SO_OK;
 }
 
 so_status so_set_step(so_ctx *c, int64_t t)
 {
     if (!c || t < 0) return SO_ERR_INVALID_ARG;
-    if (c->phase != kIdle) return SO_ERR_STATE;
-    c->t = t;
+    if (c->cur.phase != kIdle || c->pending) return SO_ERR_STATE;
+    c->prog.t = t;
     return SO_OK;
 }
 
 so_status so_pending_buckets(const so_ctx *c, int32_t *n)
 {
     if (!c || !n) return SO_ERR_INVALID_ARG;
-    *n = c->n_buckets - c->n_covered;
+    *n = c->n_buckets - c->cur.n_covered;
     return SO_OK;
 }
 
@@ -1130,6 +1437,7 @@ void so_destroy(so_ctx *c)
     if (c->reduce_done) cudaEventDestroy(c->reduce_done);
     if (c->copy_in) cudaStreamDestroy(c->copy_in);
     if (c->copy_out) cudaStreamDestroy(c->copy_out);
+    if (c->h_ptr_stage) cudaFreeHost(c->h_ptr_stage);
     if (c->h_stats) {
         if (c->h_stats_pinned) cudaFreeHost(c->h_stats);
         else std::free(c->h_stats);
@@ -1147,9 +1455,16 @@ so_status so_debug_set_dry_run(so_ctx *c, int32_t on)
 
 so_status so_debug_set_step_variant(so_ctx *c, int32_t variant)
 {
-    if (!c || (variant != 0 && variant != 1 && variant != 10 && variant != 11)) return SO_ERR_INVALID_ARG;
-    if (c->phase != kIdle) return SO_ERR_STATE;
+    if (!c || (variant != 0 && variant != 1)) return SO_ERR_INVALID_ARG;
+    if (c->cur.phase != kIdle || c->pending) return SO_ERR_STATE;
     c->step_variant = variant;
+    return SO_OK;
+}
+
+so_status so_debug_set_spin_limit(so_ctx *c, int64_t polls)
+{
+    if (!c || polls < 0 || polls > (int64_t)kSpinLimit) return SO_ERR_INVALID_ARG;
+    c->spin_limit = (uint32_t)polls;
     return SO_OK;
 }
 

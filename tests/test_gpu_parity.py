@@ -65,17 +65,6 @@ def test_register_variant_of_the_step_lockstep(name):
     assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
 
 
-@pytest.mark.parametrize("variant,dtype", [(10, "bf16"), (11, "bf16"), (11, "fp32")])
-def test_alternate_pipeline_shapes_lockstep(variant, dtype):
-    """The selectable shapes of the bulk-copy pipeline (256-element chunks,
-    16 or 12 warps, three input stages) against the oracle, ragged buckets."""
-    w = W.tiny_ragged()
-    w.grad_dtype = dtype
-    rep, _ = run_lockstep(w, steps=8, undo_slots=3, step_variant=variant)
-    assert rep.decisions[6] == S
-    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
-
-
 def test_tiny_without_clipping_commits():
     w = W.tiny()
     w.max_grad_norm = 0.0

@@ -147,8 +147,9 @@ def test_commit_repoints_buckets_and_recycles_slots():
     assert sorted(B.so_bucket_slot(ctx, b) for b in range(4)) == [0, 1, 2, 3]
     c = B.so_get_counters(ctx)
     assert (c.commits, c.skips, c.clip_resteps) == (2, 0, 0)
-    # 2 batched step launches + 2 bucket reductions, nothing else on a commit
-    assert c.kernel_launches == 4 and c.elems_stepped == 2000 and c.elems_checked == 0
+    # per iteration: the batched step, the reduction (which decides on the device)
+    # and the follow-up launch that reads the verdict (it returns at once on a commit)
+    assert c.kernel_launches == 6 and c.elems_stepped == 2000 and c.elems_checked == 0
     B.so_destroy(ctx)
 
 
@@ -262,7 +263,7 @@ def test_batches_of_more_than_128_buckets_are_split_into_several_launches():
     B.so_adam_step_speculative(ctx, hp, B.SO_ALL)
     assert B.so_get_counters(ctx).kernel_launches == 3
     B.so_validate_commit_or_rollback(ctx, hp)
-    assert B.so_get_counters(ctx).kernel_launches == 4
+    assert B.so_get_counters(ctx).kernel_launches == 3 + 1 + 3     # reduction, 3 follow-up launches
     B.so_destroy(ctx)
 
 
@@ -314,10 +315,10 @@ def test_deferred_validation_state_machine():
     B.so_validate_begin(ctx, hp)                                         # scans buckets 1..3
     assert B.so_get_counters(ctx).elems_checked == 1000 - 256
     assert B.so_validate_poll(ctx) is True
-    assert _status(B.so_adam_step_speculative, ctx, hp, 1) == B.SO_ERR_STATE
-    assert _status(B.so_grad_check, ctx, None, 1) == B.SO_ERR_STATE
     assert _status(B.so_validate_begin, ctx, hp) == B.SO_ERR_STATE       # already begun
-    st = B.so_grad_check(ctx, hp, B.SO_ALL)                              # finishing is allowed
+    assert _status(B.so_cast_params, ctx) == B.SO_ERR_STATE              # verdict not collected
+    assert _status(B.so_set_step, ctx, 3) == B.SO_ERR_STATE
+    st = B.so_grad_check(ctx, hp, B.SO_ALL)                              # its statistics: allowed
     assert st.nonfinite == 0
     assert B.so_validate_poll(ctx) is True
     r = B.so_validate_commit_or_rollback(ctx, hp)
@@ -325,6 +326,42 @@ def test_deferred_validation_state_machine():
     B.so_validate_begin(ctx, hp)                                         # check-first flow, deferred
     r = B.so_validate_commit_or_rollback(ctx, hp)
     assert r.step_after == 2 and r.buckets_speculated == 0
+    B.so_destroy(ctx)
+
+
+def test_next_iteration_may_be_assembled_while_a_verdict_is_pending():
+    """The verdict is formed on the device; the host may run one iteration
+    ahead of its own bookkeeping.  Collecting validates the older iteration
+    and leaves the newer one open."""
+    ctx, _ = _dry_ctx([1000], 256, undo=2)
+    hp = HP(max_grad_norm=1.0)
+    for b in range(4):
+        B.so_debug_set_bucket_stats(ctx, b, 0.01, 0)
+    B.so_adam_step_speculative(ctx, hp, B.SO_ALL)            # buckets 0, 1 speculated
+    B.so_validate_begin(ctx, hp)                              # 2, 3 scanned; verdict pending
+    before = [B.so_bucket_slot(ctx, b) for b in range(4)]
+    assert before == [0, 1, 2, 3]                             # host map not yet updated
+    # iteration 2 is assembled on top of the pending verdict
+    B.so_adam_step_speculative(ctx, hp, 3)
+    B.so_grad_check(ctx, None, 0)
+    assert B.so_pending_buckets(ctx) == 2
+    assert _status(B.so_adam_step_speculative, ctx, hp, 3) == B.SO_ERR_STATE     # twice
+    assert _status(B.so_grad_check, ctx, hp, B.SO_ALL) == B.SO_ERR_STATE         # a new iteration is open
+    assert _status(B.so_validate_begin, ctx, hp) == B.SO_ERR_STATE               # collect first
+    r = B.so_validate_commit_or_rollback(ctx, hp)             # collects iteration 1
+    assert r.decision == B.SO_DECISION_COMMIT and r.step_after == 1 and r.buckets_speculated == 2
+    assert [B.so_bucket_slot(ctx, b) for b in range(4)] == [4, 5, 2, 3]
+    assert B.so_pending_buckets(ctx) == 2                     # iteration 2 untouched
+    for b in range(4):
+        B.so_debug_set_bucket_stats(ctx, b, 25.0, 0)          # norm 10: clip
+    r = B.so_validate_commit_or_rollback(ctx, hp)             # now validates iteration 2
+    assert r.decision == B.SO_DECISION_CLIP_RESTEP and r.step_after == 2 and r.buckets_speculated == 1
+    # bucket 3 took spare index 0, which held slot 0 after the first commit
+    assert [B.so_bucket_slot(ctx, b) for b in range(4)] == [4, 5, 2, 0]
+    c = B.so_get_counters(ctx)
+    assert (c.commits, c.clip_resteps) == (1, 1)
+    # iteration 1: 512 speculated + 488 in place; iteration 2: 232 speculated + 1000 re-stepped
+    assert c.elems_stepped == 512 + 488 + 232 + 1000
     B.so_destroy(ctx)
 
 
