@@ -25,7 +25,7 @@ class BucketedAdamW:
 
     def __init__(self, numel: Sequence[int], bucket_elems: int, grad_dtype: str = "bf16",
                  undo_slots: int = B.SO_ALL, device: str = "cuda", guard_bands: bool = False,
-                 step_variant: int = 0):
+                 step_variant: int = 0, param_dtype: str = "bf16"):
         self.device = torch.device(device)
         gd = {"bf16": B.SO_GRAD_BF16, "fp32": B.SO_GRAD_FP32, "fp16": B.SO_GRAD_FP16}[grad_dtype]
         self.ctx, self.info = B.so_layout_init(list(numel), bucket_elems, gd, undo_slots)
@@ -34,13 +34,16 @@ class BucketedAdamW:
         self.grad_torch_dtype = {B.SO_GRAD_BF16: torch.bfloat16, B.SO_GRAD_FP32: torch.float32,
                                  B.SO_GRAD_FP16: torch.float16}[gd]
         self.guard_bands = guard_bands
+        self.param_torch_dtype = {"bf16": torch.bfloat16, "fp16": torch.float16}[param_dtype]
+        if param_dtype == "fp16":
+            B.so_param_dtype_config(self.ctx, B.SO_PARAM_FP16)
         i = self.info
         self._raw = {}
         self.master = self._arena("master", i.bytes_master, torch.float32)
         self.m = self._arena("m", i.bytes_m, torch.float32)
         self.v = self._arena("v", i.bytes_v, torch.float32)
         self.grad = self._arena("grad", i.bytes_grad, self.grad_torch_dtype)
-        self.param_bf16 = self._arena("param_bf16", i.bytes_param_bf16, torch.bfloat16)
+        self.param_bf16 = self._arena("param_bf16", i.bytes_param_bf16, self.param_torch_dtype)
         self.scratch = self._arena("scratch", i.bytes_scratch, torch.uint8)
         B.so_layout_bind(self.ctx, self.master.data_ptr(), self.m.data_ptr(), self.v.data_ptr(),
                          self.grad.data_ptr(), self.param_bf16.data_ptr(),
@@ -163,11 +166,20 @@ class BucketedAdamW:
 
     def gather_param_bf16(self) -> torch.Tensor:
         N = self.info.total_elems
-        out = torch.empty(N, dtype=torch.bfloat16, device=self.device)
+        out = torch.empty(N, dtype=self.param_torch_dtype, device=self.device)
         for b in range(self.n_buckets):
             lo, hi = self.bucket_range(b)
             out[lo:hi].copy_(self._slot_view(self.param_bf16, b, hi - lo))
         return out
+
+    def pack_grads(self, tensors, stream=None) -> None:
+        """Gradients of the individual tensors -> gradient arena, one launch."""
+        B.so_layout_pack_grads(self.ctx, [t.data_ptr() if t.numel() else 0 for t in tensors], stream)
+
+    def unpack_params(self, tensors, stream=None) -> None:
+        """Low-precision parameter arena -> the individual tensors, one launch."""
+        B.so_layout_unpack_params(self.ctx, [t.data_ptr() if t.numel() else 0 for t in tensors],
+                                  stream)
 
     # ---- the path -------------------------------------------------------
     def cast_params(self, bucket: int = B.SO_ALL, stream=None) -> None:
@@ -181,6 +193,10 @@ class BucketedAdamW:
 
     def validate(self, hp, stream=None):
         return B.so_validate_commit_or_rollback(self.ctx, hp, stream)
+
+    def validate_begin(self, hp, stream=None) -> None:
+        """Enqueue the end of the iteration (verdict formed on the device)."""
+        B.so_validate_begin(self.ctx, hp, stream)
 
     def iteration(self, hp, stream=None, speculative: bool = True):
         """One whole pass: speculate every bucket that fits, check, validate."""

@@ -53,18 +53,24 @@ class Report:
     loss_scales: list = field(default_factory=list)
 
 
+def _ordered16(bits: np.ndarray) -> np.ndarray:
+    """Monotone integer image of 16-bit sign-magnitude float patterns."""
+    u = bits.astype(np.int64)
+    return np.where(u & 0x8000, -(u & 0x7FFF), u)
+
+
 def assert_bf16_consistent(pb_dev: np.ndarray, p_dev: np.ndarray, pb_orc: np.ndarray,
-                           p_orc: np.ndarray, rep: Report) -> None:
-    """The bf16 copy must be the RNE cast of the device's own master (bit
-    exact), hence equal to the oracle's wherever the masters agree and within
-    one bf16 ulp elsewhere."""
-    want = oracle.bf16_rne(p_dev)
-    assert np.array_equal(pb_dev, want), "bf16 copy is not the RNE cast of the device master"
+                           p_orc: np.ndarray, rep: Report, cast=None) -> None:
+    """The low-precision copy must be the RNE cast of the device's own master
+    (bit exact), hence equal to the oracle's wherever the masters agree and
+    within one ulp of the low-precision format elsewhere."""
+    cast = cast or oracle.bf16_rne
+    want = cast(p_dev)
+    assert np.array_equal(pb_dev, want), "low-precision copy is not the RNE cast of the device master"
     same = p_dev.view(np.uint32) == p_orc.view(np.uint32)
     assert np.array_equal(pb_dev[same], pb_orc[same])
     if not same.all():
-        a = bf16_bits_to_f32(pb_dev[~same]).view(np.int32).astype(np.int64) >> 16
-        b = bf16_bits_to_f32(pb_orc[~same]).view(np.int32).astype(np.int64) >> 16
+        a, b = _ordered16(pb_dev[~same]), _ordered16(pb_orc[~same])
         assert np.abs(a - b).max() <= 1
         rep.bf16_mismatch += int((a != b).sum())
 
@@ -96,16 +102,31 @@ def check_stats(stats, orc_res, max_grad_norm: float, rep: Report) -> None:
     assert (stats.clip_coef < 1.0) == (own_coef < 1.0)
 
 
+def oracle_own_coefficient_replay(pre, g_host, w, t, hp, unscale, dev, rep: Report) -> None:
+    """A clip re-step once more, this time with the coefficient the oracle
+    derives from its own norm (nothing the device computed enters): the
+    device's state must still be within the element tolerance."""
+    p, m, v, pb = (a.copy() for a in pre)
+    res = oracle.iteration_stv(p, m, v, pb, g_host, w.bucket_elems, t, hp, unscale=unscale)
+    assert res.decision == oracle.DECISION_CLIP_RESTEP
+    own = Report()
+    compare_state(dev, (p, m, v), own)
+    for name in "pmv":
+        rep.max_ulp[name] = max(rep.max_ulp[name], own.max_ulp[name])
+
+
 def run_lockstep(w: W.Workload, steps: int, undo_slots: int = B.SO_ALL,
                  speculative: bool = True, guard_bands: bool = True, step_variant: int = 0,
-                 drive=None):
+                 drive=None, param_dtype: str = "bf16"):
     """Full element-by-element parity over `steps` iterations of workload w.
     `drive(opt, hp, stream, step)`, if given, issues the iteration's calls itself
     (in whatever order and granularity) and returns the validation result."""
     hp = hparams_of(w)
     stream = torch.cuda.current_stream()
     opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, undo_slots,
-                        guard_bands=guard_bands, step_variant=step_variant)
+                        guard_bands=guard_bands, step_variant=step_variant,
+                        param_dtype=param_dtype)
+    lp_cast = oracle.fp16_rne if param_dtype == "fp16" else oracle.bf16_rne
     p0 = W.initial_master(w, device="cuda")
     opt.load_state(p0)
     opt.cast_params(stream=stream)
@@ -115,7 +136,7 @@ def run_lockstep(w: W.Workload, steps: int, undo_slots: int = B.SO_ALL,
     m = np.zeros_like(p)
     v = np.zeros_like(p)
     pb = bf16_to_numpy(opt.gather_param_bf16())
-    assert np.array_equal(pb, oracle.bf16_rne(p)), "initial cast differs from the oracle"
+    assert np.array_equal(pb, lp_cast(p)), "initial cast differs from the oracle"
     rep = Report()
     t = 0
     loss_scale, good_steps = w.loss_scale, 0
@@ -134,8 +155,12 @@ def run_lockstep(w: W.Workload, steps: int, undo_slots: int = B.SO_ALL,
 
         # oracle replay from the device's pre-step state
         forced = res.stats.clip_coef if res.decision == B.SO_DECISION_CLIP_RESTEP else None
+        pre = (p.copy(), m.copy(), v.copy(), pb.copy()) if forced is not None else None
+        t_before, unscale_now = t, 1.0 / loss_scale
         orc_res = oracle.iteration_stv(p, m, v, pb, g_host, w.bucket_elems, t, hp,
-                                       forced_coef=forced, unscale=1.0 / loss_scale)
+                                       forced_coef=forced, unscale=unscale_now)
+        if param_dtype == "fp16":
+            pb = lp_cast(p)          # the oracle's iteration casts to bf16; this mode keeps binary16
         # the loss-scale schedule must follow the oracle's, exactly
         loss_scale, good_steps = oracle.loss_scale_update(
             loss_scale, good_steps, orc_res.nonfinite, w.ls_growth, w.ls_backoff, w.ls_interval)
@@ -152,7 +177,9 @@ def run_lockstep(w: W.Workload, steps: int, undo_slots: int = B.SO_ALL,
         dev = [x.cpu().numpy() for x in opt.gather_state()]
         pb_dev = bf16_to_numpy(opt.gather_param_bf16())
         compare_state(dev, (p, m, v), rep)
-        assert_bf16_consistent(pb_dev, dev[0], pb, p, rep)
+        assert_bf16_consistent(pb_dev, dev[0], pb, p, rep, lp_cast)
+        if pre is not None:
+            oracle_own_coefficient_replay(pre, g_host, w, t_before, hp, unscale_now, dev, rep)
         if res.decision == B.SO_DECISION_SKIP:
             for a, b in zip(dev, (p, m, v)):
                 assert a.tobytes() == b.tobytes(), "SKIP did not restore the state bit for bit"
@@ -269,9 +296,8 @@ def write_report(name: str, rep: Report, extra: dict | None = None) -> None:
     """Leave the parity maxima where a results table can pick them up."""
     import json
     import os
-    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    out_dir = os.path.join(root, "gpurun_out")
-    if not os.path.isdir(out_dir):
+    out_dir = os.environ.get("SO_PARITY_REPORT_DIR", "")
+    if not out_dir or not os.path.isdir(out_dir):
         return
     rec = {"workload": name, "decisions": rep.decisions, "max_ulp": rep.max_ulp,
            "n_diff": rep.n_diff, "n_elems_compared": rep.n_elems,
@@ -279,3 +305,88 @@ def write_report(name: str, rep: Report, extra: dict | None = None) -> None:
     rec.update(extra or {})
     with open(os.path.join(out_dir, f"parity_{name}.json"), "w") as fh:
         json.dump(rec, fh)
+
+
+# ---------------------------------------------------------------------------
+# the host running one iteration ahead of its own bookkeeping
+# ---------------------------------------------------------------------------
+
+def run_lockstep_pipelined(w: W.Workload, steps: int, undo_slots: int = B.SO_ALL,
+                           per_bucket: bool = False):
+    """Lock-step parity with the verdict formed on the device and collected one
+    iteration late: the speculative steps of iteration k+1 are enqueued while
+    iteration k's verdict is still pending (they choose their step index and
+    loss scale on the device), then iteration k is collected and compared with
+    the oracle, then iteration k+1's validation is enqueued."""
+    hp = hparams_of(w)
+    stream = torch.cuda.current_stream()
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, undo_slots, guard_bands=True)
+    p0 = W.initial_master(w, device="cuda")
+    opt.load_state(p0)
+    opt.cast_params(stream=stream)
+    torch.cuda.synchronize()
+    if w.grad_dtype == "fp16":
+        B.so_loss_scale_config(opt.ctx, w.loss_scale, w.ls_growth, w.ls_backoff, w.ls_interval)
+
+    p = p0.cpu().numpy()
+    m, v = np.zeros_like(p), np.zeros_like(p)
+    pb = oracle.bf16_rne(p)
+    rep = Report()
+    t = 0
+    loss_scale, good_steps = w.loss_scale, 0
+    in_flight = None                 # (host gradients, loss scale) of the iteration awaiting collection
+
+    def collect_and_compare():
+        nonlocal p, m, v, pb, t
+        g_host, scale_used = in_flight
+        res = opt.validate(hp, stream)                       # collects the pending verdict
+        forced = res.stats.clip_coef if res.decision == B.SO_DECISION_CLIP_RESTEP else None
+        orc_res = oracle.iteration_stv(p, m, v, pb, g_host, w.bucket_elems, t, hp,
+                                       forced_coef=forced, unscale=1.0 / scale_used)
+        own_coef = oracle.clip_coef(orc_res.norm, hp.max_grad_norm)
+        assert res.decision == oracle.decision(orc_res.nonfinite, own_coef) == orc_res.decision
+        check_stats(res.stats, orc_res, hp.max_grad_norm, rep)
+        t = orc_res.step_after
+        assert res.step_after == t == opt.step_count
+        rep.decisions.append(res.decision)
+        rep.loss_scales.append(res.loss_scale)
+        # fp32 state as committed by that iteration (the next iteration's
+        # speculative kernels only write spare slots and the low-precision copy)
+        dev = [x.cpu().numpy() for x in opt.gather_state()]
+        compare_state(dev, (p, m, v), rep)
+        if res.decision == B.SO_DECISION_SKIP:
+            for a, b in zip(dev, (p, m, v)):
+                assert a.tobytes() == b.tobytes(), "SKIP did not restore the state bit for bit"
+        p, m, v = dev
+        pb = oracle.bf16_rne(p)
+        return res
+
+    for step in range(1, steps + 1):
+        g = W.gradients(w, step, device="cuda", loss_scale=loss_scale)
+        g_host = grads_to_numpy(g)
+        opt.load_grads(g)
+        if per_bucket:
+            for b in range(opt.n_buckets):
+                try:
+                    opt.step_speculative(hp, b, stream)
+                except B.SuperOffloadError as e:
+                    assert e.status == B.SO_ERR_UNDO_EXHAUSTED
+                    opt.grad_check(hp, b, stream)
+        else:
+            opt.step_speculative(hp, B.SO_ALL, stream)
+        if in_flight is not None:
+            collect_and_compare()
+            assert B.so_get_loss_scale(opt.ctx) == loss_scale      # what this iteration was stored with
+        opt.validate_begin(hp, stream)
+        in_flight = (g_host, loss_scale)
+        # the producer of the next gradients follows the schedule from the data alone
+        bad = int(not np.isfinite(g_host.astype(np.float32) if g_host.dtype != np.uint16
+                                  else bf16_bits_to_f32(g_host)).all())
+        loss_scale, good_steps = oracle.loss_scale_update(loss_scale, good_steps, bad, w.ls_growth,
+                                                          w.ls_backoff, w.ls_interval)
+    collect_and_compare()
+    torch.cuda.synchronize()
+    pb_dev = bf16_to_numpy(opt.gather_param_bf16())
+    assert np.array_equal(pb_dev, oracle.bf16_rne(p)), "low-precision copy is not the cast of the master"
+    assert opt.guard_bands_intact(), "a kernel wrote outside its arena"
+    return rep, opt

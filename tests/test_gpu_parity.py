@@ -583,3 +583,189 @@ def test_random_call_sequences_lockstep(seed, undo, dtype):
     if undo not in (B.SO_ALL,):
         assert exhausted[0] > 0
     opt.close()
+
+
+# ---------------------------------------------------------------------------
+# verdict on the device, host one iteration behind
+# ---------------------------------------------------------------------------
+
+def _mixed_outcome_workload():
+    """Ragged tensors, norm alternating below / above the clip threshold, one
+    +inf and one NaN: COMMIT, CLIP_RESTEP and SKIP all occur."""
+    w = W.tiny_ragged()
+    w.name = "tiny_ragged_mixed"
+    w.sigma_g = 1.0
+    w.target_norm = lambda step: 0.5 if step % 2 == 1 else 3.0
+    w.faults = (W.Fault(step=3, flat_index=2 * 250_003 + 17, kind="inf"),
+                W.Fault(step=6, flat_index=5, kind="nan"))
+    return w
+
+
+@pytest.mark.parametrize("undo,per_bucket", [(B.SO_ALL, False), (2, False), (3, True)])
+def test_pipelined_iterations_with_the_verdict_on_the_device_lockstep(undo, per_bucket):
+    """The next iteration's speculative steps are enqueued before the host has
+    collected the previous verdict; windowed undo; every outcome."""
+    from gpu_harness import run_lockstep_pipelined
+    rep, opt = run_lockstep_pipelined(_mixed_outcome_workload(), steps=9, undo_slots=undo,
+                                      per_bucket=per_bucket)
+    assert rep.decisions == [C, R, S, R, C, S, C, R, C]
+    assert opt.step_count == 7
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+    # the same trajectory as collecting every verdict at once, bit for bit
+    ref, ref_opt = run_lockstep(_mixed_outcome_workload(), steps=9, undo_slots=undo)
+    assert ref.decisions == rep.decisions
+    assert _state_bytes(opt) == _state_bytes(ref_opt)
+
+
+def test_pipelined_fp16_gradients_pick_the_loss_scale_on_the_device():
+    """Dynamic loss scaling: the scale of iteration k+1 depends on how
+    iteration k ended, which its kernels read on the device."""
+    from gpu_harness import run_lockstep_pipelined
+    w = W.tiny_fp16()
+    rep, opt = run_lockstep_pipelined(w, steps=12, undo_slots=3)
+    ref, ref_opt = run_lockstep(W.tiny_fp16(), steps=12, undo_slots=3)
+    assert rep.decisions == ref.decisions and S in rep.decisions and R in rep.decisions
+    assert rep.loss_scales == ref.loss_scales
+    assert _state_bytes(opt) == _state_bytes(ref_opt)
+
+
+def test_a_kernel_that_gives_up_its_wait_ends_the_iteration_cleanly():
+    """The bulk-copy step kernel polls a bounded number of times for a chunk's
+    loads.  With the limit at zero every warp gives up at once (its copies are
+    still waited for, with the full limit, before the block exits): the device
+    raises its status word, the validation reports SO_ERR_TIMEOUT, the committed
+    state is untouched, and the same iteration then runs normally."""
+    w = W.tiny()
+    hp = hparams_of(w)
+    stream = torch.cuda.current_stream()
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, 3, guard_bands=True)
+    opt.load_state(W.initial_master(w, device="cuda"))
+    opt.cast_params(stream=stream)
+    g = W.gradients(w, 1, device="cuda")
+    opt.load_grads(g)
+    torch.cuda.synchronize()
+    before = _state_bytes(opt)
+    B.so_debug_set_spin_limit(opt.ctx, 0)
+    opt.step_speculative(hp, B.SO_ALL, stream)           # buckets 0..2, all warps give up
+    B.so_debug_set_spin_limit(opt.ctx, 1 << 20)
+    with pytest.raises(B.SuperOffloadError) as err:
+        opt.validate(hp, stream)
+    assert err.value.status == B.SO_ERR_TIMEOUT
+    torch.cuda.synchronize()
+    c = opt.counters()
+    assert c.timeouts == 1 and (c.commits, c.skips, c.clip_resteps) == (0, 0, 0)
+    assert opt.step_count == 0 and B.so_pending_buckets(opt.ctx) == 4
+    assert _state_bytes(opt) == before                    # fp32 state and the re-derived bf16 copy
+    # the status was consumed: the iteration is repeated and matches the oracle
+    res = opt.iteration(hp, stream=stream)
+    torch.cuda.synchronize()
+    p = W.initial_master(w, device="cuda").cpu().numpy()
+    m, v = np.zeros_like(p), np.zeros_like(p)
+    pb = oracle.bf16_rne(p)
+    ref = oracle.iteration_stv(p, m, v, pb, grads_to_numpy(g), w.bucket_elems, 0, hp,
+                               forced_coef=res.stats.clip_coef)
+    assert res.decision == ref.decision == R and opt.step_count == 1
+    dev = [x.cpu().numpy() for x in opt.gather_state()]
+    for a, b in zip(dev, (p, m, v)):
+        assert ulp_distance(a, b).max() <= 2
+    assert opt.counters().timeouts == 1 and opt.guard_bands_intact()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_second_moments_that_overflow_fp32_follow_the_oracle(dtype):
+    """Finite gradients around 1e21 with clipping off: (1 - beta2) g^2 exceeds
+    the fp32 range, the stored second moment becomes +Inf, and the update of
+    those elements is exactly the decay term, on both sides, from then on."""
+    w = W.Workload(name="huge_grads", numel=[5000], bucket_elems=2048, sigma_g=1e21, steps=3,
+                   max_grad_norm=0.0, grad_dtype=dtype)
+    rep, opt = run_lockstep(w, steps=3)
+    assert rep.decisions == [C] * 3
+    v = opt.gather_state()[2]
+    assert torch.isinf(v).any() and not torch.isnan(opt.gather_state()[0]).any()
+    assert rep.max_ulp["p"] <= 2 and rep.n_diff["v"] == 0
+
+
+# ---------------------------------------------------------------------------
+# binary16 parameter copy (the paper's FP16 runs)
+# ---------------------------------------------------------------------------
+
+def _is_fp16_nan(bits):
+    b = bits.astype(np.uint32)
+    return ((b & 0x7C00) == 0x7C00) & ((b & 0x03FF) != 0)
+
+
+def test_fp16_cast_is_rne_for_all_2_to_32_patterns():
+    chunk = 1 << 26
+    opt = BucketedAdamW([chunk], 1 << 24, undo_slots=0, param_dtype="fp16")
+    stream = torch.cuda.current_stream()
+    for c in range((1 << 32) // chunk):
+        pats = torch.arange(c * chunk, (c + 1) * chunk, dtype=torch.int64, device="cuda")
+        bits = pats.to(torch.int32) if c < 32 else (pats - (1 << 32)).to(torch.int32)
+        opt.master[:chunk].copy_(bits.view(torch.float32))
+        opt.cast_params(stream=stream)
+        got = opt.param_bf16[:chunk].view(torch.int16)
+        host_in = bits.view(torch.float32).cpu().numpy()
+        want = oracle.fp16_rne(host_in)
+        want_t = torch.from_numpy(want.view(np.int16)).cuda()
+        nan = torch.from_numpy(np.isnan(host_in)).cuda()
+        assert torch.equal(got[~nan], want_t[~nan]), f"chunk {c}"
+        if nan.any():
+            got_nan = got[nan].cpu().numpy().view(np.uint16)
+            assert _is_fp16_nan(got_nan).all(), f"chunk {c}: NaN lost"
+
+
+@pytest.mark.parametrize("name", ["tiny_ragged", "tiny_fp16"])
+def test_fp16_parameter_copy_lockstep(name):
+    """The fused step writes binary16 parameters (with fp16 gradients and loss
+    scaling this is the paper's own precision recipe)."""
+    rep, opt = run_lockstep(W.by_name(name), steps=8, undo_slots=3, param_dtype="fp16")
+    assert S in rep.decisions and rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+    assert opt.param_bf16.dtype == torch.float16
+
+
+# ---------------------------------------------------------------------------
+# flattening on the device: tensor list <-> bucket arenas in one launch
+# ---------------------------------------------------------------------------
+
+@pytest.mark.parametrize("name,dtype", [("tiny_ragged", "bf16"), ("tiny_ragged", "fp32"),
+                                        ("gpt2_small", "bf16")])
+def test_pack_and_unpack_match_the_per_tensor_copies(name, dtype):
+    w = W.by_name(name)
+    w.grad_dtype = dtype
+    stream = torch.cuda.current_stream()
+    opt = BucketedAdamW(w.numel, w.bucket_elems, dtype, 0, guard_bands=True)
+    flat = W.gradients(w, 1, device="cuda")
+    # every tensor in a buffer of its own, starting at an odd element offset for
+    # every other one (no 16-byte alignment to rely on)
+    tensors, pos = [], 0
+    for i, n in enumerate(w.numel):
+        buf = torch.empty(n + 8, dtype=flat.dtype, device="cuda")
+        t = buf[(i % 2) * 3:(i % 2) * 3 + n]
+        t.copy_(flat[pos:pos + n])
+        tensors.append(t)
+        pos += n
+    opt.pack_grads(tensors, stream)
+    torch.cuda.synchronize()
+    packed = opt.grad.clone()
+    opt.grad.zero_()
+    opt.load_grads(flat)                                   # the per-bucket torch copies
+    torch.cuda.synchronize()
+    assert torch.equal(packed.view(torch.uint8), opt.grad.view(torch.uint8))
+
+    opt.load_state(W.initial_master(w, device="cuda"))
+    opt.cast_params(stream=stream)
+    want = opt.gather_param_bf16()
+    outs = []
+    for i, n in enumerate(w.numel):
+        buf = torch.full((n + 8,), 7.0, dtype=torch.bfloat16, device="cuda")
+        outs.append((buf, buf[(i % 2) * 5:(i % 2) * 5 + n]))
+    opt.unpack_params([t for _, t in outs], stream)
+    torch.cuda.synchronize()
+    pos = 0
+    for i, (buf, t) in enumerate(outs):
+        n = w.numel[i]
+        assert torch.equal(t.view(torch.int16), want[pos:pos + n].view(torch.int16)), i
+        lead = (i % 2) * 5
+        assert (buf[:lead] == 7.0).all() and (buf[lead + n:] == 7.0).all()     # nothing around it
+        pos += n
+    assert opt.guard_bands_intact()
