@@ -60,6 +60,24 @@ __device__ __forceinline__ int outcome_index(int32_t pick, const Verdict *verdic
     return d == kDecisionSkip ? kAfterSkipped : d == kDecisionAbandon ? kAfterAbandoned : kAfterKept;
 }
 
+// Copy the verdict in scratch into mapped host memory: the fields, one
+// system-wide fence, then the stamp -- a host that sees the stamp sees the rest.
+// One thread does it (the first thread of a step kernel that was enqueued while
+// the verdict was pending, else a one-thread kernel of its own).
+__device__ __forceinline__ void verdict_to_host(const Verdict *src, Verdict *host)
+{
+    volatile Verdict *dst = host;
+    dst->sumsq = __ldcg(&src->sumsq);
+    dst->norm = __ldcg(&src->norm);
+    dst->coef = __ldcg(&src->coef);
+    dst->nonfinite = __ldcg(&src->nonfinite);
+    dst->decision = __ldcg(&src->decision);
+    dst->status = __ldcg(&src->status);
+    const int32_t seq = __ldcg(&src->seq);
+    __threadfence_system();
+    dst->seq = seq;
+}
+
 // The slot tables and the verdict are rewritten by one kernel and read by the
 // next, which may already be resident when they change (dependent launches):
 // they are always read from L2 (ld.global.cg), never from an SM's L1.
@@ -384,12 +402,13 @@ __device__ __forceinline__ void adamw_quad(const float (&gq)[4], float (&pq)[4],
 //                fixed and no sums: after a clip every bucket of the launch
 //                (speculated ones from their prior state, the others in
 //                place), after a commit only the buckets that were merely
-//                checked, after a skip nothing.
+//                checked, after a skip nothing (the low-precision copy of the
+//                speculated buckets is then derived again by the cast kernel).
 // Source and destination slots may be the same slot (in-place): every element
 // is read and written by the same thread, reads first.
 
 // What a follow-up launch does, read from the device verdict.
-struct FollowUp { bool step_all, step_inplace, recast; double scale; };
+struct FollowUp { bool step_all, step_inplace; double scale; };
 
 __device__ __forceinline__ FollowUp follow_up_of(const Verdict *verdict)
 {
@@ -397,40 +416,8 @@ __device__ __forceinline__ FollowUp follow_up_of(const Verdict *verdict)
     FollowUp f;
     f.step_all = d == kDecisionClip;
     f.step_inplace = d == kDecisionCommit;
-    f.recast = d == kDecisionSkip || d == kDecisionAbandon;
     f.scale = d == kDecisionClip ? __ldcg(&verdict->coef) : 1.0;
     return f;
-}
-
-// bf16/fp16 copy of a speculated bucket derived again from its untouched
-// committed master (after a skip): tiles dealt round-robin to all warps.
-__device__ __forceinline__ void recast_speculated(const BucketEntry *e, int n_entries,
-                                                  const SlotTables &tab, const Geometry &geo,
-                                                  const float *master, uint16_t *param_lp, bool fp16,
-                                                  uint32_t warp, uint32_t n_warps, uint32_t lane)
-{
-    const uint32_t tps = geo.tiles_per_slot;
-    const uint32_t total_tiles = (uint32_t)n_entries * tps;
-    for (uint32_t tile = warp; tile < total_tiles; tile += n_warps) {
-        const uint32_t j = tile / tps;
-        const uint32_t lt = tile - j * tps;
-        if (e[j].free_idx < 0) continue;
-        const int32_t b = e[j].bucket;
-        const uint32_t n = (b == geo.last_bucket) ? geo.last_elems : geo.bucket_elems;
-        const uint32_t base = lt * kTileElems;
-        if (base >= n) continue;
-        const float *p = master + (int64_t)__ldcg(&tab.slot_of[b]) * geo.stride;
-        uint16_t *pb = param_lp + (int64_t)b * geo.stride;
-#pragma unroll 2
-        for (int r = 0; r < kRowsPerTile; ++r) {
-            const uint32_t idx = base + r * kRowElems + lane * 4;
-            if (idx < n) {
-                float pq[4];
-                load_quad(p, idx, n, pq);
-                store_quad_lp(pb, idx, n, pq, fp16);
-            }
-        }
-    }
 }
 
 template <typename GradT, bool kSpec, int kRowsInFlight>
@@ -444,6 +431,8 @@ __global__ void __launch_bounds__(kThreads, 2) adamw_step_kernel(const __grid_co
     const uint32_t total_tiles = (uint32_t)a.n_entries * tps;
     const AdamScalars &k = a.k[outcome_index(a.pick, a.tab.verdict)];
     const bool fp16 = a.param_fp16 != 0;
+    if (a.publish_to != nullptr && blockIdx.x == 0 && threadIdx.x == 0)
+        verdict_to_host(a.tab.verdict, a.publish_to);
 
     FollowUp f{};
     f.scale = 1.0;
@@ -452,11 +441,7 @@ __global__ void __launch_bounds__(kThreads, 2) adamw_step_kernel(const __grid_co
             a.tab.spec_idx[a.e[threadIdx.x].bucket] = a.e[threadIdx.x].free_idx;
     } else {
         f = follow_up_of(a.tab.verdict);
-        if (f.recast) {
-            recast_speculated(a.e, a.n_entries, a.tab, a.geo, a.master, a.param_lp, fp16, warp,
-                              n_warps, lane);
-            return;
-        }
+        if (!f.step_all && !f.step_inplace) return;      // skipped: nothing is stepped
     }
 
     for (uint32_t tile = warp; tile < total_tiles; tile += n_warps) {
@@ -662,14 +647,14 @@ grad_check_kernel(const __grid_constant__ CheckArgs a)
 // A bucket's tile sums are cut into segments of 4096 tiles.  One block folds
 // one segment (each thread adds up to 8 strided tile sums, then a shared-memory
 // tree); the block that finishes a bucket's last outstanding segment folds the
-// segment sums the same way and publishes the bucket's record; the block that
-// publishes the last bucket folds the bucket sums in index order, forms the
-// verdict (norm, clip coefficient, decision), re-points the speculated buckets
-// at their new slots if the iteration is kept, and leaves records and verdict
-// in mapped host memory.  Segment boundaries and all fold orders are fixed, so
-// the result does not depend on which block happens to come last.  The arrival
-// counters start at zero (bind) and are put back to zero by the publishing
-// blocks.
+// tree).  The block that arrives last (one counter for the whole launch) does
+// the rest alone: per bucket the segment sums, then the bucket sums, each added
+// one after the other in index order; then the verdict (norm, clip coefficient,
+// decision); if the iteration is kept it re-points the speculated buckets at
+// their new slots; the verdict stays in scratch for the kernels that follow.
+// Segment boundaries and all fold orders are fixed, so the result does not
+// depend on which block happens to come last.  The arrival counter starts at
+// zero (bind) and is put back to zero by that last block.
 
 // Fold `count` doubles starting at src (stride 1) in the fixed block order.
 __device__ __forceinline__ void block_fold(const double *src, uint32_t count, double *s_sum,
@@ -725,10 +710,10 @@ __device__ __forceinline__ Verdict make_verdict(double sumsq, int nonfinite, int
 
 // Executed by one whole block of kReduceThreads threads: act on the verdict
 // (a kept iteration swaps every speculated bucket's committed and spare slot;
-// any verdict clears the speculation marks), then publish it, device copy
-// first, host copy with its stamp last.
+// any verdict clears the speculation marks), then leave it in scratch for the
+// kernels that follow.
 __device__ __forceinline__ void publish_verdict(const Verdict &v, const SlotTables &tab,
-                                                int32_t n_buckets, Verdict *host_verdict)
+                                                int32_t n_buckets)
 {
     const bool kept = v.decision == kDecisionCommit || v.decision == kDecisionClip;
     for (int32_t b = threadIdx.x; b < n_buckets; b += kReduceThreads) {
@@ -742,21 +727,7 @@ __device__ __forceinline__ void publish_verdict(const Verdict &v, const SlotTabl
             tab.spec_idx[b] = -1;
         }
     }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        *const_cast<Verdict *>(tab.verdict) = v;
-        if (host_verdict) {
-            volatile Verdict *h = host_verdict;
-            h->sumsq = v.sumsq;
-            h->norm = v.norm;
-            h->coef = v.coef;
-            h->nonfinite = v.nonfinite;
-            h->decision = v.decision;
-            h->status = v.status;
-            __threadfence_system();
-            h->seq = v.seq;
-        }
-    }
+    if (threadIdx.x == 0) *const_cast<Verdict *>(tab.verdict) = v;
 }
 
 static __global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(const ReduceArgs a)
@@ -764,6 +735,7 @@ static __global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(co
     __shared__ double s_sum[kReduceThreads];
     __shared__ int s_bad[kReduceThreads];
     __shared__ int s_last;
+    __shared__ Verdict s_verdict;
     wait_for_prior_kernels();
     allow_dependent_launch();      // the kernel after this one waits for our completion itself
     const int32_t b = (int32_t)(blockIdx.x / a.segs_per_slot);
@@ -775,70 +747,51 @@ static __global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(co
     const uint32_t lo = seg * kSegTiles;
     const uint32_t count = n_tiles - lo < (uint32_t)kSegTiles ? n_tiles - lo : (uint32_t)kSegTiles;
 
+    // first level: this block's segment of tile sums
     double sum;
     int bad;
     block_fold(a.partials + (int64_t)b * a.geo.tiles_per_slot + lo, count, s_sum, s_bad, sum, bad);
-    SegSum *segs = a.seg + (int64_t)b * a.segs_per_slot;
     if (threadIdx.x == 0) {
-        segs[seg].sum = sum;
-        segs[seg].bad = bad;
+        SegSum *mine = a.seg + (int64_t)b * a.segs_per_slot + seg;
+        mine->sum = sum;
+        mine->bad = bad;
         __threadfence();
-        s_last = (atomicAdd(&a.arrivals[b], 1u) == n_segs - 1);
+        s_last = (atomicAdd(a.blocks_done, 1u) == a.n_active_blocks - 1u);
     }
     __syncthreads();
     if (!s_last) return;
     __threadfence();
 
-    // this block completed the bucket: fold its segment sums in index order
-    double acc = 0.0;
-    int any_bad = 0;
-    for (uint32_t i = threadIdx.x; i < n_segs; i += kReduceThreads) {
-        acc = __dadd_rn(acc, __ldcg(&segs[i].sum));
-        any_bad |= __ldcg(&segs[i].bad);
-    }
-    s_sum[threadIdx.x] = acc;
-    s_bad[threadIdx.x] = any_bad;
-    __syncthreads();
-    for (int s = kReduceThreads / 2; s > 0; s >>= 1) {
-        if ((int)threadIdx.x < s) {
-            s_sum[threadIdx.x] = __dadd_rn(s_sum[threadIdx.x], s_sum[threadIdx.x + s]);
-            s_bad[threadIdx.x] |= s_bad[threadIdx.x + s];
-        }
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) {
-        BucketStats r;
-        r.sumsq = s_sum[0];
-        r.nonfinite = s_bad[0];
-        r.pad = 0;
-        a.stats[b] = r;
-        a.arrivals[b] = 0;
-        __threadfence();
-        s_last = (atomicAdd(a.buckets_done, 1u) == (uint32_t)a.n_buckets - 1u);
-    }
-    __syncthreads();
-    if (!s_last) return;
-
-    // This block published the last bucket.  It alone writes to the mapped
-    // host copy: all records, the verdict, one system-wide fence, then the
-    // stamp -- a host that sees the stamp therefore sees everything, and the
-    // kernel pays for two trips to host memory instead of one per bucket.
-    __threadfence();
+    // The last block to arrive does the rest.  Second level: one thread per
+    // bucket adds that bucket's segment sums one after the other in index order
+    // and writes the bucket's record.  Third level: the bucket sums, again one
+    // after the other in index order, by one thread (records pass through shared
+    // memory in runs of 512).  Segment sums of other blocks are read from L2.
     double total = 0.0;
     int flag = 0;
     for (int32_t first = 0; first < a.n_buckets; first += kReduceThreads) {
         const int32_t i = first + (int32_t)threadIdx.x;
         __syncthreads();
         if (i < a.n_buckets) {
-            // records of other blocks: read them from L2, not from a stale L1 line
-            const int4 rec = __ldcg(reinterpret_cast<const int4 *>(a.stats + i));
-            if (a.host_stats) *reinterpret_cast<int4 *>(a.host_stats + i) = rec;
-            s_sum[threadIdx.x] = __hiloint2double(rec.y, rec.x);
-            s_bad[threadIdx.x] = rec.z;
+            const uint32_t ni = (i == a.geo.last_bucket) ? a.geo.last_elems : a.geo.bucket_elems;
+            const uint32_t segs_i = ((ni + kTileElems - 1) / kTileElems + kSegTiles - 1) / kSegTiles;
+            const SegSum *segs = a.seg + (int64_t)i * a.segs_per_slot;
+            double acc = 0.0;
+            int any_bad = 0;
+            for (uint32_t q = 0; q < segs_i; ++q) {
+                acc = __dadd_rn(acc, __ldcg(&segs[q].sum));
+                any_bad |= __ldcg(&segs[q].bad);
+            }
+            BucketStats r;
+            r.sumsq = acc;
+            r.nonfinite = any_bad;
+            r.pad = 0;
+            a.stats[i] = r;
+            s_sum[threadIdx.x] = acc;
+            s_bad[threadIdx.x] = any_bad;
         }
         __syncthreads();
         if (threadIdx.x == 0) {
-            // bucket sums are added one after the other in index order
             const int32_t m = a.n_buckets - first < kReduceThreads ? a.n_buckets - first : kReduceThreads;
             for (int32_t q = 0; q < m; ++q) {
                 total = __dadd_rn(total, s_sum[q]);
@@ -846,33 +799,21 @@ static __global__ void __launch_bounds__(kReduceThreads) bucket_reduce_kernel(co
             }
         }
     }
-    __shared__ Verdict s_verdict;
     if (threadIdx.x == 0) {
-        *a.buckets_done = 0;
+        *a.blocks_done = 0;
         const int status = atomicExch(a.status, 0);
         s_verdict = make_verdict(total, flag, status, a.max_grad_norm, a.seq);
         if (!a.decide) s_verdict.decision = -1;
     }
     __syncthreads();
-    Verdict *host_verdict =
-        a.host_stats ? reinterpret_cast<Verdict *>(a.host_stats + a.n_buckets) : nullptr;
-    if (a.decide) {
-        publish_verdict(s_verdict, a.tab, a.n_buckets, host_verdict);
-    } else if (threadIdx.x == 0 && host_verdict) {
-        // a check without a decision: only the sum, the flag and the stamp travel
-        volatile Verdict *h = host_verdict;
-        h->sumsq = s_verdict.sumsq;
-        h->nonfinite = s_verdict.nonfinite;
-        h->decision = -1;
-        h->status = s_verdict.status;
-        __threadfence_system();
-        h->seq = s_verdict.seq;
-    }
-    if (!a.decide && threadIdx.x == 0) {
-        // the device copy that follows the records (read back when the host copy is not mapped)
-        Verdict *d = reinterpret_cast<Verdict *>(a.stats + a.n_buckets);
-        *d = s_verdict;
-    }
+    if (a.decide) publish_verdict(s_verdict, a.tab, a.n_buckets);
+    else if (threadIdx.x == 0) *const_cast<Verdict *>(a.tab.verdict) = s_verdict;
+}
+
+static __global__ void publish_to_host_kernel(const Verdict *src, Verdict *host)
+{
+    wait_for_prior_kernels();
+    if (threadIdx.x == 0) verdict_to_host(src, host);
 }
 
 // The verdict from a sum and a flag the host supplies: after so_grad_check(SO_ALL)
@@ -886,7 +827,7 @@ static __global__ void __launch_bounds__(kReduceThreads) apply_verdict_kernel(co
     if (threadIdx.x == 0)
         s_verdict = make_verdict(a.sumsq, a.nonfinite, a.abandon, a.max_grad_norm, a.seq);
     __syncthreads();
-    publish_verdict(s_verdict, a.tab, a.n_buckets, a.host_verdict);
+    publish_verdict(s_verdict, a.tab, a.n_buckets);
 }
 
 // ---------------------------------------------------------------------------
@@ -895,6 +836,12 @@ static __global__ void __launch_bounds__(kReduceThreads) apply_verdict_kernel(co
 static __global__ void __launch_bounds__(kThreads) cast_params_kernel(const __grid_constant__ CastArgs a)
 {
     wait_for_prior_kernels();
+    if (a.only_after_skip) {
+        // the follow-up of a validation: after a skip (or a give-up) the copy of
+        // the speculated buckets is derived again from their untouched master
+        const int32_t d = __ldcg(&a.tab.verdict->decision);
+        if (d != kDecisionSkip && d != kDecisionAbandon) return;
+    }
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     const uint32_t n_warps = gridDim.x * kWarpsPerBlock;

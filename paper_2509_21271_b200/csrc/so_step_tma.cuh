@@ -189,6 +189,9 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
     const AdamScalars &k = a.k[outcome_index(a.pick, a.tab.verdict)];
     const bool fp16 = a.param_fp16 != 0;
     double scale = 1.0;
+    // the verdict this launch was enqueued behind sets out for the host from here
+    if (a.publish_to != nullptr && blockIdx.x == 0 && threadIdx.x == 0)
+        verdict_to_host(a.tab.verdict, a.publish_to);
     if constexpr (kSpec) {
         for (int i = threadIdx.x; i < a.n_entries; i += S::kThreads) {
             entries[i] = resolve_speculative(a.tab, a.e[i]);
@@ -197,11 +200,7 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
         if (threadIdx.x == 0) *n_active_smem = a.n_entries;
     } else {
         const FollowUp f = follow_up_of(a.tab.verdict);
-        if (f.recast) {
-            recast_speculated(a.e, a.n_entries, a.tab, a.geo, a.master, a.param_lp, fp16,
-                              blockIdx.x * kTmaWarps + wib, n_warps, lane);
-            return;
-        }
+        if (!f.step_all && !f.step_inplace) return;      // skipped: nothing is stepped
         scale = f.scale;
         if (threadIdx.x == 0) {
             int32_t n = 0;

@@ -98,6 +98,8 @@ struct StepArgs {
     int32_t pick;                         // 1: choose k[] by the device verdict, 0: k[0]
     int32_t param_fp16;                   // low-precision copy is IEEE binary16 instead of bf16
     uint32_t spin_limit;                  // polls of the wait for a chunk's loads
+    Verdict *publish_to;                  // mapped host memory: the first thread of the launch copies
+                                          // the (pending) verdict there before it starts; else nullptr
     int32_t n_entries;
     BucketEntry e[kMaxBatch];
 };
@@ -119,6 +121,7 @@ struct CastArgs {
     Geometry geo;
     SlotTables tab;
     int32_t param_fp16;
+    int32_t only_after_skip;              // 1: do nothing unless the device verdict is a skip / give-up
     int32_t n_entries;
     int32_t bucket[kMaxBatch];
 };
@@ -131,7 +134,7 @@ struct SegSum { double sum; int32_t bad; int32_t pad; };
 // ring of {next tile, finished warps} counter pairs, one pair per launch.
 struct ControlBlock {
     int32_t status;
-    uint32_t buckets_done;                // arrival counter of the bucket reduction
+    uint32_t blocks_done;                 // arrival counter of the bucket reduction
     int32_t pad[2];
     uint32_t counters[kCounterPairs][2];
 };
@@ -139,11 +142,10 @@ struct ControlBlock {
 struct ReduceArgs {
     const double *partials;               // tile sums
     SegSum *seg;                          // n_buckets x segs_per_slot
-    uint32_t *arrivals;                   // n_buckets
     BucketStats *stats;                   // device copy of the records (a Verdict follows them)
-    BucketStats *host_stats;              // mapped host copy of the same layout, or nullptr
     int32_t *status;                      // device status word: read, reported and cleared
-    uint32_t *buckets_done;               // arrival counter over buckets (starts and ends at zero)
+    uint32_t *blocks_done;                // arrival counter over the launch's blocks (starts and ends at zero)
+    uint32_t n_active_blocks;             // blocks that fold a segment (sum over buckets of their segments)
     SlotTables tab;                       // tab.verdict is the device record to write
     double max_grad_norm;
     int32_t decide;                       // 1: form the verdict and re-point the slots here
@@ -157,7 +159,6 @@ struct ReduceArgs {
 // sum and flag: after so_grad_check(SO_ALL), or combined over ranks).
 struct VerdictArgs {
     SlotTables tab;
-    Verdict *host_verdict;                // mapped host copy, or nullptr
     double sumsq, max_grad_norm;
     int32_t nonfinite;
     int32_t abandon;                      // 1: the host gives the iteration up

@@ -82,7 +82,6 @@ struct so_ctx {
     Verdict *d_verdict = nullptr;
     ControlBlock *d_ctrl = nullptr;
     SegSum *d_seg = nullptr;            // per-bucket segment sums of the reduction
-    uint32_t *d_arrivals = nullptr;     // per-bucket arrival counters of the reduction
     int32_t *d_slot_of = nullptr, *d_free_slot = nullptr, *d_spec_idx = nullptr;
     PackTensor *d_tensors = nullptr;    // per-tensor (pointer, flat offset, numel) for pack / unpack
     uint64_t *h_ptr_stage = nullptr;    // pinned staging of a tensor pointer list
@@ -90,11 +89,11 @@ struct so_ctx {
     uint32_t launch_seq = 0;            // picks the counter pair of each pipeline launch
     int step_variant = 0;               // 0: bulk-copy pipeline, 1: register path
     uint32_t spin_limit = kSpinLimit;   // polls a step kernel waits for a chunk (debug hook)
-    BucketStats *h_stats = nullptr;     // host copy: n_buckets records, then a Verdict
-    BucketStats *h_stats_dev = nullptr; // device view of h_stats when it is mapped pinned memory
-    bool h_stats_pinned = false;
+    Verdict *h_verdict = nullptr;       // host copy of the verdict
+    Verdict *h_verdict_dev = nullptr;   // device view of it when it is mapped pinned memory
+    bool h_verdict_pinned = false;
     int32_t reduce_seq = 0;             // stamp of the latest reduction (never 0)
-    cudaEvent_t reduce_done = nullptr;  // completion of the copy-back when h_stats is not mapped
+    cudaEvent_t reduce_done = nullptr;  // completion of the copy-back when the host copy is not mapped
     int occ_step = 0, occ_check = 0, occ_cast = 0;
     // ---- slot map (host mirror of the device tables) ----
     std::vector<int32_t> slot_of;       // committed slot of each bucket
@@ -106,6 +105,8 @@ struct so_ctx {
     bool pend_known = false;            // its verdict was formed from host-supplied statistics
     Verdict pend_verdict{};             //   (then this is it)
     cudaStream_t pend_stream = nullptr;
+    bool pend_published = false;        // something that sends its verdict to the host is enqueued
+    cudaStream_t pend_wait_stream = nullptr;   // stream whose completion implies the verdict is in
     so_grad_stats stats{};              // result of the last completed check
     Progress prog;
     double ls_growth = 2.0, ls_backoff = 0.5;
@@ -144,10 +145,7 @@ SlotTables tables_of(const so_ctx *c)
     return t;
 }
 
-Verdict *host_verdict_of(const so_ctx *c)
-{
-    return reinterpret_cast<Verdict *>(c->h_stats + c->n_buckets);
-}
+Verdict *host_verdict_of(const so_ctx *c) { return c->h_verdict; }
 
 int64_t elems_of(const so_ctx *c, int32_t b)
 {
@@ -360,6 +358,13 @@ so_status launch_steps(so_ctx *c, const std::vector<BucketEntry> &entries, const
         }
         a.param_fp16 = c->param_dtype == SO_PARAM_FP16;
         a.spin_limit = c->spin_limit;
+        a.publish_to = nullptr;
+        if (c->pending && !c->pend_known && !c->pend_published && c->h_verdict_dev && !c->dry_run) {
+            // the pending verdict rides to the host with this launch
+            a.publish_to = c->h_verdict_dev;
+            c->pend_published = true;
+            c->pend_wait_stream = stream;
+        }
         a.n_entries = n;
         for (int i = 0; i < n; ++i) a.e[i] = entries[first + i];
         for (int i = n; i < kMaxBatch; ++i) a.e[i] = BucketEntry{0, -1};
@@ -413,7 +418,10 @@ so_status launch_checks(so_ctx *c, const std::vector<int32_t> &buckets, cudaStre
     return SO_OK;
 }
 
-so_status launch_casts(so_ctx *c, const std::vector<int32_t> &buckets, cudaStream_t stream)
+// only_after_skip: the follow-up of a validation, which casts only if the
+// device verdict is a skip (its elements are counted when the verdict is known).
+so_status launch_casts(so_ctx *c, const std::vector<int32_t> &buckets, cudaStream_t stream,
+                       bool only_after_skip = false)
 {
     const Geometry geo = geometry_of(c);
     for (size_t first = 0; first < buckets.size(); first += kMaxBatch) {
@@ -424,10 +432,11 @@ so_status launch_casts(so_ctx *c, const std::vector<int32_t> &buckets, cudaStrea
         a.geo = geo;
         a.tab = tables_of(c);
         a.param_fp16 = c->param_dtype == SO_PARAM_FP16;
+        a.only_after_skip = only_after_skip ? 1 : 0;
         a.n_entries = n;
         for (int i = 0; i < n; ++i) {
             a.bucket[i] = buckets[first + i];
-            c->counters.elems_cast += elems_of(c, a.bucket[i]);
+            if (!only_after_skip) c->counters.elems_cast += elems_of(c, a.bucket[i]);
         }
         for (int i = n; i < kMaxBatch; ++i) a.bucket[i] = 0;
         cudaError_t e = cudaSuccess;
@@ -456,7 +465,7 @@ so_status scan_uncovered(so_ctx *c, cudaStream_t stream)
 }
 
 // The per-bucket reduction; with `decide` its last block also forms the verdict
-// and re-points the slots.  Its records travel to the host on their own.
+// and re-points the slots.
 so_status launch_reduce(so_ctx *c, double max_grad_norm, bool decide, cudaStream_t stream)
 {
     c->reduce_seq = c->reduce_seq == 0x7FFFFFFF ? 1 : c->reduce_seq + 1;
@@ -466,11 +475,13 @@ so_status launch_reduce(so_ctx *c, double max_grad_norm, bool decide, cudaStream
         ReduceArgs r;
         r.partials = c->d_partials;
         r.seg = c->d_seg;
-        r.arrivals = c->d_arrivals;
         r.stats = c->d_stats;
-        r.host_stats = c->h_stats_dev;     // records land in host memory directly
         r.status = &c->d_ctrl->status;
-        r.buckets_done = &c->d_ctrl->buckets_done;
+        r.blocks_done = &c->d_ctrl->blocks_done;
+        int64_t active = 0;
+        for (int32_t b = 0; b < c->n_buckets; ++b)
+            active += ((elems_of(c, b) + kTileElems - 1) / kTileElems + kSegTiles - 1) / kSegTiles;
+        r.n_active_blocks = (uint32_t)active;
         r.tab = tables_of(c);
         r.max_grad_norm = max_grad_norm;
         r.decide = decide ? 1 : 0;
@@ -481,18 +492,26 @@ so_status launch_reduce(so_ctx *c, double max_grad_norm, bool decide, cudaStream
         const int64_t blocks = (int64_t)c->n_buckets * c->segs_per_slot;
         e = launch_dependent(bucket_reduce_kernel, (unsigned)blocks, kReduceThreads, 0, stream, r);
     }
-    so_status s = after_launch(c, e);
-    if (s != SO_OK) return s;
-    if (!c->dry_run && !c->h_stats_dev) {
-        e = cudaMemcpyAsync(c->h_stats, c->d_stats,
-                            sizeof(BucketStats) * (size_t)c->n_buckets + sizeof(Verdict),
-                            cudaMemcpyDeviceToHost, stream);
-        if (e == cudaSuccess && !c->reduce_done)
-            e = cudaEventCreateWithFlags(&c->reduce_done, cudaEventDisableTiming);
-        if (e == cudaSuccess) e = cudaEventRecord(c->reduce_done, stream);
-        if (e != cudaSuccess) return cuda_fail(c, e);
+    return after_launch(c, e);
+}
+
+// Send the verdict of the latest reduction to the host with a kernel of its
+// own (used when no step kernel is there to carry it).
+so_status publish_to_host(so_ctx *c, cudaStream_t stream)
+{
+    if (c->dry_run || c->n_buckets == 0) return SO_OK;
+    cudaError_t e = cudaSuccess;
+    c->pend_wait_stream = stream;
+    if (c->h_verdict_dev) {
+        e = launch_dependent(publish_to_host_kernel, 1u, 32u, 0, stream,
+                             static_cast<const Verdict *>(c->d_verdict), c->h_verdict_dev);
+        return after_launch(c, e);
     }
-    return SO_OK;
+    e = cudaMemcpyAsync(c->h_verdict, c->d_verdict, sizeof(Verdict), cudaMemcpyDeviceToHost, stream);
+    if (e == cudaSuccess && !c->reduce_done)
+        e = cudaEventCreateWithFlags(&c->reduce_done, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventRecord(c->reduce_done, stream);
+    return e == cudaSuccess ? SO_OK : cuda_fail(c, e);
 }
 
 // The verdict from statistics the host holds (after so_grad_check(SO_ALL), or
@@ -504,7 +523,6 @@ so_status launch_verdict(so_ctx *c, const Verdict &v, double max_grad_norm, cuda
     if (!c->dry_run) {
         VerdictArgs a;
         a.tab = tables_of(c);
-        a.host_verdict = nullptr;
         a.sumsq = v.sumsq;
         a.max_grad_norm = max_grad_norm;
         a.nonfinite = v.nonfinite;
@@ -516,16 +534,28 @@ so_status launch_verdict(so_ctx *c, const Verdict &v, double max_grad_norm, cuda
     return after_launch(c, e);
 }
 
-// The launch that follows a verdict: every bucket of the open iteration, with
-// the spare slot index of the speculated ones; the kernels read on the device
-// what there is to do.
+// What is enqueued behind a verdict; the kernels read on the device what there
+// is to do.  After a skip the low-precision copy of the speculated buckets is
+// derived again (a light kernel that returns at once otherwise).  The step
+// kernel is launched only when the verdict can call for it: buckets that were
+// merely checked take their step in place after a commit or a clip, and with
+// clipping enabled a clip re-steps every bucket.
 so_status launch_follow_up(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
 {
     std::vector<BucketEntry> all;
+    std::vector<int32_t> speculated;
     all.reserve((size_t)c->n_buckets);
-    for (int32_t b = 0; b < c->n_buckets; ++b)
-        all.push_back(BucketEntry{b, c->cur.cover[b] == kSpeculated ? c->cur.free_idx[b] : -1});
-    if (all.empty()) return SO_OK;
+    for (int32_t b = 0; b < c->n_buckets; ++b) {
+        const bool spec = c->cur.cover[b] == kSpeculated;
+        all.push_back(BucketEntry{b, spec ? c->cur.free_idx[b] : -1});
+        if (spec) speculated.push_back(b);
+    }
+    if (!speculated.empty()) {
+        const so_status s = launch_casts(c, speculated, stream, /*only_after_skip=*/true);
+        if (s != SO_OK) return s;
+    }
+    const bool may_step = speculated.size() < all.size() || hp.max_grad_norm > 0.0;
+    if (all.empty() || !may_step) return SO_OK;
     return launch_steps(c, all, hp, /*speculative=*/false, stream);
 }
 
@@ -535,7 +565,7 @@ so_status launch_follow_up(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
 bool reduction_arrived(so_ctx *c)
 {
     if (c->dry_run || c->n_buckets == 0) return true;
-    if (c->h_stats_dev) {
+    if (c->h_verdict_dev) {
         const volatile int32_t *stamp = &host_verdict_of(c)->seq;
         return *stamp == c->reduce_seq;
     }
@@ -548,8 +578,8 @@ so_status wait_for_reduction(so_ctx *c, cudaStream_t stream)
 {
     if (c->dry_run || c->n_buckets == 0) return SO_OK;
     cudaError_t e = cudaSuccess;
-    if (c->h_stats_dev) {
-        // The records arrive in mapped host memory; watching for the stamp
+    if (c->h_verdict_dev) {
+        // The verdict arrives in mapped host memory; watching for the stamp
         // that follows them is several microseconds quicker than waiting for
         // the stream's completion to be signalled.
         const auto t0 = std::chrono::steady_clock::now();
@@ -580,7 +610,6 @@ void inject_records(so_ctx *c, double max_grad_norm, bool decide, bool consume_s
     double sumsq = 0.0;
     int flag = 0;
     for (int32_t b = 0; b < c->n_buckets; ++b) {
-        c->h_stats[b] = c->injected[b];
         sumsq += c->injected[b].sumsq;
         flag |= c->injected[b].nonfinite != 0;
     }
@@ -618,6 +647,7 @@ so_status begin_validation(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
     if (s != SO_OK) return s;
     make_pending(c, hp, stream);
     c->pend_known = false;
+    c->pend_published = false;      // the next step launch carries it, or whoever asks first sends it
     return SO_OK;
 }
 
@@ -647,7 +677,13 @@ so_status pending_verdict(so_ctx *c, Verdict *v, bool consume_status)
     if (c->dry_run) {
         inject_records(c, c->pend.hp.max_grad_norm, /*decide=*/true, consume_status);
     } else {
-        const so_status s = wait_for_reduction(c, c->pend_stream);
+        so_status s = SO_OK;
+        if (!c->pend_published) {
+            s = publish_to_host(c, c->pend_stream);
+            if (s != SO_OK) return s;
+            c->pend_published = true;
+        }
+        s = wait_for_reduction(c, c->pend_wait_stream);
         if (s != SO_OK) return s;
     }
     if (c->n_buckets > 0) std::memcpy(v, host_verdict_of(c), sizeof(*v));
@@ -738,7 +774,7 @@ cudaError_t grad_check_occupancy(int grad_dtype, int *blocks_per_sm)
 // ============================================================================
 
 // Scratch: tile sums | per-bucket records + verdict | control block | segment
-// sums | arrival counters | slot tables | tensor table of pack / unpack.
+// sums | slot tables | tensor table of pack / unpack.
 static uint64_t round256(uint64_t x) { return (x + 255u) / 256u * 256u; }
 
 extern "C" {
@@ -824,7 +860,6 @@ so_status so_layout_get_info(const so_ctx *c, so_layout_info *info)
                           round256(nb * sizeof(BucketStats) + sizeof(Verdict)) +
                           round256(sizeof(ControlBlock)) +
                           round256(nb * segs * sizeof(SegSum)) +
-                          round256(nb * 4u) +
                           round256((2u * nb + (uint64_t)c->undo_slots) * 4u) +
                           round256((uint64_t)c->numel.size() * sizeof(PackTensor)) + 256u;
     return SO_OK;
@@ -876,26 +911,40 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
         e = allow_smem<uint16_t, ShapeBf16>();
         if (e == cudaSuccess) e = allow_smem<half_t, ShapeBf16>();
         if (e == cudaSuccess) e = allow_smem<float, ShapeFp32>();
+        // The small kernels that run between step kernels ask for the same
+        // shared-memory / L1 split as those: an SM does not have to be drained
+        // and reconfigured every time one follows the other.
+        const auto same_split = [&](const void *kernel) {
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                         cudaSharedmemCarveoutMaxShared);
+        };
+        same_split(reinterpret_cast<const void *>(bucket_reduce_kernel));
+        same_split(reinterpret_cast<const void *>(apply_verdict_kernel));
+        same_split(reinterpret_cast<const void *>(publish_to_host_kernel));
+        same_split(reinterpret_cast<const void *>(cast_params_kernel));
+        same_split(reinterpret_cast<const void *>(grad_check_kernel<uint16_t>));
+        same_split(reinterpret_cast<const void *>(grad_check_kernel<half_t>));
+        same_split(reinterpret_cast<const void *>(grad_check_kernel<float>));
         if (e != cudaSuccess) return cuda_fail(c, e);
     } else {
         c->num_sms = 148;
         c->occ_step = c->occ_check = c->occ_cast = 2;
     }
-    if (!c->h_stats) {
-        const size_t bytes = sizeof(BucketStats) * (size_t)c->n_buckets + sizeof(Verdict);
-        if (!c->dry_run && cudaHostAlloc(reinterpret_cast<void **>(&c->h_stats), bytes,
+    if (!c->h_verdict) {
+        if (!c->dry_run && cudaHostAlloc(reinterpret_cast<void **>(&c->h_verdict), sizeof(Verdict),
                                          cudaHostAllocMapped) == cudaSuccess) {
-            c->h_stats_pinned = true;
-            std::memset(c->h_stats, 0, bytes);
+            c->h_verdict_pinned = true;
+            std::memset(c->h_verdict, 0, sizeof(Verdict));
             void *dev_view = nullptr;
-            if (cudaHostGetDevicePointer(&dev_view, c->h_stats, 0) == cudaSuccess)
-                c->h_stats_dev = static_cast<BucketStats *>(dev_view);
+            if (cudaHostGetDevicePointer(&dev_view, c->h_verdict, 0) == cudaSuccess)
+                c->h_verdict_dev = static_cast<Verdict *>(dev_view);
             else
                 cudaGetLastError();                   // fall back to an explicit copy
         } else {
             if (!c->dry_run) cudaGetLastError();      // clear the failed pinned allocation
-            c->h_stats = static_cast<BucketStats *>(std::calloc(1, bytes));
-            if (!c->h_stats) return SO_ERR_NOMEM;
+            c->h_verdict = static_cast<Verdict *>(std::calloc(1, sizeof(Verdict)));
+            if (!c->h_verdict) return SO_ERR_NOMEM;
         }
     }
     c->master = static_cast<float *>(master);
@@ -917,21 +966,18 @@ so_status so_layout_bind(so_ctx *c, void *master, void *m, void *v, void *grad,
     at += round256(sizeof(ControlBlock));
     c->d_seg = reinterpret_cast<SegSum *>(at);
     at += round256(nb * (uint64_t)c->segs_per_slot * sizeof(SegSum));
-    c->d_arrivals = reinterpret_cast<uint32_t *>(at);
-    at += round256(nb * 4u);
     c->d_slot_of = reinterpret_cast<int32_t *>(at);
     c->d_spec_idx = c->d_slot_of + nb;
     c->d_free_slot = c->d_spec_idx + nb;
     at += round256((2u * nb + (uint64_t)c->undo_slots) * 4u);
     c->d_tensors = reinterpret_cast<PackTensor *>(at);
     if (!c->dry_run && c->n_buckets > 0) {
-        // the control block, the verdict and the arrival counters start at zero,
+        // the control block (status word, arrival counter) and the verdict start at zero,
         // the slot tables at the host's current map; the rest of scratch is
         // written before it is read.  (An empty model binds nothing and touches
         // no device memory.)
         cudaError_t e = cudaMemset(c->d_ctrl, 0, sizeof(ControlBlock));
         if (e == cudaSuccess) e = cudaMemset(c->d_verdict, 0, sizeof(Verdict));
-        if (e == cudaSuccess) e = cudaMemset(c->d_arrivals, 0, sizeof(uint32_t) * nb);
         if (e == cudaSuccess) e = cudaMemset(c->d_spec_idx, 0xFF, sizeof(int32_t) * nb);
         if (e == cudaSuccess)
             e = cudaMemcpy(c->d_slot_of, c->slot_of.data(), sizeof(int32_t) * nb, cudaMemcpyHostToDevice);
@@ -989,6 +1035,8 @@ so_status so_grad_check(so_ctx *c, const so_hparams *hp, int32_t bucket, void *s
         s = scan_uncovered(c, st);
         if (s != SO_OK) return s;
         s = launch_reduce(c, hp->max_grad_norm, /*decide=*/false, st);
+        if (s != SO_OK) return s;
+        s = publish_to_host(c, st);
         if (s != SO_OK) return s;
         if (c->dry_run) inject_records(c, hp->max_grad_norm, false, true);
         else if ((s = wait_for_reduction(c, st)) != SO_OK) return s;
@@ -1111,6 +1159,11 @@ so_status so_validate_poll(so_ctx *c, int32_t *ready)
 {
     if (!c || !ready) return SO_ERR_INVALID_ARG;
     if (c->pending) {
+        if (!c->pend_known && !c->pend_published && !c->dry_run) {
+            const so_status s = publish_to_host(c, c->pend_stream);
+            if (s != SO_OK) return s;
+            c->pend_published = true;
+        }
         *ready = (c->pend_known || reduction_arrived(c)) ? 1 : 0;
         return SO_OK;
     }
@@ -1438,9 +1491,9 @@ void so_destroy(so_ctx *c)
     if (c->copy_in) cudaStreamDestroy(c->copy_in);
     if (c->copy_out) cudaStreamDestroy(c->copy_out);
     if (c->h_ptr_stage) cudaFreeHost(c->h_ptr_stage);
-    if (c->h_stats) {
-        if (c->h_stats_pinned) cudaFreeHost(c->h_stats);
-        else std::free(c->h_stats);
+    if (c->h_verdict) {
+        if (c->h_verdict_pinned) cudaFreeHost(c->h_verdict);
+        else std::free(c->h_verdict);
     }
     delete c;
 }

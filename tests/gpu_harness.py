@@ -102,17 +102,37 @@ def check_stats(stats, orc_res, max_grad_norm: float, rep: Report) -> None:
     assert (stats.clip_coef < 1.0) == (own_coef < 1.0)
 
 
-def oracle_own_coefficient_replay(pre, g_host, w, t, hp, unscale, dev, rep: Report) -> None:
+def oracle_own_coefficient_replay(pre, g_host, w, t, hp, unscale, dev, dev_coef, rep: Report) -> None:
     """A clip re-step once more, this time with the coefficient the oracle
-    derives from its own norm (nothing the device computed enters): the
-    device's state must still be within the element tolerance."""
+    derives from its own norm (nothing the device computed enters).  The two
+    coefficients differ by a rounding or two of the norm; that difference enters
+    every element through the scaled gradient, so the device's state must be
+    within the element tolerance PLUS the change of the scaled-gradient term:
+    (1-b1)|c g| d for m, 2 (1-b2) (c g)^2 d for v, and a few lr d for p, with d
+    the relative difference of the coefficients.  Where the terms of a moment
+    cancel, that is more than 2 ulp of the result; such elements must be rare."""
     p, m, v, pb = (a.copy() for a in pre)
     res = oracle.iteration_stv(p, m, v, pb, g_host, w.bucket_elems, t, hp, unscale=unscale)
     assert res.decision == oracle.DECISION_CLIP_RESTEP
-    own = Report()
-    compare_state(dev, (p, m, v), own)
-    for name in "pmv":
-        rep.max_ulp[name] = max(rep.max_ulp[name], own.max_ulp[name])
+    d = abs(dev_coef - res.clip_coef) / res.clip_coef
+    assert d <= NORM_RTOL
+    if g_host.dtype == np.uint16:
+        g64 = bf16_bits_to_f32(g_host).astype(np.float64)
+    else:
+        g64 = g_host.astype(np.float64)
+    gs = np.abs(g64 * unscale * res.clip_coef)
+    slack = {"p": 8.0 * hp.lr * d, "m": 2.0 * (1.0 - hp.beta1) * gs * d,
+             "v": 4.0 * (1.0 - hp.beta2) * gs * gs * d}
+    for name, a, b in zip("pmv", dev, (p, m, v)):
+        ulps = ulp_distance(a, b)
+        beyond = ulps > MAX_ULP_STATE
+        if beyond.any():
+            gap = np.abs(a.astype(np.float64) - b.astype(np.float64))
+            spacing = np.spacing(np.abs(b).astype(np.float32)).astype(np.float64)
+            allowed = MAX_ULP_STATE * spacing + slack[name]
+            assert (gap[beyond] <= allowed[beyond] if np.ndim(allowed) else gap[beyond] <= allowed).all(), \
+                f"{name}: beyond tolerance even allowing for the coefficients' difference"
+            assert beyond.sum() <= max(2, 1e-5 * a.size), f"{name}: {int(beyond.sum())} elements beyond 2 ulp"
 
 
 def run_lockstep(w: W.Workload, steps: int, undo_slots: int = B.SO_ALL,
@@ -179,7 +199,8 @@ def run_lockstep(w: W.Workload, steps: int, undo_slots: int = B.SO_ALL,
         compare_state(dev, (p, m, v), rep)
         assert_bf16_consistent(pb_dev, dev[0], pb, p, rep, lp_cast)
         if pre is not None:
-            oracle_own_coefficient_replay(pre, g_host, w, t_before, hp, unscale_now, dev, rep)
+            oracle_own_coefficient_replay(pre, g_host, w, t_before, hp, unscale_now, dev,
+                                          res.stats.clip_coef, rep)
         if res.decision == B.SO_DECISION_SKIP:
             for a, b in zip(dev, (p, m, v)):
                 assert a.tobytes() == b.tobytes(), "SKIP did not restore the state bit for bit"
