@@ -170,6 +170,62 @@ def whole_job_value(world: int, params_per_replica: int, ms_per_step: float) -> 
     return world * params_per_replica / (ms_per_step * 1e-3)
 
 
+def sharded_steps(shard, hp, steps: int, stream=None):
+    """`steps` iterations of this rank's shard (speculative steps of the local
+    buckets, local check, the one small all-reduce, validation on the global
+    values).  Returns the decisions; all ranks see the same ones."""
+    return [shard.iteration(hp, stream).decision for _ in range(steps)]
+
+
+def run_sharded(args, w, torch, dist, rank, world, local_rank):
+    """Optimizer states sharded by bucket ranges over the ranks (the paper's
+    multi-Superchip mode): strong scaling of one model, one 24-byte all-reduce
+    per iteration inside the timed region."""
+    from paper_2509_21271_b200 import binding as B
+    from paper_2509_21271_b200 import workloads as W
+    from paper_2509_21271_b200.sharded import ShardedAdamW
+
+    hp = _hparams(w)
+    stream = torch.cuda.current_stream()
+    shard = ShardedAdamW(w.total, w.bucket_elems, w.grad_dtype, args.undo_slots if args.undo_slots >= 0
+                         else B.SO_ALL)
+    n_local = shard.hi - shard.lo
+    mine = W.Workload(name=f"{w.name}_shard{rank}", numel=[n_local], bucket_elems=w.bucket_elems,
+                      sigma_g=w.sigma_g, seed=w.seed + 17 * rank, max_grad_norm=w.max_grad_norm,
+                      grad_dtype=w.grad_dtype)
+    shard.local.load_state_stream(W.iter_initial_master(mine, device="cuda"))
+    shard.local.cast_params(stream=stream)
+    shard.local.load_grads_stream(W.iter_gradients(mine, 1, device="cuda"))
+    torch.cuda.synchronize()
+    sharded_steps(shard, hp, args.warmup, stream)
+    torch.cuda.synchronize()
+    dist.barrier()
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    decisions = sharded_steps(shard, hp, args.steps, stream)
+    t1.record(stream)
+    torch.cuda.synchronize()
+    dist.barrier()
+    torch.cuda.synchronize()
+    (elapsed_ms,) = max_over_ranks([t0.elapsed_time(t1)], "cuda")
+    if rank == 0:
+        ms = elapsed_ms / args.steps
+        from paper_2509_21271_b200.binding import DECISION_NAMES
+        print(json.dumps({
+            "metric": METRIC, "value": w.total / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "params": w.total, "bucket_elems": w.bucket_elems,
+                       "parallelism": "zero_buckets", "buckets_rank0": shard.info.n_buckets,
+                       "exchange_bytes_per_step": shard.exchange_bytes,
+                       "decisions": sorted({DECISION_NAMES[d] for d in decisions}),
+                       "verdict": "global statistics combined on the host (one all-reduce), "
+                                  "applied on the device"},
+            "hbm_gbs_whole_step": BYTES_PER_PARAM[w.grad_dtype] * w.total / (ms * 1e-3) / 1e9}))
+    shard.close()
+
+
 def _hparams(w, oracle_mod=None):
     from paper_2509_21271_b200.binding import so_hparams
     return so_hparams(w.lr, w.beta1, w.beta2, w.eps, w.weight_decay, w.max_grad_norm)
@@ -385,6 +441,9 @@ def main():
     ap.add_argument("--sync-verdict", action="store_true",
                     help="collect every verdict on the host before the next iteration is enqueued "
                          "(default: one iteration late)")
+    ap.add_argument("--sharded", action="store_true",
+                    help="shard the optimizer states by bucket ranges over the ranks (strong "
+                         "scaling, one small all-reduce per iteration) instead of running replicas")
     ap.add_argument("--no-kernel-events", action="store_true",
                     help="no event pairs around speculative launches in the timed region (no roofline)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -421,6 +480,15 @@ def main():
         so_build.build_library()
     if dist is not None:
         dist.barrier()
+
+    if args.sharded:
+        if dist is None:
+            import torch.distributed as dist
+            dist.init_process_group("nccl", init_method="tcp://127.0.0.1:29371", rank=0, world_size=1,
+                                    device_id=torch.device("cuda", local_rank))
+        run_sharded(args, w, torch, dist, rank, world, local_rank)
+        dist.destroy_process_group()
+        return
 
     hp = _hparams(w)
     stream = torch.cuda.current_stream()

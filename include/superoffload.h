@@ -298,13 +298,26 @@ so_status so_validate_poll(so_ctx *ctx, int32_t *ready);
  * 4.7: with ZeRO-style partitioning each process updates only its own subset
  * of the parameters).  The norm and the NaN/Inf check are global quantities:
  * a process that holds a shard calls so_grad_check(SO_ALL) to get its LOCAL
- * sum of squares and flag, combines them with the other shards' (one 16-byte
- * all-reduce: sum of the sums, OR of the flags), hands the result back here,
+ * sum of squares and flag, combines them with the other shards' (one small
+ * all-reduce: sum of the sums, sum of the flags), hands the result back here,
  * and then calls so_validate_commit_or_rollback, which decides and acts on the
  * global values.  Only after so_grad_check(SO_ALL) and before validation
  * (SO_ERR_STATE otherwise).  Host-only.
  */
 so_status so_set_global_grad_stats(so_ctx *ctx, double global_sumsq, int32_t global_nonfinite);
+
+/*
+ * so_abandon_iteration -- give the open iteration up (the caller's side of what
+ * SO_ERR_TIMEOUT does by itself; Section 4.7: with sharded states every process
+ * must end an iteration the same way, so a process told that another one failed
+ * drops its own).  Speculative slots are released, the low-precision copy of the
+ * speculated buckets is derived again from the committed master (one predicated
+ * launch on `stream`), step count and loss scale stay, so_counters.timeouts
+ * counts it, and the context is idle.  Allowed while buckets are covered or
+ * after so_grad_check(SO_ALL); SO_ERR_STATE while a begun validation is
+ * pending; a no-op on an idle context.
+ */
+so_status so_abandon_iteration(so_ctx *ctx, void *stream);
 
 /*
  * so_cast_params -- fp32 master -> bf16 parameter copy, round to nearest even
@@ -349,6 +362,9 @@ so_status so_iteration_host(so_ctx *ctx, const so_hparams *hp, const void *host_
  * It calls no cudaMalloc / cudaFree and nothing else that allocates.
  *   grad          DEVICE, flat gradient of n_elems values in grad_dtype,
  *                 16-byte aligned (input; not modified)
+ *   grad_dtype    SO_GRAD_BF16 or SO_GRAD_FP32 only: binary16 gradients need a
+ *                 loss scale, which lives in a context, and are refused here
+ *                 with SO_ERR_INVALID_ARG
  *   n_elems       0 .. SO_STATIC_CHECK_MAX_ELEMS; larger -> SO_ERR_TOO_LARGE
  *   max_grad_norm clip threshold for the coefficient (<= 0: coefficient 1)
  *   out_device    DEVICE, 8-byte aligned so_grad_stats written by the call

@@ -75,7 +75,7 @@ _lib = None
 
 EXPORTS = ["so_layout_init", "so_layout_get_info", "so_layout_tensor", "so_layout_bind",
            "so_param_dtype_config", "so_layout_pack_grads", "so_layout_unpack_params",
-           "so_debug_set_spin_limit",
+           "so_debug_set_spin_limit", "so_abandon_iteration",
            "so_grad_check", "so_adam_step_speculative", "so_validate_commit_or_rollback",
            "so_validate_begin", "so_validate_poll", "so_set_global_grad_stats",
            "so_cast_params", "so_iteration_host", "so_grad_check_static",
@@ -106,6 +106,7 @@ def lib() -> C.CDLL:
         "so_layout_pack_grads": [vp, P(vp), vp],
         "so_layout_unpack_params": [vp, P(vp), vp],
         "so_debug_set_spin_limit": [vp, i64],
+        "so_abandon_iteration": [vp, vp],
         "so_grad_check": [vp, P(so_hparams), i32, vp, P(so_grad_stats)],
         "so_adam_step_speculative": [vp, P(so_hparams), i32, vp],
         "so_validate_commit_or_rollback": [vp, P(so_hparams), vp, P(so_step_result)],
@@ -263,6 +264,10 @@ def so_validate_poll(ctx) -> bool:
 def so_set_global_grad_stats(ctx, global_sumsq: float, global_nonfinite: int) -> None:
     _ok(ctx, lib().so_set_global_grad_stats(ctx, global_sumsq, int(global_nonfinite)),
         "so_set_global_grad_stats")
+
+
+def so_abandon_iteration(ctx, stream=None) -> None:
+    _ok(ctx, lib().so_abandon_iteration(ctx, _stream(stream)), "so_abandon_iteration")
 
 
 def so_cast_params(ctx, bucket: int = SO_ALL, stream=None) -> None:

@@ -41,8 +41,11 @@ struct DeviceSetup {
 DeviceSetup g_setup[kMaxDevices];
 std::mutex g_setup_mutex;
 
-// Fold the tile sums of one flat gradient in the order bucket_reduce_kernel
-// uses for a bucket (strided per-thread sums, then a shared-memory tree), then
+// Fold the tile sums of one flat gradient (strided per-thread sums, then a
+// shared-memory tree: for up to 4096 tiles, i.e. 4 Mi elements, this is the order
+// in which the regular reduction folds a one-segment bucket, so the bits agree;
+// beyond that the regular check folds per 4096-tile segment first and the two
+// results are equal to rounding), then
 // derive norm and clip coefficient on the device (IEEE sqrt and division are
 // correctly rounded, so the values equal a host computation from the same sum)
 // and write the result record to the caller's device buffer.

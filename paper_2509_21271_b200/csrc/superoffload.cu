@@ -1143,6 +1143,23 @@ so_status so_validate_begin(so_ctx *c, const so_hparams *hp, void *stream)
     return begin_validation(c, *hp, static_cast<cudaStream_t>(stream));
 }
 
+so_status so_abandon_iteration(so_ctx *c, void *stream)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (!c->bound || c->pending) return SO_ERR_STATE;
+    if (c->cur.phase == kIdle) return SO_OK;
+    so_hparams hp = c->cur.hp;
+    if (!c->cur.have_hp) {
+        // only scans so far: any valid constants do, no step follows a give-up
+        hp = so_hparams{0.0, 0.9, 0.999, 1e-8, 0.0, 0.0};
+    }
+    const Verdict gave_up = verdict_of(0.0, 0, 1, hp.max_grad_norm, 0);
+    so_status s = begin_validation_known(c, hp, gave_up, static_cast<cudaStream_t>(stream));
+    if (s != SO_OK) return s;
+    s = collect_validation(c, nullptr);
+    return s == SO_ERR_TIMEOUT ? SO_OK : s;
+}
+
 so_status so_set_global_grad_stats(so_ctx *c, double global_sumsq, int32_t global_nonfinite)
 {
     if (!c) return SO_ERR_INVALID_ARG;

@@ -4,13 +4,19 @@ Each rank owns a contiguous range of the global buckets and a
 :class:`BucketedAdamW` over just that range (the paper's multi-Superchip mode,
 Section 4.7: every process updates only its own subset of the parameters).
 The element updates need nothing from the other ranks; the only exchange is
-the global gradient check: one all-reduce of the local sum of squares (SUM)
-and of the local NaN/Inf flag (MAX), 16 bytes, handed back to the library with
-``so_set_global_grad_stats`` before validation.  An all-gather of the bf16
-parameter shards is offered for callers that keep a full low-precision copy.
+the global gradient check: ONE all-reduce (SUM) of three doubles -- the local
+sum of squares, the local NaN/Inf flag and a local error flag -- whose result
+is handed back to the library with ``so_set_global_grad_stats`` before
+validation.  The error flag keeps the ranks in step: a rank whose local check
+failed (a kernel gave up a bounded wait, a CUDA error) still takes part in the
+exchange, and when any rank reports an error every rank gives the iteration up
+and raises, instead of the healthy ranks blocking in a collective the failed
+one never joins.  An all-gather of the low-precision parameter shards is
+offered for callers that keep a full copy.  Data lands in this rank's own
+memory before any kernel reads it; no kernel is ever given a peer's pointer.
 
-Plumbing only: ``torch.distributed`` moves two doubles; every step of the path
-runs in the library's kernels.
+Plumbing only: ``torch.distributed`` moves three doubles; every step of the
+path runs in the library's kernels.
 """
 from __future__ import annotations
 
@@ -33,6 +39,17 @@ def shard_range(total_elems: int, bucket_elems: int, rank: int, world: int) -> T
     lo = min(first * bucket_elems, total_elems)
     hi = min((first + count) * bucket_elems, total_elems)
     return lo, hi
+
+
+class ShardFailure(RuntimeError):
+    """Some rank's local gradient check failed; every rank gave the iteration up."""
+
+    def __init__(self, failed_ranks: int, local_error: Optional[BaseException]):
+        self.failed_ranks = failed_ranks
+        self.local_error = local_error
+        where = "this rank among them" if local_error is not None else "not this rank"
+        super().__init__(f"{failed_ranks} rank(s) failed their local gradient check ({where}); "
+                         "the iteration was given up on every rank")
 
 
 class ShardedAdamW:
@@ -60,34 +77,44 @@ class ShardedAdamW:
                                        device=device)
             self.ctx, self.info = self.local.ctx, self.local.info
             self.reduce_device = self.local.device
+        self.exchange_bytes = 24
 
     def iteration(self, hp, stream=None):
-        """Speculate the local buckets, check locally, all-reduce the two
-        scalars, validate on the global values."""
-        B.so_adam_step_speculative(self.ctx, hp, B.SO_ALL, stream)
-        local = B.so_grad_check(self.ctx, hp, B.SO_ALL, stream)
-        sums = torch.tensor([local.sumsq], dtype=torch.float64, device=self.reduce_device)
-        flag = torch.tensor([float(local.nonfinite)], dtype=torch.float64,
-                            device=self.reduce_device)
-        if self.world > 1:
-            dist.all_reduce(sums, op=dist.ReduceOp.SUM, group=self.group)
-            dist.all_reduce(flag, op=dist.ReduceOp.MAX, group=self.group)
-        B.so_set_global_grad_stats(self.ctx, float(sums.item()), int(flag.item() != 0.0))
+        """Speculate the local buckets, check locally, exchange three doubles
+        in one all-reduce, validate on the global values."""
+        failure = None
+        sumsq = nonfinite = 0.0
+        try:
+            B.so_adam_step_speculative(self.ctx, hp, B.SO_ALL, stream)
+            local = B.so_grad_check(self.ctx, hp, B.SO_ALL, stream)
+            sumsq, nonfinite = local.sumsq, float(local.nonfinite)
+        except B.SuperOffloadError as e:       # still take part in the exchange
+            failure = e
+        packed = torch.tensor([sumsq, nonfinite, 0.0 if failure is None else 1.0],
+                              dtype=torch.float64, device=self.reduce_device)
+        dist.all_reduce(packed, op=dist.ReduceOp.SUM, group=self.group)
+        g_sumsq, g_nonfinite, g_errors = (float(x) for x in packed.tolist())
+        if g_errors != 0.0:
+            if failure is None or failure.status != B.SO_ERR_TIMEOUT:
+                # the library has not ended this rank's iteration by itself
+                try:
+                    B.so_abandon_iteration(self.ctx, stream)
+                except B.SuperOffloadError:
+                    pass                       # a dead context stays dead; the caller learns below
+            raise ShardFailure(int(g_errors), failure)
+        B.so_set_global_grad_stats(self.ctx, g_sumsq, int(g_nonfinite != 0.0))
         return B.so_validate_commit_or_rollback(self.ctx, hp, stream)
 
     def all_gather_param_bf16(self) -> torch.Tensor:
-        """The full bf16 parameter vector, assembled from every rank's shard."""
+        """The full low-precision parameter vector, assembled from every rank's shard."""
         mine = self.local.gather_param_bf16()
         sizes = [shard_range(self.total_elems, self.info.bucket_elems, r, self.world)
                  for r in range(self.world)]
         longest = max(hi - lo for lo, hi in sizes)
-        padded = torch.zeros(longest, dtype=torch.bfloat16, device=mine.device)
+        padded = torch.zeros(longest, dtype=mine.dtype, device=mine.device)
         padded[:mine.numel()] = mine
         parts = [torch.empty_like(padded) for _ in range(self.world)]
-        if self.world > 1:
-            dist.all_gather(parts, padded, group=self.group)
-        else:
-            parts = [padded]
+        dist.all_gather(parts, padded, group=self.group)
         return torch.cat([p[:hi - lo] for p, (lo, hi) in zip(parts, sizes)])
 
     def close(self) -> None:

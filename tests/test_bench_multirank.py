@@ -59,3 +59,46 @@ def test_reference_arm_prints_one_line_on_rank_zero_only():
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle"
     assert line["value"] > 0 and line["e2e"]["h2d_bytes_per_step"] == 0
     assert line["unit"] == "params/s" and line["n_gpus"] == 2
+
+
+def _sharded_worker(rank, world, port, q):
+    sys.path.insert(0, ROOT)
+    import bench
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2509_21271_b200 import binding as B
+    from paper_2509_21271_b200.sharded import ShardedAdamW
+
+    class HP:
+        lr, beta1, beta2, eps, weight_decay, max_grad_norm = 1e-3, 0.9, 0.999, 1e-8, 0.01, 1.0
+
+    shard = ShardedAdamW(10 * 512 + 7, 512, dry_run=True)
+    for b in range(shard.info.n_buckets):
+        B.so_debug_set_bucket_stats(shard.ctx, b, 4.0 if rank == 1 else 0.001, 0)
+    decisions = bench.sharded_steps(shard, HP(), 3)
+    q.put((rank, decisions, shard.info.n_buckets, B.so_get_step(shard.ctx), shard.exchange_bytes))
+    shard.close()
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_sharded_bench_loop_with_two_gloo_ranks():
+    """The loop `bench.py --sharded` times, on two CPU ranks in dry-run mode:
+    bucket ranges per rank, one exchange per iteration, the same global verdict
+    (rank 1's large gradients make both ranks clip)."""
+    from paper_2509_21271_b200 import binding as B
+    from paper_2509_21271_b200 import build as so_build
+    so_build.build_library()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 27500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_sharded_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = {r[0]: r[1:] for r in (q.get(timeout=180) for _ in procs)}
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert got[0][0] == got[1][0] == [B.SO_DECISION_CLIP_RESTEP] * 3
+    assert got[0][1] + got[1][1] == 11 and abs(got[0][1] - got[1][1]) <= 1
+    assert got[0][2] == got[1][2] == 3 and got[0][3] == 24

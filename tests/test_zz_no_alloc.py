@@ -11,6 +11,8 @@ from __future__ import annotations
 import ctypes
 
 import numpy as np
+
+import oracle
 import pytest
 import torch
 
@@ -71,6 +73,14 @@ def _close(a, b):
     return abs(a - b) <= NORM_RTOL * max(abs(b), 1e-300)
 
 
+def _oracle_check(g: torch.Tensor, max_norm: float):
+    """The CPU oracle on the same bits: (sumsq, norm, clip coefficient, flag)."""
+    host = g.view(torch.int16).cpu().numpy().view(np.uint16) if g.dtype == torch.bfloat16 \
+        else g.cpu().numpy()
+    sumsq, norm, flag = oracle.global_grad_check(host, max(host.size, 1))
+    return sumsq, norm, oracle.clip_coef(norm, max_norm), flag
+
+
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
 def test_static_check_matches_the_regular_check_on_two_calls_in_a_row(dtype):
     gen = torch.Generator(device="cuda").manual_seed(11)
@@ -84,6 +94,8 @@ def test_static_check_matches_the_regular_check_on_two_calls_in_a_row(dtype):
     assert got1[3] == ref1[3] == 0
     assert _close(got1[0], ref1[0]) and _close(got1[1], ref1[1]) and _close(got1[2], ref1[2])
     assert got1[2] < 1.0                                        # norm ~ 17 > 1: clip active
+    want1 = _oracle_check(g1, 1.0)                              # and against the CPU oracle itself
+    assert got1[3] == want1[3] and all(_close(a, b) for a, b in zip(got1[:3], want1[:3]))
 
     # call 2, straight after, smaller: the array still holds call 1's tile sums
     # beyond this call's range, which must not leak into the result
@@ -94,6 +106,8 @@ def test_static_check_matches_the_regular_check_on_two_calls_in_a_row(dtype):
     assert got2[3] == ref2[3] == 0
     assert _close(got2[0], ref2[0]) and _close(got2[1], ref2[1])
     assert got2[2] == ref2[2] == 1.0                            # norm ~ 0.26: no clip
+    want2 = _oracle_check(g2, 1.0)
+    assert want2[2] == 1.0 and _close(got2[0], want2[0]) and _close(got2[1], want2[1])
 
     # with a single bucket the two entry points fold in the same order: same bits
     one_bucket = _regular_check(g2, n2 + 63 - (n2 + 63) % 64, 1.0)
@@ -104,7 +118,7 @@ def test_static_check_matches_the_regular_check_on_two_calls_in_a_row(dtype):
     g3[n2 - 1] = float("inf")
     got3 = _static_check(g3, 0.0, out)
     ref3 = _regular_check(g3, 1 << 16, 0.0)
-    assert got3[3] == ref3[3] == 1
+    assert got3[3] == ref3[3] == _oracle_check(g3, 0.0)[3] == 1
 
 
 def test_static_check_rejects_what_it_cannot_hold_and_handles_empty_input():
@@ -124,3 +138,30 @@ def test_static_check_rejects_what_it_cannot_hold_and_handles_empty_input():
     # exactly representable case: 1024 ones -> norm 32
     ones = torch.ones(1024, dtype=torch.bfloat16, device="cuda")
     assert _static_check(ones, 0.0, out) == (1024.0, 32.0, 1.0, 0)
+
+
+@pytest.mark.parametrize("n", [5 * (1 << 20) + 1, B.SO_STATIC_CHECK_MAX_ELEMS])
+def test_static_check_on_inputs_of_several_segments_and_at_its_capacity(n):
+    """Beyond 4 Mi elements the regular check folds per segment first: the two
+    entry points agree to rounding, and both with the oracle; the largest
+    input the built-in array holds is accepted."""
+    gen = torch.Generator(device="cuda").manual_seed(12)
+    out = torch.zeros(ctypes.sizeof(B.so_grad_stats), dtype=torch.uint8, device="cuda")
+    g = (torch.randn(n, generator=gen, device="cuda") * 1e-3).to(torch.bfloat16)
+    got = _static_check(g, 1.0, out)
+    ref = _regular_check(g, n + (-n) % 64, 1.0)
+    want = _oracle_check(g, 1.0)
+    assert got[3] == ref[3] == want[3] == 0
+    for a, b, c in zip(got[:3], ref[:3], want[:3]):
+        assert _close(a, b) and _close(a, c)
+    again = _static_check(g, 1.0, out)                          # a second call in a row: same bits
+    assert again == got
+
+
+def test_static_check_refuses_fp16_gradients():
+    out = torch.zeros(ctypes.sizeof(B.so_grad_stats), dtype=torch.uint8, device="cuda")
+    g = torch.zeros(1024, dtype=torch.float16, device="cuda")
+    with pytest.raises(B.SuperOffloadError) as err:
+        B.so_grad_check_static(g.data_ptr(), 1024, B.SO_GRAD_FP16, 1.0, torch.cuda.current_stream(),
+                               out.data_ptr())
+    assert err.value.status == B.SO_ERR_INVALID_ARG
