@@ -226,6 +226,100 @@ def run_sharded(args, w, torch, dist, rank, world, local_rank):
     shard.close()
 
 
+def measure_link(torch, n_bytes: int = 1 << 30, repeats: int = 5):
+    """Pinned host <-> device copy rates of this machine (one cudaMemcpyAsync of
+    `n_bytes` each way, best of `repeats`, CUDA events), in bytes/s."""
+    host = torch.empty(n_bytes, dtype=torch.uint8, pin_memory=True)
+    dev = torch.empty(n_bytes, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+    best = {}
+    for name, dst, src in (("h2d", dev, host), ("d2h", host, dev)):
+        times = []
+        for _ in range(repeats + 1):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            dst.copy_(src, non_blocking=True)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        best[name] = n_bytes / (min(times[1:]) * 1e-3)
+    return best
+
+
+PLACEMENT_CONFIGS = (("gpt2_small", 124_439_808, 25_000_000), ("llama_1b", 1_235_814_400, 100_000_000),
+                     ("llama_8b", 8_030_261_248, 200_000_000))
+
+
+def placement_table(step_gpu: float, step_cpu: float, h2d_bytes_s: float, d2h_bytes_s: float,
+                    gemm_flops: float, seq: int = 1024, batches=(1, 4, 8)):
+    """The paper's two placement models fed with rates measured on this machine.
+
+    Section 4.3 (Eq. 4-5): n = buckets whose optimizer state should stay on the
+    GPU so that the last offloaded bucket (gradient out, CPU step, parameters
+    back) hides behind the backward pass and the GPU-side step of those n
+    buckets; the backward pass costs 4 * bsz * seq FLOPs per parameter.
+    Section 4.2 (Eq. 1-3): the smallest batch size at which streaming the
+    low-precision weights in hides behind the forward pass (efficiency 60 %)."""
+    from paper_2509_21271_b200 import placement_model as M
+    rows = []
+    for name, total, bucket in PLACEMENT_CONFIGS:
+        nb = -(-total // bucket)
+        for bsz in batches:
+            rates = M.Rates(move_grad=d2h_bytes_s / 2.0, move_param=h2d_bytes_s / 2.0,
+                            step_cpu=step_cpu, step_gpu=step_gpu,
+                            bwd=gemm_flops / (4.0 * bsz * seq))
+            rows.append({"workload": name, "n_buckets": nb, "bucket_elems": bucket, "batch": bsz,
+                         "seq": seq, "n_gpu_resident": M.gpu_resident_buckets(bucket, nb, rates)})
+    try:
+        min_batch = M.min_batch_for_efficiency(0.6, seq, gemm_flops, h2d_bytes_s)
+    except ValueError:
+        min_batch = None
+    return {"rows": rows, "min_batch_for_60pct_forward_efficiency": min_batch,
+            "forward_efficiency_at_batch_4": M.forward_efficiency(1.0, 4, seq, gemm_flops, h2d_bytes_s)}
+
+
+def run_placement(args, torch):
+    """`--placement`: measure this box's rates and print what the paper's
+    models make of them (one JSON line)."""
+    from paper_2509_21271_b200 import binding as B
+    from paper_2509_21271_b200 import workloads as W
+    from paper_2509_21271_b200.optimizer import BucketedAdamW
+
+    link = measure_link(torch)
+    w = W.by_name("llama_1b" if args.workload == DEFAULT_WORKLOAD else args.workload)
+    hp = _hparams(w)
+    stream = torch.cuda.current_stream()
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, B.SO_ALL)
+    opt.load_state_stream(W.iter_initial_master(w, device="cuda"))
+    opt.cast_params(stream=stream)
+    opt.load_grads_stream(W.iter_gradients(w, 1, device="cuda"))
+    for _ in range(3):
+        opt.iteration(hp, stream=stream)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(10):
+        opt.iteration(hp, stream=stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    step_gpu = w.total * 10 / (e0.elapsed_time(e1) * 1e-3)
+    opt.close()
+    cpu = _oracle_all_cores(w, 5.0)
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            gemm = float(json.load(fh)["bf16_tflops_sustained"]) * 1e12
+        gemm_kind = "measured (sustained bf16 GEMM)"
+    except Exception:
+        gemm, gemm_kind = 1.4e15, "fallback"
+    table = placement_table(step_gpu, cpu["value"], link["h2d"], link["d2h"], gemm)
+    print(json.dumps({"placement": table,
+                      "inputs": {"step_gpu_params_s": step_gpu, "step_gpu_workload": w.name,
+                                 "step_cpu_params_s": cpu["value"], "cpu_cores": cpu["cores"],
+                                 "cpu_model": cpu.get("cpu_model"),
+                                 "h2d_gbs": link["h2d"] / 1e9, "d2h_gbs": link["d2h"] / 1e9,
+                                 "gemm_flops": gemm, "gemm_kind": gemm_kind}}))
+
+
 def _hparams(w, oracle_mod=None):
     from paper_2509_21271_b200.binding import so_hparams
     return so_hparams(w.lr, w.beta1, w.beta2, w.eps, w.weight_decay, w.max_grad_norm)
@@ -441,6 +535,9 @@ def main():
     ap.add_argument("--sync-verdict", action="store_true",
                     help="collect every verdict on the host before the next iteration is enqueued "
                          "(default: one iteration late)")
+    ap.add_argument("--placement", action="store_true",
+                    help="measure this box's rates (fused step, pinned copies, all-cores oracle) and "
+                         "print what the paper's placement models (Eq. 1-5) make of them")
     ap.add_argument("--sharded", action="store_true",
                     help="shard the optimizer states by bucket ranges over the ranks (strong "
                          "scaling, one small all-reduce per iteration) instead of running replicas")
@@ -481,6 +578,12 @@ def main():
     if dist is not None:
         dist.barrier()
 
+    if args.placement:
+        if rank == 0:
+            run_placement(args, torch)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
     if args.sharded:
         if dist is None:
             import torch.distributed as dist
@@ -640,6 +743,7 @@ def main():
             e2e_ms = e0.elapsed_time(e1) / n_e2e
             e2e = {"ms": e2e_ms, "h2d": N * gsz, "d2h": N * 2 + 40, "steps": n_e2e}
             del host_g, host_p
+            e2e["link"] = measure_link(torch)
 
     # ---- max over ranks ----------------------------------------------------
     if dist is not None:
@@ -707,7 +811,13 @@ def main():
         line["e2e"] = {"value": world * N / (e2e["ms"] * 1e-3), "unit": UNIT,
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                        "ms_per_step": e2e["ms"], "steps": e2e["steps"],
-                       "link_gbs_each_way": e2e["h2d"] / (e2e["ms"] * 1e-3) / 1e9}
+                       "link_gbs_each_way": e2e["h2d"] / (e2e["ms"] * 1e-3) / 1e9,
+                       # ceiling: both directions run at once, so a step cannot be
+                       # shorter than the slower direction's copy at the measured rate
+                       "pinned_h2d_gbs": e2e["link"]["h2d"] / 1e9,
+                       "pinned_d2h_gbs": e2e["link"]["d2h"] / 1e9,
+                       "frac_of_link": max(e2e["h2d"] / e2e["link"]["h2d"],
+                                           e2e["d2h"] / e2e["link"]["d2h"]) / (e2e["ms"] * 1e-3)}
     elif e2e:
         line["e2e"] = e2e
     if args.overlap and world == 1:

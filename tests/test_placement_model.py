@@ -48,3 +48,30 @@ def test_gpu_resident_buckets_by_hand():
     fast = M.Rates(100e9, 100e9, 230e9, 230e9, 50e9)
     assert M.gpu_resident_buckets(bucket, 100, fast) < n
     assert M.gpu_resident_buckets(bucket, 3, r) == 3
+
+
+def test_placement_table_from_measured_style_rates():
+    """The table `bench.py --placement` prints, on fixed inputs: with a slow
+    host link and CPU (this build's B200 machine: ~55 GB/s pinned copies, ~1.2 G
+    params/s on all host cores) every bucket stays on the GPU; with the paper's
+    Superchip figures (450 GB/s each way, Table 3's 13 G params/s CPU Adam)
+    only the last few do, and the count shrinks as the batch grows."""
+    import os
+    import sys
+    sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    import bench
+    slow = bench.placement_table(step_gpu=2.2e11, step_cpu=1.2e9, h2d_bytes_s=55e9, d2h_bytes_s=52e9,
+                                 gemm_flops=1.37e15)
+    for row in slow["rows"]:
+        if row["batch"] == 1:
+            assert row["n_gpu_resident"] == row["n_buckets"]
+    fast = bench.placement_table(step_gpu=2.2e11, step_cpu=13e9, h2d_bytes_s=450e9, d2h_bytes_s=450e9,
+                                 gemm_flops=989e12)
+    by = {(r["workload"], r["batch"]): r["n_gpu_resident"] for r in fast["rows"]}
+    assert by[("llama_8b", 8)] <= by[("llama_8b", 4)] <= by[("llama_8b", 1)] <= 41
+    assert 1 <= by[("llama_8b", 8)] < 41
+    # hand-worked: bucket 2e8; exposed = 2e8/225e9 * 2 + 2e8/13e9 = 17.16 ms;
+    # batch 8: bwd rate 989e12/(4*8*1024) = 3.018e10 params/s -> 6.63 ms per bucket,
+    # plus 0.91 ms of GPU step: 7.54 ms per bucket -> 2 buckets cover 15.07 ms, 3 cover 22.6 ms
+    assert by[("llama_8b", 8)] == 3
+    assert fast["min_batch_for_60pct_forward_efficiency"] == 4     # the paper's own statement
