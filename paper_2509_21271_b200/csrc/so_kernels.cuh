@@ -264,40 +264,40 @@ __device__ __forceinline__ double warp_fold(double x)
 // in a million for N(0, 0.02) weights and lr = 1e-3); above that ratio the two
 // orders differ by less than 1 % of half an fp32 ulp of the result.
 
-// sqrt(x) for x >= 0 in double, to within about an ulp: hardware reciprocal-
-// square-root seed (about 20 bits, from the upper word) and two coupled Newton
-// steps on g ~ sqrt(x), h ~ 1/(2 sqrt(x)).  Straight-line code: the library
+// sqrt(x) for x >= 0 in double, to within an ulp or two: hardware reciprocal-
+// square-root seed (about 20 bits, from the upper word) and one third-order
+// step on it (fewer double-precision operations than two Newton steps: on a
+// power-capped part the arithmetic's energy, not its time, is what costs
+// bandwidth), times x.  Straight-line code: the library
 // routine's range checks and slow path are not needed here (x is a finite,
 // non-negative, never subnormal second moment).  The seed is taken of
 // x + 1e-300: every non-zero second moment is at least 1e-93 (the square of the
 // smallest fp32 denormal times 1 - beta2), so the addition returns x itself,
-// and for x = 0 it keeps the seed finite so that g = 0 * seed = 0 comes out
-// exactly.  For x = +Inf (a second moment that overflowed fp32) the result is
+// and for x = 0 it keeps the seed finite so that 0 * (refined seed) = 0 comes
+// out exactly.  For x = +Inf (a second moment that overflowed fp32) the result is
 // NaN (Inf * 0); the caller then forms the element again with IEEE operations.
 __device__ __forceinline__ double sqrt_nonneg(double x)
 {
     double y;
     const double xs = __dadd_rn(x, 1e-300);
     asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(xs));
-    double g = __dmul_rn(x, y);
-    double h = __dmul_rn(0.5, y);
-    double r = __fma_rn(-g, h, 0.5);
-    g = __fma_rn(g, r, g);
-    h = __fma_rn(h, r, h);
-    r = __fma_rn(-g, h, 0.5);
-    return __fma_rn(g, r, g);
+    // one third-order step: with e = 1 - x y^2 (about 2^-20 from the seed),
+    // 1/sqrt(x) = y (1 + e/2 + 3 e^2/8 + O(e^3)); the remainder is below 2^-58
+    const double a = __dmul_rn(x, y);
+    const double e = __fma_rn(-a, y, 1.0);
+    const double t = __dmul_rn(e, __fma_rn(e, 0.375, 0.5));
+    return __dmul_rn(x, __fma_rn(y, t, y));
 }
 
 // 1 / b for finite, normal b > 0, to within an ulp or two: reciprocal seed
-// (about 20 bits) and two Newton steps.
+// (about 20 bits) and one third-order step, 1/b = y (1 + e + e^2 + O(e^3)) with
+// e = 1 - b y.
 __device__ __forceinline__ double rcp_pos(double b)
 {
     double y;
     asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(b));
-    double e = __fma_rn(-b, y, 1.0);
-    y = __fma_rn(y, e, y);
-    e = __fma_rn(-b, y, 1.0);
-    return __fma_rn(y, e, y);
+    const double e = __fma_rn(-b, y, 1.0);
+    return __fma_rn(y, __fma_rn(e, e, e), y);
 }
 
 // One element, fast order.  Returns true when the new parameter came out below
