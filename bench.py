@@ -192,7 +192,7 @@ def run_sharded(args, w, torch, dist, rank, world, local_rank):
     n_local = shard.hi - shard.lo
     mine = W.Workload(name=f"{w.name}_shard{rank}", numel=[n_local], bucket_elems=w.bucket_elems,
                       sigma_g=w.sigma_g, seed=w.seed + 17 * rank, max_grad_norm=w.max_grad_norm,
-                      grad_dtype=w.grad_dtype)
+                      grad_dtype=w.grad_dtype, target_norm=w.target_norm)
     shard.local.load_state_stream(W.iter_initial_master(mine, device="cuda"))
     shard.local.cast_params(stream=stream)
     shard.local.load_grads_stream(W.iter_gradients(mine, 1, device="cuda"))

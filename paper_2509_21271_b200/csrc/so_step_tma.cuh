@@ -335,13 +335,12 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
             __syncwarp();
             const unsigned char *in = wbase + stage * L::kInStage;
             unsigned char *out = out_base + ostage * L::kOutStage;
-            // one row (4 elements per lane) at a time: keeps the register
-            // footprint small (the alternate 16-warp shape has 128 registers per thread)
-#pragma unroll 1
-            for (int r = 0; r < kChunkRows; ++r) {
-                const uint32_t off = r * kRowElems + lane * 4;     // element within the chunk
-                if (off >= len) break;
-                float gq[4], pq[4], mq[4], vq[4];
+            // Two rows (8 elements per lane) in flight at a time: the eight
+            // dependent chains of conversions, seeds and fp64 operations
+            // interleave, which is what hides their latency with only ten warps
+            // per SM when a power cap holds the SM clock down.
+            auto load_row = [&](uint32_t off, float (&gq)[4], float (&pq)[4], float (&mq)[4],
+                                float (&vq)[4]) {
                 const float4 p4 = *reinterpret_cast<const float4 *>(in + off * 4);
                 const float4 m4 = *reinterpret_cast<const float4 *>(in + L::kF32Bytes + off * 4);
                 const float4 v4 = *reinterpret_cast<const float4 *>(in + 2 * L::kF32Bytes + off * 4);
@@ -356,24 +355,19 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                     const float4 g4 = *reinterpret_cast<const float4 *>(in + 3 * L::kF32Bytes + off * 4);
                     gq[0] = g4.x; gq[1] = g4.y; gq[2] = g4.z; gq[3] = g4.w;
                 }
-                adamw_quad<!kSpec, grad_traits<GradT>::kUnscale>(
-                    gq, pq, mq, vq, k, scale, acc,
-                    [&]() {
-                        // the input stage is refilled only after this loop
-                        float4 g0;
-                        const float4 p0 = *reinterpret_cast<const float4 *>(in + off * 4);
-                        const float4 m0 = *reinterpret_cast<const float4 *>(in + L::kF32Bytes + off * 4);
-                        const float4 v0 = *reinterpret_cast<const float4 *>(in + 2 * L::kF32Bytes + off * 4);
-                        if constexpr (sizeof(GradT) == 2) {
-                            const uint2 h2 = *reinterpret_cast<const uint2 *>(in + 3 * L::kF32Bytes + off * 2);
-                            unpack2<GradT>(h2.x, g0.x, g0.y);
-                            unpack2<GradT>(h2.y, g0.z, g0.w);
-                        } else {
-                            g0 = *reinterpret_cast<const float4 *>(in + 3 * L::kF32Bytes + off * 4);
-                        }
-                        return adamw_exact_quad<!kSpec, grad_traits<GradT>::kUnscale>(g0, p0, m0, v0, k,
-                                                                                      scale);
-                    });
+            };
+            // the quad again in the textbook order, from its inputs in the stage
+            // (which is refilled only after the chunk)
+            auto redo_row = [&](uint32_t off) {
+                float g0[4], p0[4], m0[4], v0[4];
+                load_row(off, g0, p0, m0, v0);
+                return adamw_exact_quad<!kSpec, grad_traits<GradT>::kUnscale>(
+                    make_float4(g0[0], g0[1], g0[2], g0[3]), make_float4(p0[0], p0[1], p0[2], p0[3]),
+                    make_float4(m0[0], m0[1], m0[2], m0[3]), make_float4(v0[0], v0[1], v0[2], v0[3]), k,
+                    scale);
+            };
+            auto store_row = [&](uint32_t off, const float (&pq)[4], const float (&mq)[4],
+                                 const float (&vq)[4]) {
                 *reinterpret_cast<float4 *>(out + off * 4) = make_float4(pq[0], pq[1], pq[2], pq[3]);
                 *reinterpret_cast<float4 *>(out + L::kF32Bytes + off * 4) =
                     make_float4(mq[0], mq[1], mq[2], mq[3]);
@@ -381,6 +375,38 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                     make_float4(vq[0], vq[1], vq[2], vq[3]);
                 *reinterpret_cast<uint2 *>(out + 3 * L::kF32Bytes + off * 2) =
                     make_uint2(pack_lp(pq[0], pq[1], fp16), pack_lp(pq[2], pq[3], fp16));
+            };
+            constexpr int kAtOnce = 2;     // four at once spill (168 registers + 80 bytes of stack)
+            static_assert(kChunkRows % kAtOnce == 0, "rows are taken in groups");
+#pragma unroll 1
+            for (int r = 0; r < kChunkRows; r += kAtOnce) {
+                const uint32_t off0 = r * kRowElems + lane * 4;    // element within the chunk
+                if (off0 >= len) break;
+                float gq[kAtOnce][4], pq[kAtOnce][4], mq[kAtOnce][4], vq[kAtOnce][4];
+                if (off0 + (kAtOnce - 1) * kRowElems < len) {
+#pragma unroll
+                    for (int u = 0; u < kAtOnce; ++u)
+                        load_row(off0 + u * kRowElems, gq[u], pq[u], mq[u], vq[u]);
+                    // (the sums still take the rows in order: same order as ever)
+#pragma unroll
+                    for (int u = 0; u < kAtOnce; ++u)
+                        adamw_quad<!kSpec, grad_traits<GradT>::kUnscale>(
+                            gq[u], pq[u], mq[u], vq[u], k, scale, acc,
+                            [&]() { return redo_row(off0 + u * kRowElems); });
+#pragma unroll
+                    for (int u = 0; u < kAtOnce; ++u)
+                        store_row(off0 + u * kRowElems, pq[u], mq[u], vq[u]);
+                } else {
+                    // the ragged end of a chunk: row by row
+                    for (int u = 0; u < kAtOnce; ++u) {
+                        const uint32_t off = off0 + u * kRowElems;
+                        if (off >= len) break;
+                        load_row(off, gq[0], pq[0], mq[0], vq[0]);
+                        adamw_quad<!kSpec, grad_traits<GradT>::kUnscale>(
+                            gq[0], pq[0], mq[0], vq[0], k, scale, acc, [&]() { return redo_row(off); });
+                        store_row(off, pq[0], mq[0], vq[0]);
+                    }
+                }
             }
             fence_async_smem();        // generic writes -> visible to the async proxy
             // every lane is done with the input stage and has filled its part
