@@ -113,8 +113,10 @@ typedef struct {
 typedef struct {
     int64_t commits, skips, clip_resteps;      /* validated iterations by outcome    */
     int64_t kernel_launches;                   /* kernels this context has launched  */
-    int64_t elems_stepped, elems_checked, elems_cast;  /* work done by those kernels */
-    int64_t timeouts;                          /* iterations given up with SO_ERR_TIMEOUT */
+    int64_t elems_stepped, elems_checked, elems_cast;  /* work done by those kernels; what a
+                                                  verdict's follow-up launches did is added
+                                                  when the host collects that verdict        */
+    int64_t timeouts;                          /* iterations given up (SO_ERR_TIMEOUT, so_abandon_iteration) */
 } so_counters;
 
 /*
@@ -224,6 +226,10 @@ so_status so_grad_check(so_ctx *ctx, const so_hparams *hp, int32_t bucket, void 
  * Enqueues only; no synchronisation.  Calls for different buckets may go to
  * different streams and their kernels may overlap; at most 4096 step launches
  * of one context may be outstanding (enqueued and unfinished) at any time.
+ * While a validation begun with so_validate_begin is pending, the call opens
+ * the NEXT iteration: its kernels take the step index and the loss scale that
+ * follow from the pending verdict, read on the device (the first such launch
+ * also carries that verdict to the host).
  */
 so_status so_adam_step_speculative(so_ctx *ctx, const so_hparams *hp, int32_t bucket,
                                    void *stream);
@@ -320,9 +326,10 @@ so_status so_set_global_grad_stats(so_ctx *ctx, double global_sumsq, int32_t glo
 so_status so_abandon_iteration(so_ctx *ctx, void *stream);
 
 /*
- * so_cast_params -- fp32 master -> bf16 parameter copy, round to nearest even
- * (Section 4.5: the cast runs on the GPU).  bucket >= 0 or SO_ALL.  Only
- * between iterations (SO_ERR_STATE while buckets are covered).  Enqueues only.
+ * so_cast_params -- fp32 master -> low-precision parameter copy (bf16, or
+ * binary16 after so_param_dtype_config), round to nearest even (Section 4.5:
+ * the cast runs on the GPU).  bucket >= 0 or SO_ALL.  Only between iterations
+ * (SO_ERR_STATE while buckets are covered or a verdict is pending).  Enqueues only.
  */
 so_status so_cast_params(so_ctx *ctx, int32_t bucket, void *stream);
 

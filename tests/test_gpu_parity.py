@@ -96,6 +96,24 @@ def test_empty_model_on_the_device():
     assert res.decision == C and res.stats.norm == 0.0 and opt.step_count == 1
 
 
+def test_empty_model_binds_without_any_device_memory():
+    """An empty tensor list needs no arenas: all pointers may be NULL, bind
+    touches no device memory, and the iteration is a valid no-op."""
+    ctx, info = B.so_layout_init([], 1024)
+    assert info.n_buckets == 0
+    B.so_layout_bind(ctx, 0, 0, 0, 0, 0, 0)
+    hp = oracle.HParams()
+    stream = torch.cuda.current_stream()
+    B.so_adam_step_speculative(ctx, hp, B.SO_ALL, stream)
+    B.so_validate_begin(ctx, hp, stream)
+    assert B.so_validate_poll(ctx) is True
+    res = B.so_validate_commit_or_rollback(ctx, hp, stream)
+    assert res.decision == C and res.step_after == 1 and res.stats.norm == 0.0
+    B.so_cast_params(ctx, B.SO_ALL, stream)
+    assert B.so_get_counters(ctx).kernel_launches == 0
+    B.so_destroy(ctx)
+
+
 # ---------------------------------------------------------------------------
 # exactness of speculation (Section 4.4) and of the rollback
 # ---------------------------------------------------------------------------
