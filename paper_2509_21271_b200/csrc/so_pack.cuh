@@ -5,11 +5,12 @@
 // The flat parameter space [0, N) is cut into runs of 2048 elements dealt
 // round-robin to the warps of a persistent grid.  A lane moves groups of 16
 // bytes (8 two-byte or 4 four-byte elements).  A group that lies inside one
-// tensor and one bucket with both addresses 16-byte aligned is one 128-bit load
-// and one 128-bit store; any other group (a tensor or bucket boundary inside
-// it, an odd tensor start) is moved element by element.  Which tensor holds a
-// flat index is found by bisection over the tensors' flat offsets once per lane
-// and run, then by walking forward.
+// tensor and one bucket is one 128-bit load and one 128-bit store where the
+// addresses are 16-byte aligned (a tensor that starts at an odd element offset
+// is read or written element by element on its own side only); a group with a
+// tensor or bucket boundary inside it is moved element by element.  Which
+// tensor holds a flat index is found by bisection over the tensors' flat
+// offsets once per lane and run, then by walking forward.
 #pragma once
 
 #include "so_kernels.cuh"
@@ -33,7 +34,7 @@ __device__ __forceinline__ int32_t tensor_of(const PackTensor *t, int32_t n_tens
 }
 
 template <typename ElemT, bool kPack>
-__global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
+__global__ void __launch_bounds__(kThreads, 8) pack_kernel(const PackArgs a)
 {
     wait_for_prior_kernels();
     constexpr int kVec = 16 / (int)sizeof(ElemT);          // elements per 16-byte group
@@ -58,12 +59,29 @@ __global__ void __launch_bounds__(kThreads) pack_kernel(const PackArgs a)
             const int64_t in_bucket = f - bucket * a.bucket_elems;
             ElemT *slot = arena + bucket * a.stride + in_bucket;
             ElemT *own = static_cast<ElemT *>(t.ptr) + (f - t.flat_offset);
-            const bool whole = f + kVec <= t.flat_offset + t.numel &&
-                               in_bucket + kVec <= a.bucket_elems &&
-                               ((reinterpret_cast<uintptr_t>(slot) | reinterpret_cast<uintptr_t>(own)) & 15u) == 0;
-            if (whole) {
-                if (kPack) __stcs(reinterpret_cast<uint4 *>(slot), __ldcs(reinterpret_cast<const uint4 *>(own)));
-                else __stcs(reinterpret_cast<uint4 *>(own), __ldcs(reinterpret_cast<const uint4 *>(slot)));
+            const bool whole = f + kVec <= t.flat_offset + t.numel && in_bucket + kVec <= a.bucket_elems;
+            const bool slot_ok = (reinterpret_cast<uintptr_t>(slot) & 15u) == 0;
+            const bool own_ok = (reinterpret_cast<uintptr_t>(own) & 15u) == 0;
+            if (whole && (slot_ok || own_ok)) {
+                // the group lies in one tensor and one bucket: 128-bit access on
+                // every side whose address allows it, elements on the other
+                const ElemT *src = kPack ? own : slot;
+                ElemT *dst = kPack ? slot : own;
+                const bool src_ok = kPack ? own_ok : slot_ok;
+                const bool dst_ok = kPack ? slot_ok : own_ok;
+                union { uint4 q; ElemT e[kVec]; } g;
+                if (src_ok) {
+                    g.q = __ldcs(reinterpret_cast<const uint4 *>(src));
+                } else {
+#pragma unroll
+                    for (int k = 0; k < kVec; ++k) g.e[k] = __ldcs(src + k);
+                }
+                if (dst_ok) {
+                    __stcs(reinterpret_cast<uint4 *>(dst), g.q);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < kVec; ++k) __stcs(dst + k, g.e[k]);
+                }
             } else {
                 int32_t tj = ti;
                 for (int k = 0; k < kVec; ++k) {
