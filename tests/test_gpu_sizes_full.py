@@ -112,8 +112,9 @@ def test_sweep_one_bucket_per_combination(bucket_mi, grad_dtype):
 
 
 # ---------------------------------------------------------------------------
-# the recipes at their full number of steps (config 2 always; the longer ones,
-# about 50 minutes, on request)
+# the recipes at their full number of steps (config 2 and the 8-step recipe of
+# config 4 always; the 100-step recipe of config 3 and the long soaks, about
+# half an hour, on request)
 # ---------------------------------------------------------------------------
 
 full_length = pytest.mark.skipif(os.environ.get("SO_FULL_LENGTH") != "1",
@@ -179,7 +180,6 @@ def test_soak_long(dtype, steps):
     _soak(dtype, steps)
 
 
-@full_length
 def test_llama_8b_clip_and_nan_through_the_undo_window():
     """The 8 B-parameter workload with the clip active on every other step and
     a NaN on steps 4 and 8: re-steps write speculated buckets from their old
