@@ -354,6 +354,29 @@ so_status so_iteration_host(so_ctx *ctx, const so_hparams *hp, const void *host_
                             void *host_param_bf16, void *stream, so_step_result *out);
 
 /*
+ * so_iteration_host_pipelined / so_iteration_host_wait -- the same iteration
+ * without the wait at its end, so that consecutive iterations overlap on the
+ * link (Section 4.3's point, carried across the iteration boundary: the link is
+ * full duplex, and the parameters that can only leave after the verdict -- those
+ * of the buckets beyond the undo window, or all of them after a clip -- travel
+ * while the next iteration's gradients arrive).  The call returns once the
+ * verdict is known (it fills `out`) and every copy is enqueued; the next call's
+ * kernels wait on the device for the previous call's outgoing copies before they
+ * overwrite the parameter arena, its incoming copies do not.
+ * Until so_iteration_host_wait (or the next blocking call) has returned:
+ *   - host_param_bf16 of the previous call is still being written;
+ *   - host_grad of this call has been read completely only after this call's
+ *     own return (all its incoming copies precede its verdict), so a gradient
+ *     buffer may be refilled as soon as the call that was given it returns;
+ *   - any other work of the context must go to `stream` (it is ordered behind
+ *     the iteration's kernels there).
+ * so_iteration_host_wait waits for the outgoing copies and for `stream`.
+ */
+so_status so_iteration_host_pipelined(so_ctx *ctx, const so_hparams *hp, const void *host_grad,
+                                      void *host_param_bf16, void *stream, so_step_result *out);
+so_status so_iteration_host_wait(so_ctx *ctx, void *stream);
+
+/*
  * so_grad_check_static -- the gradient check for callers that cannot allocate.
  * (The paper has no counterpart: this is a packaging variant of so_grad_check,
  * not a step of its method.)

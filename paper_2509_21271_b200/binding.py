@@ -78,7 +78,8 @@ EXPORTS = ["so_layout_init", "so_layout_get_info", "so_layout_tensor", "so_layou
            "so_debug_set_spin_limit", "so_abandon_iteration",
            "so_grad_check", "so_adam_step_speculative", "so_validate_commit_or_rollback",
            "so_validate_begin", "so_validate_poll", "so_set_global_grad_stats",
-           "so_cast_params", "so_iteration_host", "so_grad_check_static",
+           "so_cast_params", "so_iteration_host", "so_iteration_host_pipelined",
+           "so_iteration_host_wait", "so_grad_check_static",
            "so_loss_scale_config", "so_get_loss_scale", "so_state_export", "so_state_import",
            "so_bucket_slot", "so_get_step", "so_set_step", "so_pending_buckets",
            "so_get_counters", "so_last_cuda_error", "so_strerror", "so_destroy",
@@ -115,6 +116,8 @@ def lib() -> C.CDLL:
         "so_set_global_grad_stats": [vp, dbl, i32],
         "so_cast_params": [vp, i32, vp],
         "so_iteration_host": [vp, P(so_hparams), vp, vp, vp, P(so_step_result)],
+        "so_iteration_host_pipelined": [vp, P(so_hparams), vp, vp, vp, P(so_step_result)],
+        "so_iteration_host_wait": [vp, vp],
         "so_grad_check_static": [vp, i64, i32, dbl, vp, vp],
         "so_loss_scale_config": [vp, dbl, dbl, dbl, i64],
         "so_get_loss_scale": [vp, P(dbl)],
@@ -281,6 +284,21 @@ def so_iteration_host(ctx, hp, host_grad: int, host_param_bf16: int, stream=None
     _ok(ctx, lib().so_iteration_host(ctx, C.byref(h), host_grad, host_param_bf16 or None,
                                      _stream(stream), C.byref(out)), "so_iteration_host")
     return out
+
+
+def so_iteration_host_pipelined(ctx, hp, host_grad: int, host_param_bf16: int,
+                                stream=None) -> so_step_result:
+    """Like so_iteration_host, without the wait at the end (see the header)."""
+    h = _hp(hp)
+    out = so_step_result()
+    _ok(ctx, lib().so_iteration_host_pipelined(ctx, C.byref(h), host_grad, host_param_bf16 or None,
+                                               _stream(stream), C.byref(out)),
+        "so_iteration_host_pipelined")
+    return out
+
+
+def so_iteration_host_wait(ctx, stream=None) -> None:
+    _ok(ctx, lib().so_iteration_host_wait(ctx, _stream(stream)), "so_iteration_host_wait")
 
 
 def so_grad_check_static(grad: int, n_elems: int, grad_dtype: int, max_grad_norm: float,

@@ -120,6 +120,7 @@ struct so_ctx {
     // ---- host-fed iteration: copy streams and ordering events (lazy) ----
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     std::vector<cudaEvent_t> events;
+    bool copies_in_flight = false;      // a pipelined call's outgoing parameters may still be travelling
 };
 
 namespace {
@@ -1204,27 +1205,53 @@ so_status so_cast_params(so_ctx *c, int32_t bucket, void *stream)
 }
 
 static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void *host_grad,
-                                     void *host_param_bf16, void *stream, so_step_result *out);
+                                     void *host_param_bf16, void *stream, so_step_result *out,
+                                     bool wait_at_end);
 
-so_status so_iteration_host(so_ctx *c, const so_hparams *hp, const void *host_grad,
-                            void *host_param_bf16, void *stream, so_step_result *out)
+static so_status iteration_host_checked(so_ctx *c, const so_hparams *hp, const void *host_grad,
+                                        void *host_param_bf16, void *stream, so_step_result *out,
+                                        bool wait_at_end)
 {
     if (!c) return SO_ERR_INVALID_ARG;
     if (!c->bound || c->cur.phase != kIdle || c->pending) return SO_ERR_STATE;
     if (!hparams_ok(hp) || (c->n_buckets > 0 && !host_grad)) return SO_ERR_INVALID_ARG;
     if (c->dry_run) return SO_ERR_UNSUPPORTED;
-    const so_status s = iteration_host_body(c, hp, host_grad, host_param_bf16, stream, out);
+    const so_status s = iteration_host_body(c, hp, host_grad, host_param_bf16, stream, out, wait_at_end);
     if (s != SO_OK && c->copy_in) {
         // leave no copy in flight from or into the caller's buffers
         cudaStreamSynchronize(c->copy_in);
         cudaStreamSynchronize(c->copy_out);
         cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+        c->copies_in_flight = false;
     }
     return s;
 }
 
+so_status so_iteration_host(so_ctx *c, const so_hparams *hp, const void *host_grad,
+                            void *host_param_bf16, void *stream, so_step_result *out)
+{
+    return iteration_host_checked(c, hp, host_grad, host_param_bf16, stream, out, true);
+}
+
+so_status so_iteration_host_pipelined(so_ctx *c, const so_hparams *hp, const void *host_grad,
+                                      void *host_param_bf16, void *stream, so_step_result *out)
+{
+    return iteration_host_checked(c, hp, host_grad, host_param_bf16, stream, out, false);
+}
+
+so_status so_iteration_host_wait(so_ctx *c, void *stream)
+{
+    if (!c) return SO_ERR_INVALID_ARG;
+    if (!c->copies_in_flight) return SO_OK;
+    cudaError_t e = cudaStreamSynchronize(c->copy_out);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    c->copies_in_flight = false;
+    return e == cudaSuccess ? SO_OK : cuda_fail(c, e);
+}
+
 static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void *host_grad,
-                                     void *host_param_bf16, void *stream, so_step_result *out)
+                                     void *host_param_bf16, void *stream, so_step_result *out,
+                                     bool wait_at_end)
 {
     cudaStream_t main = static_cast<cudaStream_t>(stream);
     cudaError_t e;
@@ -1234,7 +1261,7 @@ static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void
         e = cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking);
         if (e != cudaSuccess) return cuda_fail(c, e);
     }
-    while ((int32_t)c->events.size() < 2 * c->n_buckets + 1) {
+    while ((int32_t)c->events.size() < 2 * c->n_buckets + 2) {
         cudaEvent_t ev;
         e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
         if (e != cudaSuccess) return cuda_fail(c, e);
@@ -1245,12 +1272,22 @@ static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void
     char *hp_out = static_cast<char *>(host_param_bf16);
     char *dgrad = static_cast<char *>(c->grad);
     cudaEvent_t start = c->events[2 * c->n_buckets];
+    cudaEvent_t drained = c->events[2 * c->n_buckets + 1];
 
-    // the copy streams start after whatever the caller queued on `stream`
+    // The incoming copies start after whatever the caller queued on `stream`
+    // (which, after a pipelined call, ends with the kernels that read the
+    // previous gradients).  The outgoing stream may still be sending the
+    // previous call's parameters: this call's kernels overwrite the parameter
+    // arena, so `stream` waits for that, while the incoming copies do not --
+    // the previous parameters leave while the next gradients arrive.
     e = cudaEventRecord(start, main);
     if (e != cudaSuccess) return cuda_fail(c, e);
     if ((e = cudaStreamWaitEvent(c->copy_in, start, 0)) != cudaSuccess) return cuda_fail(c, e);
     if ((e = cudaStreamWaitEvent(c->copy_out, start, 0)) != cudaSuccess) return cuda_fail(c, e);
+    if (c->copies_in_flight) {
+        if ((e = cudaEventRecord(drained, c->copy_out)) != cudaSuccess) return cuda_fail(c, e);
+        if ((e = cudaStreamWaitEvent(main, drained, 0)) != cudaSuccess) return cuda_fail(c, e);
+    }
 
     for (int32_t b = 0; b < c->n_buckets; ++b) {
         const size_t n = (size_t)elems_of(c, b);
@@ -1276,6 +1313,7 @@ static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void
                                 c->param_lp + (size_t)b * (size_t)c->stride, n * 2,
                                 cudaMemcpyDeviceToHost, c->copy_out);
             if (e != cudaSuccess) return cuda_fail(c, e);
+            c->copies_in_flight = true;
         }
     }
     std::vector<uint8_t> was_speculated(c->cur.cover.begin(), c->cur.cover.end());
@@ -1295,12 +1333,16 @@ static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void
                                 c->param_lp + (size_t)b * (size_t)c->stride, n * 2,
                                 cudaMemcpyDeviceToHost, c->copy_out);
             if (e != cudaSuccess) return cuda_fail(c, e);
+            c->copies_in_flight = true;
         }
     }
-    e = cudaStreamSynchronize(c->copy_out);
-    if (e != cudaSuccess) return cuda_fail(c, e);
-    e = cudaStreamSynchronize(main);
-    if (e != cudaSuccess) return cuda_fail(c, e);
+    if (wait_at_end) {
+        e = cudaStreamSynchronize(c->copy_out);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        e = cudaStreamSynchronize(main);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        c->copies_in_flight = false;
+    }
     if (out) *out = res;
     return SO_OK;
 }

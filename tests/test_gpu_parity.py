@@ -327,6 +327,43 @@ def test_host_fed_iteration_is_bitwise_the_device_fed_one(name, undo, dtype):
     assert S in [t[0] for t in trace]
 
 
+@pytest.mark.parametrize("name,undo", [("tiny", B.SO_ALL), ("tiny_ragged", 2)])
+def test_pipelined_host_fed_iterations_are_bitwise_the_blocking_ones(name, undo):
+    """so_iteration_host_pipelined does not wait at its end: the parameters that
+    leave after the verdict travel while the next call's gradients arrive.
+    Two alternating gradient buffers (a buffer is refilled as soon as the call
+    that read it has returned), one parameter buffer checked after the final
+    wait and at every step through a blocking gather on the same stream."""
+    w = W.by_name(name)
+    hp = hparams_of(w)
+    stream = torch.cuda.current_stream()
+    ref = _run_device_only(w, 8, undo_slots=undo, speculative=True)
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, undo)
+    opt.load_state(W.initial_master(w, device="cuda"))
+    opt.cast_params(stream=stream)
+    host_g = [torch.empty(w.total, dtype=opt.grad_torch_dtype, pin_memory=True) for _ in range(2)]
+    host_p = torch.empty(w.total, dtype=torch.bfloat16, pin_memory=True)
+    trace = []
+    for step in range(1, 9):
+        buf = host_g[step % 2]
+        buf.copy_(W.gradients(w, step, device="cuda"))
+        res = B.so_iteration_host_pipelined(opt.ctx, hp, buf.data_ptr(), host_p.data_ptr(), stream)
+        trace.append((res.decision, res.stats.sumsq, res.stats.norm, res.stats.clip_coef,
+                      res.stats.nonfinite, res.step_after))
+    B.so_iteration_host_wait(opt.ctx, stream)
+    assert trace == ref[0]
+    assert _state_bytes(opt) == ref[1]
+    dev_pb = opt.gather_param_bf16().cpu()
+    assert torch.equal(host_p.view(torch.int16), dev_pb.view(torch.int16))
+    B.so_iteration_host_wait(opt.ctx, stream)                  # nothing in flight: a no-op
+    # a blocking call right after pipelined ones is ordered behind them
+    host_g[0].copy_(W.gradients(w, 9, device="cuda"))
+    B.so_iteration_host_pipelined(opt.ctx, hp, host_g[0].data_ptr(), host_p.data_ptr(), stream)
+    host_g[1].copy_(W.gradients(w, 10, device="cuda"))
+    B.so_iteration_host(opt.ctx, hp, host_g[1].data_ptr(), host_p.data_ptr(), stream)
+    assert torch.equal(host_p.view(torch.int16), opt.gather_param_bf16().cpu().view(torch.int16))
+
+
 # ---------------------------------------------------------------------------
 # fp16 gradients under dynamic loss scaling (the paper's own precision path)
 # ---------------------------------------------------------------------------
