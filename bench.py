@@ -243,6 +243,25 @@ def measure_link(torch, n_bytes: int = 1 << 30, repeats: int = 5):
             torch.cuda.synchronize()
             times.append(e0.elapsed_time(e1))
         best[name] = n_bytes / (min(times[1:]) * 1e-3)
+    # both directions at once (what overlapped iterations ask of the link): the
+    # rate each way while the other is busy, from the time both copies took
+    host2 = torch.empty(n_bytes, dtype=torch.uint8, pin_memory=True)
+    dev2 = torch.empty(n_bytes, dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    times = []
+    for _ in range(repeats + 1):
+        e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        e0.record(stream)
+        side.wait_event(e0)
+        dev.copy_(host, non_blocking=True)
+        with torch.cuda.stream(side):
+            host2.copy_(dev2, non_blocking=True)
+            e2.record(side)
+        stream.wait_event(e2)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    best["both"] = n_bytes / (min(times[1:]) * 1e-3)
     return best
 
 
@@ -739,7 +758,7 @@ def main():
                 B.so_iteration_host(opt.ctx, hp, host_g.data_ptr(), host_p.data_ptr(), stream)
             barrier()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            n_e2e = max(3, min(args.steps, 10)) if N < (1 << 31) else 4
+            n_e2e = max(3, min(args.steps, 10)) if N < (1 << 31) else 6
             e0.record(stream)
             for _ in range(n_e2e):
                 B.so_iteration_host_pipelined(opt.ctx, hp, host_g.data_ptr(), host_p.data_ptr(), stream)
@@ -822,8 +841,11 @@ def main():
                        # shorter than the slower direction's copy at the measured rate
                        "pinned_h2d_gbs": e2e["link"]["h2d"] / 1e9,
                        "pinned_d2h_gbs": e2e["link"]["d2h"] / 1e9,
+                       "pinned_each_way_when_both_gbs": e2e["link"]["both"] / 1e9,
                        "frac_of_link": max(e2e["h2d"] / e2e["link"]["h2d"],
-                                           e2e["d2h"] / e2e["link"]["d2h"]) / (e2e["ms"] * 1e-3)}
+                                           e2e["d2h"] / e2e["link"]["d2h"]) / (e2e["ms"] * 1e-3),
+                       "frac_of_link_both_ways": max(e2e["h2d"], e2e["d2h"]) / e2e["link"]["both"]
+                                                 / (e2e["ms"] * 1e-3)}
     elif e2e:
         line["e2e"] = e2e
     if args.overlap and world == 1:
