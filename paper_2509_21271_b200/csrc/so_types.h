@@ -175,6 +175,7 @@ struct PackTensor {
 };
 
 constexpr int kPackTileElems = 2048;      // flat elements one warp moves at a time
+constexpr int kPackRunsPerWarp = 4;       // such runs per warp of a pack / unpack block
 
 struct PackArgs {
     const PackTensor *tensors;            // device table, flat offsets ascending

@@ -1435,10 +1435,8 @@ so_status pack_or_unpack(so_ctx *c, const void *const *tensor_ptrs, bool pack, c
         a.bucket_elems = c->bucket_elems;
         a.stride = c->stride;
         const int64_t tiles = (c->total + kPackTileElems - 1) / kPackTileElems;
-        int64_t blocks = (tiles + kWarpsPerBlock - 1) / kWarpsPerBlock;
-        const int64_t cap = (int64_t)c->num_sms * 8;
-        if (blocks > cap) blocks = cap;
-        const unsigned grid = (unsigned)blocks;
+        const int64_t per_block = (int64_t)kWarpsPerBlock * kPackRunsPerWarp;
+        const unsigned grid = (unsigned)((tiles + per_block - 1) / per_block);
         if (esz == 4) {
             if (pack) e = launch_dependent(pack_kernel<uint32_t, true>, grid, kThreads, 0, stream, a);
             else e = launch_dependent(pack_kernel<uint32_t, false>, grid, kThreads, 0, stream, a);

@@ -824,3 +824,53 @@ def test_pack_and_unpack_match_the_per_tensor_copies(name, dtype):
         assert (buf[:lead] == 7.0).all() and (buf[lead + n:] == 7.0).all()     # nothing around it
         pos += n
     assert opt.guard_bands_intact()
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+@pytest.mark.parametrize("bucket", [100_000, 100_003])
+def test_pack_and_unpack_at_every_offset_from_the_16_byte_grid(dtype, bucket):
+    """Tensors that start 0, 1, ... 7 elements into their buffers (every offset
+    from the 16-byte grid the element size allows), long enough that whole runs
+    lie inside one tensor, against aligned and unaligned bucket starts."""
+    w = W.by_name("tiny")
+    w.numel = [50_000 + 37 * i for i in range(16)]
+    w.bucket_elems = bucket
+    w.grad_dtype = dtype
+    stream = torch.cuda.current_stream()
+    opt = BucketedAdamW(w.numel, w.bucket_elems, dtype, 0, guard_bands=True)
+    total = sum(w.numel)
+    gen = torch.Generator(device="cuda").manual_seed(11)
+    flat = torch.randn(total, device="cuda", generator=gen).to(opt.grad_torch_dtype)
+    tensors, pos = [], 0
+    for i, n in enumerate(w.numel):
+        buf = torch.empty(n + 8, dtype=flat.dtype, device="cuda")
+        t = buf[i % 8:i % 8 + n]
+        t.copy_(flat[pos:pos + n])
+        tensors.append(t)
+        pos += n
+    opt.pack_grads(tensors, stream)
+    torch.cuda.synchronize()
+    packed = opt.grad.clone()
+    opt.grad.zero_()
+    opt.load_grads(flat)
+    torch.cuda.synchronize()
+    assert torch.equal(packed.view(torch.uint8), opt.grad.view(torch.uint8))
+
+    master = torch.randn(total, device="cuda", generator=gen)
+    opt.load_state(master)
+    opt.cast_params(stream=stream)
+    want = opt.gather_param_bf16()
+    outs = []
+    for i, n in enumerate(w.numel):
+        lead = (3 * i + 1) % 8
+        buf = torch.full((n + 8,), 7.0, dtype=torch.bfloat16, device="cuda")
+        outs.append((buf, lead, buf[lead:lead + n]))
+    opt.unpack_params([t for _, _, t in outs], stream)
+    torch.cuda.synchronize()
+    pos = 0
+    for i, (buf, lead, t) in enumerate(outs):
+        n = w.numel[i]
+        assert torch.equal(t.view(torch.int16), want[pos:pos + n].view(torch.int16)), i
+        assert (buf[:lead] == 7.0).all() and (buf[lead + n:] == 7.0).all(), i
+        pos += n
+    assert opt.guard_bands_intact()
