@@ -758,7 +758,7 @@ def main():
                 B.so_iteration_host(opt.ctx, hp, host_g.data_ptr(), host_p.data_ptr(), stream)
             barrier()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            n_e2e = max(3, min(args.steps, 10)) if N < (1 << 31) else 6
+            n_e2e = max(3, min(args.steps, 10))
             e0.record(stream)
             for _ in range(n_e2e):
                 B.so_iteration_host_pipelined(opt.ctx, hp, host_g.data_ptr(), host_p.data_ptr(), stream)

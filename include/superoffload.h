@@ -362,7 +362,12 @@ so_status so_iteration_host(so_ctx *ctx, const so_hparams *hp, const void *host_
  * while the next iteration's gradients arrive).  The call returns once the
  * verdict is known (it fills `out`) and every copy is enqueued; the next call's
  * kernels wait on the device for the previous call's outgoing copies before they
- * overwrite the parameter arena, its incoming copies do not.
+ * overwrite the parameter arena, its incoming copies do not.  Directly after
+ * another pipelined call those incoming copies wait only for the library's own
+ * kernels that still read the gradient bucket they overwrite (none for a bucket
+ * that was speculated in a committed iteration: its last reader ran before the
+ * verdict), not for other work the caller put on `stream` in between -- such
+ * work must leave the gradient arena alone.
  * Until so_iteration_host_wait (or the next blocking call) has returned:
  *   - host_param_bf16 of the previous call is still being written;
  *   - host_grad of this call has been read completely only after this call's

@@ -121,6 +121,12 @@ struct so_ctx {
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     std::vector<cudaEvent_t> events;
     bool copies_in_flight = false;      // a pipelined call's outgoing parameters may still be travelling
+    // After a pipelined call, which gradient buckets its kernels are done with
+    // (everything that reads them ran before the verdict the call waited for)
+    // and an event behind the kernels that still read the others.
+    bool after_pipelined = false;
+    std::vector<uint8_t> grad_done;
+    cudaEvent_t grads_read = nullptr;
 };
 
 namespace {
@@ -638,17 +644,23 @@ void make_pending(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
 
 // Enqueue the end of the open iteration: scan what is uncovered, reduce and
 // decide on the device, follow up.  The iteration becomes the pending one.
-so_status begin_validation(so_ctx *c, const so_hparams &hp, cudaStream_t stream)
+// publish_now: the caller is about to wait for the verdict, so it is sent to the
+// host straight behind the reduction, ahead of the follow-up launches (which can
+// be the step of every bucket beyond the undo window): the host learns it
+// without waiting for them.
+so_status begin_validation(so_ctx *c, const so_hparams &hp, cudaStream_t stream, bool publish_now)
 {
     so_status s = scan_uncovered(c, stream);
     if (s != SO_OK) return s;
     s = launch_reduce(c, hp.max_grad_norm, /*decide=*/true, stream);
     if (s != SO_OK) return s;
+    if (publish_now && (s = publish_to_host(c, stream)) != SO_OK) return s;
     s = launch_follow_up(c, hp, stream);
     if (s != SO_OK) return s;
     make_pending(c, hp, stream);
     c->pend_known = false;
-    c->pend_published = false;      // the next step launch carries it, or whoever asks first sends it
+    // otherwise the next step launch carries it, or whoever asks first sends it
+    c->pend_published = publish_now && !c->dry_run;
     return SO_OK;
 }
 
@@ -1010,6 +1022,7 @@ so_status so_grad_check(so_ctx *c, const so_hparams *hp, int32_t bucket, void *s
                         so_grad_stats *out)
 {
     if (!c) return SO_ERR_INVALID_ARG;
+    c->after_pipelined = false;     // the gradient arena is in use outside the host-fed pipeline
     if (!c->bound) return SO_ERR_STATE;
     if (c->cur.phase == kChecked) return SO_ERR_STATE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1076,6 +1089,7 @@ so_status so_grad_check(so_ctx *c, const so_hparams *hp, int32_t bucket, void *s
 so_status so_adam_step_speculative(so_ctx *c, const so_hparams *hp, int32_t bucket, void *stream)
 {
     if (!c) return SO_ERR_INVALID_ARG;
+    c->after_pipelined = false;     // the gradient arena is in use outside the host-fed pipeline
     if (!c->bound) return SO_ERR_STATE;
     if (c->cur.phase == kChecked) return SO_ERR_STATE;
     so_status s = note_hparams(c->cur, hp);
@@ -1128,7 +1142,7 @@ so_status so_validate_commit_or_rollback(so_ctx *c, const so_hparams *hp, void *
         const Verdict v = verdict_of(c->stats.sumsq, c->stats.nonfinite, 0, hp->max_grad_norm, 0);
         s = begin_validation_known(c, *hp, v, st);
     } else {
-        s = begin_validation(c, *hp, st);
+        s = begin_validation(c, *hp, st, /*publish_now=*/true);
     }
     if (s != SO_OK) return s;
     return collect_validation(c, out);
@@ -1137,11 +1151,12 @@ so_status so_validate_commit_or_rollback(so_ctx *c, const so_hparams *hp, void *
 so_status so_validate_begin(so_ctx *c, const so_hparams *hp, void *stream)
 {
     if (!c) return SO_ERR_INVALID_ARG;
+    c->after_pipelined = false;     // the gradient arena is in use outside the host-fed pipeline
     if (!c->bound) return SO_ERR_STATE;
     if (c->pending || c->cur.phase == kChecked) return SO_ERR_STATE;
     const so_status s = note_hparams(c->cur, hp);
     if (s != SO_OK) return s;
-    return begin_validation(c, *hp, static_cast<cudaStream_t>(stream));
+    return begin_validation(c, *hp, static_cast<cudaStream_t>(stream), /*publish_now=*/false);
 }
 
 so_status so_abandon_iteration(so_ctx *c, void *stream)
@@ -1223,6 +1238,7 @@ static so_status iteration_host_checked(so_ctx *c, const so_hparams *hp, const v
         cudaStreamSynchronize(c->copy_out);
         cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
         c->copies_in_flight = false;
+        c->after_pipelined = false;
     }
     return s;
 }
@@ -1242,10 +1258,11 @@ so_status so_iteration_host_pipelined(so_ctx *c, const so_hparams *hp, const voi
 so_status so_iteration_host_wait(so_ctx *c, void *stream)
 {
     if (!c) return SO_ERR_INVALID_ARG;
-    if (!c->copies_in_flight) return SO_OK;
-    cudaError_t e = cudaStreamSynchronize(c->copy_out);
+    if (!c->copies_in_flight && !c->after_pipelined) return SO_OK;
+    cudaError_t e = c->copy_out ? cudaStreamSynchronize(c->copy_out) : cudaSuccess;
     if (e == cudaSuccess) e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
     c->copies_in_flight = false;
+    c->after_pipelined = false;
     return e == cudaSuccess ? SO_OK : cuda_fail(c, e);
 }
 
@@ -1280,10 +1297,19 @@ static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void
     // previous call's parameters: this call's kernels overwrite the parameter
     // arena, so `stream` waits for that, while the incoming copies do not --
     // the previous parameters leave while the next gradients arrive.
+    // Straight after another pipelined call the incoming copies wait for less:
+    // that call returned with its verdict, so every kernel that ran before the
+    // verdict is over, and a bucket whose gradient only those kernels read (a
+    // speculated bucket of a committed iteration, every bucket of a skipped
+    // one) can be overwritten at once; the others wait for the follow-up step
+    // that still reads them, not for the whole stream.
+    const bool early = c->after_pipelined;
+    c->after_pipelined = false;
     e = cudaEventRecord(start, main);
     if (e != cudaSuccess) return cuda_fail(c, e);
-    if ((e = cudaStreamWaitEvent(c->copy_in, start, 0)) != cudaSuccess) return cuda_fail(c, e);
+    if (!early && (e = cudaStreamWaitEvent(c->copy_in, start, 0)) != cudaSuccess) return cuda_fail(c, e);
     if ((e = cudaStreamWaitEvent(c->copy_out, start, 0)) != cudaSuccess) return cuda_fail(c, e);
+    bool waited_for_readers = !early;
     if (c->copies_in_flight) {
         if ((e = cudaEventRecord(drained, c->copy_out)) != cudaSuccess) return cuda_fail(c, e);
         if ((e = cudaStreamWaitEvent(main, drained, 0)) != cudaSuccess) return cuda_fail(c, e);
@@ -1291,6 +1317,10 @@ static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void
 
     for (int32_t b = 0; b < c->n_buckets; ++b) {
         const size_t n = (size_t)elems_of(c, b);
+        if (!waited_for_readers && !c->grad_done[b]) {
+            if ((e = cudaStreamWaitEvent(c->copy_in, c->grads_read, 0)) != cudaSuccess) return cuda_fail(c, e);
+            waited_for_readers = true;
+        }
         e = cudaMemcpyAsync(dgrad + (size_t)b * (size_t)c->stride * gsz,
                             hg + (size_t)b * (size_t)c->bucket_elems * gsz, n * gsz,
                             cudaMemcpyHostToDevice, c->copy_in);
@@ -1342,6 +1372,20 @@ static so_status iteration_host_body(so_ctx *c, const so_hparams *hp, const void
         e = cudaStreamSynchronize(main);
         if (e != cudaSuccess) return cuda_fail(c, e);
         c->copies_in_flight = false;
+    } else {
+        // what the next pipelined call may overwrite without waiting
+        if (!c->grads_read) {
+            e = cudaEventCreateWithFlags(&c->grads_read, cudaEventDisableTiming);
+            if (e != cudaSuccess) return cuda_fail(c, e);
+        }
+        if ((e = cudaEventRecord(c->grads_read, main)) != cudaSuccess) return cuda_fail(c, e);
+        c->grad_done.assign((size_t)c->n_buckets, 0);
+        for (int32_t b = 0; b < c->n_buckets; ++b) {
+            const bool speculated = was_speculated[b] == kSpeculated;
+            c->grad_done[b] = res.decision == SO_DECISION_SKIP ||
+                              (res.decision == SO_DECISION_COMMIT && speculated);
+        }
+        c->after_pipelined = true;
     }
     if (out) *out = res;
     return SO_OK;
@@ -1457,6 +1501,7 @@ so_status so_layout_pack_grads(so_ctx *c, const void *const *tensor_grads, void 
     if (!c) return SO_ERR_INVALID_ARG;
     if (!c->bound) return SO_ERR_STATE;
     if (c->cur.phase != kIdle) return SO_ERR_STATE;         // its gradients are in use
+    c->after_pipelined = false;
     return pack_or_unpack(c, tensor_grads, /*pack=*/true, static_cast<cudaStream_t>(stream));
 }
 
@@ -1545,6 +1590,7 @@ void so_destroy(so_ctx *c)
     if (!c) return;
     for (cudaEvent_t ev : c->events) cudaEventDestroy(ev);
     if (c->reduce_done) cudaEventDestroy(c->reduce_done);
+    if (c->grads_read) cudaEventDestroy(c->grads_read);
     if (c->copy_in) cudaStreamDestroy(c->copy_in);
     if (c->copy_out) cudaStreamDestroy(c->copy_out);
     if (c->h_ptr_stage) cudaFreeHost(c->h_ptr_stage);

@@ -327,6 +327,40 @@ def test_host_fed_iteration_is_bitwise_the_device_fed_one(name, undo, dtype):
     assert S in [t[0] for t in trace]
 
 
+def test_pipelined_host_fed_iterations_overwrite_no_gradient_still_in_use():
+    """Copies long enough (50 MB per bucket) that an incoming gradient which
+    started too early would land under a kernel still reading the bucket: five
+    buckets, two of them speculated, and a commit, a clip, a skip, a clip and a
+    commit in a row, so that the next call follows every kind of verdict (after
+    a commit the speculated buckets may be overwritten at once, after a skip all
+    of them, after a clip none before the re-step has run)."""
+    w = W.by_name("gpt2_small")
+    w.max_grad_norm = 1.0
+    w.target_norm = lambda step: 0.5 if step % 2 == 1 else 3.0
+    w.faults = (W.Fault(step=3, flat_index=3 * w.bucket_elems + 12345, kind="inf"),)
+    hp = hparams_of(w)
+    stream = torch.cuda.current_stream()
+    ref = _run_device_only(w, 5, undo_slots=2, speculative=True)
+    C, S, R = B.SO_DECISION_COMMIT, B.SO_DECISION_SKIP, B.SO_DECISION_CLIP_RESTEP
+    assert [t[0] for t in ref[0]] == [C, R, S, R, C]
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, 2)
+    opt.load_state(W.initial_master(w, device="cuda"))
+    opt.cast_params(stream=stream)
+    host_g = [torch.empty(w.total, dtype=opt.grad_torch_dtype, pin_memory=True) for _ in range(2)]
+    host_p = torch.empty(w.total, dtype=torch.bfloat16, pin_memory=True)
+    trace = []
+    for step in range(1, 6):
+        buf = host_g[step % 2]
+        buf.copy_(W.gradients(w, step, device="cuda"))
+        res = B.so_iteration_host_pipelined(opt.ctx, hp, buf.data_ptr(), host_p.data_ptr(), stream)
+        trace.append((res.decision, res.stats.sumsq, res.stats.norm, res.stats.clip_coef,
+                      res.stats.nonfinite, res.step_after))
+    B.so_iteration_host_wait(opt.ctx, stream)
+    assert trace == ref[0]
+    assert _state_bytes(opt) == ref[1]
+    assert torch.equal(host_p.view(torch.int16), opt.gather_param_bf16().cpu().view(torch.int16))
+
+
 @pytest.mark.parametrize("name,undo", [("tiny", B.SO_ALL), ("tiny_ragged", 2)])
 def test_pipelined_host_fed_iterations_are_bitwise_the_blocking_ones(name, undo):
     """so_iteration_host_pipelined does not wait at its end: the parameters that
