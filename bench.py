@@ -339,6 +339,72 @@ def run_placement(args, torch):
                                  "gemm_flops": gemm, "gemm_kind": gemm_kind}}))
 
 
+def run_pack(args, torch):
+    """`--pack`: time the one-launch flattening (`so_layout_pack_grads`,
+    `so_layout_unpack_params`) over the workload's tensor list, each tensor in a
+    buffer of its own, against the per-tensor copies it replaces (one JSON
+    line; bytes moved = 2 x element size x N per call)."""
+    from paper_2509_21271_b200 import workloads as W
+    from paper_2509_21271_b200.optimizer import BucketedAdamW
+
+    w = W.by_name("llama_1b" if args.workload == DEFAULT_WORKLOAD else args.workload)
+    stream = torch.cuda.current_stream()
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            peak, peak_kind = float(json.load(fh)["hbm_gbs"]), "of measured"
+    except Exception:
+        peak, peak_kind = 6650.0, "of fallback"
+    rows = []
+    for off_grid in (False, True):
+        opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, 0)
+        esz = opt.grad.element_size()
+        grads, params = [], []
+        for i, n in enumerate(w.numel):
+            lead = (i % 2) * 3 if off_grid else 0          # every other tensor 3 elements off the 16-byte grid
+            grads.append(torch.zeros(n + 8, dtype=opt.grad_torch_dtype, device="cuda")[lead:lead + n])
+            params.append(torch.zeros(n + 8, dtype=torch.bfloat16, device="cuda")[lead:lead + n])
+        row = {"tensors_off_the_16_byte_grid": off_grid}
+        for what, fn, bytes_moved in (("pack", lambda: opt.pack_grads(grads, stream), 2 * esz * w.total),
+                                      ("unpack", lambda: opt.unpack_params(params, stream), 4 * w.total)):
+            for _ in range(max(3, args.warmup)):
+                fn()
+            torch.cuda.synchronize()
+            times = []
+            for _ in range(max(5, args.steps)):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                fn()
+                e1.record(stream)
+                torch.cuda.synchronize()
+                times.append(e0.elapsed_time(e1))
+            times.sort()
+            med = times[len(times) // 2]
+            row[what] = {"ms_median": med, "gbs": bytes_moved / med / 1e6,
+                         "frac": bytes_moved / med / 1e6 / peak}
+
+        def per_tensor_copies():
+            pos = 0
+            for t in grads:
+                opt._scatter(opt.grad, pos, t)
+                pos += t.numel()
+        for _ in range(2):
+            per_tensor_copies()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        per_tensor_copies()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        row["per_tensor_copies_ms"] = e0.elapsed_time(e1)
+        rows.append(row)
+        opt.close()
+        del grads, params
+        torch.cuda.empty_cache()
+    print(json.dumps({"pack": rows, "workload": w.name, "tensors": len(w.numel), "params": w.total,
+                      "peak_gbs": peak, "peak_kind": peak_kind,
+                      "timing": "CUDA events around each call (pointer upload and launch included)"}))
+
+
 def _hparams(w, oracle_mod=None):
     from paper_2509_21271_b200.binding import so_hparams
     return so_hparams(w.lr, w.beta1, w.beta2, w.eps, w.weight_decay, w.max_grad_norm)
@@ -557,6 +623,8 @@ def main():
     ap.add_argument("--placement", action="store_true",
                     help="measure this box's rates (fused step, pinned copies, all-cores oracle) and "
                          "print what the paper's placement models (Eq. 1-5) make of them")
+    ap.add_argument("--pack", action="store_true",
+                    help="time the one-launch pack / unpack between per-tensor buffers and the arenas")
     ap.add_argument("--sharded", action="store_true",
                     help="shard the optimizer states by bucket ranges over the ranks (strong "
                          "scaling, one small all-reduce per iteration) instead of running replicas")
@@ -597,9 +665,9 @@ def main():
     if dist is not None:
         dist.barrier()
 
-    if args.placement:
+    if args.placement or args.pack:
         if rank == 0:
-            run_placement(args, torch)
+            (run_placement if args.placement else run_pack)(args, torch)
         if dist is not None:
             dist.destroy_process_group()
         return
