@@ -183,9 +183,11 @@ so_status so_param_dtype_config(so_ctx *ctx, int32_t param_dtype);
  * Tensors may start at any element alignment and straddle buckets; interior
  * runs move as 128-bit accesses, ragged heads and tails element by element.
  * Pack only between iterations (SO_ERR_STATE once a bucket is covered); unpack
- * at any time, ordered on `stream` like any other work.  Enqueues only (a
- * second call on the same context first waits for `stream`, because the
- * pointer list is staged in one pinned buffer).
+ * at any time, ordered on `stream` like any other work.  Enqueues only (the
+ * pointer list is staged in one pinned buffer and one device table: a second
+ * call on the same context first waits for the previous call's upload of the
+ * list, a few microseconds of copy, and calls that go to different streams
+ * must be ordered by the caller).
  */
 so_status so_layout_pack_grads(so_ctx *ctx, const void *const *tensor_grads, void *stream);
 so_status so_layout_unpack_params(so_ctx *ctx, void *const *tensor_params, void *stream);

@@ -85,6 +85,7 @@ struct so_ctx {
     int32_t *d_slot_of = nullptr, *d_free_slot = nullptr, *d_spec_idx = nullptr;
     PackTensor *d_tensors = nullptr;    // per-tensor (pointer, flat offset, numel) for pack / unpack
     uint64_t *h_ptr_stage = nullptr;    // pinned staging of a tensor pointer list
+    cudaEvent_t ptrs_uploaded = nullptr;    // behind the latest upload from it
     int64_t segs_per_slot = 1;
     uint32_t launch_seq = 0;            // picks the counter pair of each pipeline launch
     int step_variant = 0;               // 0: bulk-copy pipeline, 1: register path
@@ -1460,16 +1461,19 @@ so_status pack_or_unpack(so_ctx *c, const void *const *tensor_ptrs, bool pack, c
         if (!c->h_ptr_stage) {
             e = cudaHostAlloc(reinterpret_cast<void **>(&c->h_ptr_stage), nt * sizeof(uint64_t),
                               cudaHostAllocDefault);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ptrs_uploaded, cudaEventDisableTiming);
             if (e != cudaSuccess) return cuda_fail(c, e);
         } else {
             // the staging buffer may still feed the previous call's upload
-            e = cudaStreamSynchronize(stream);
+            // (only that copy is waited for, not the stream)
+            e = cudaEventSynchronize(c->ptrs_uploaded);
             if (e != cudaSuccess) return cuda_fail(c, e);
         }
         for (size_t i = 0; i < nt; ++i) c->h_ptr_stage[i] = reinterpret_cast<uint64_t>(tensor_ptrs[i]);
         // the pointer is the first member of each table entry
         e = cudaMemcpy2DAsync(c->d_tensors, sizeof(PackTensor), c->h_ptr_stage, sizeof(uint64_t),
                               sizeof(uint64_t), nt, cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess) e = cudaEventRecord(c->ptrs_uploaded, stream);
         if (e != cudaSuccess) return cuda_fail(c, e);
         PackArgs a;
         a.tensors = c->d_tensors;
@@ -1591,6 +1595,7 @@ void so_destroy(so_ctx *c)
     for (cudaEvent_t ev : c->events) cudaEventDestroy(ev);
     if (c->reduce_done) cudaEventDestroy(c->reduce_done);
     if (c->grads_read) cudaEventDestroy(c->grads_read);
+    if (c->ptrs_uploaded) cudaEventDestroy(c->ptrs_uploaded);
     if (c->copy_in) cudaStreamDestroy(c->copy_in);
     if (c->copy_out) cudaStreamDestroy(c->copy_out);
     if (c->h_ptr_stage) cudaFreeHost(c->h_ptr_stage);
