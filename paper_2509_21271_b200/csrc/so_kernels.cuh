@@ -268,25 +268,29 @@ __device__ __forceinline__ double warp_fold(double x)
 // square-root seed (about 20 bits, from the upper word) and one third-order
 // step on it (fewer double-precision operations than two Newton steps: on a
 // power-capped part the arithmetic's energy, not its time, is what costs
-// bandwidth), times x.  Straight-line code: the library
+// bandwidth), applied to x times the seed.  Straight-line code: the library
 // routine's range checks and slow path are not needed here (x is a finite,
 // non-negative, never subnormal second moment).  The seed is taken of
 // x + 1e-300: every non-zero second moment is at least 1e-93 (the square of the
 // smallest fp32 denormal times 1 - beta2), so the addition returns x itself,
 // and for x = 0 it keeps the seed finite so that 0 * (refined seed) = 0 comes
-// out exactly.  For x = +Inf (a second moment that overflowed fp32) the result is
-// NaN (Inf * 0); the caller then forms the element again with IEEE operations.
+// out exactly.  (Flooring the upper word with an integer maximum instead of the
+// addition measured the same.)  For x = +Inf (a second moment that overflowed
+// fp32) the result is NaN (Inf * 0); the caller then forms the element again
+// with IEEE operations.
 __device__ __forceinline__ double sqrt_nonneg(double x)
 {
     double y;
     const double xs = __dadd_rn(x, 1e-300);
     asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(xs));
     // one third-order step: with e = 1 - x y^2 (about 2^-20 from the seed),
-    // 1/sqrt(x) = y (1 + e/2 + 3 e^2/8 + O(e^3)); the remainder is below 2^-58
+    // sqrt(x) = x y (1 + e/2 + 3 e^2/8 + O(e^3)); the remainder is below 2^-58.
+    // a = x y is sqrt(x) to the seed's accuracy already and the correction is
+    // applied to it (the rounding of a enters e and is half taken out again).
     const double a = __dmul_rn(x, y);
     const double e = __fma_rn(-a, y, 1.0);
     const double t = __dmul_rn(e, __fma_rn(e, 0.375, 0.5));
-    return __dmul_rn(x, __fma_rn(y, t, y));
+    return __fma_rn(a, t, a);
 }
 
 // 1 / b for finite, normal b > 0, to within an ulp or two: reciprocal seed
@@ -321,8 +325,11 @@ __device__ __forceinline__ bool adamw_element(float g, float &p, float &m, float
     // negated >=, so that a NaN here (a second moment that reached +Inf makes the
     // straight-line square root produce one) also takes the textbook order,
     // whose IEEE operations handle infinities
-    const bool cancelled = !(fabs(p64) >= __dmul_rn(fabs((double)p), 0x1p-16));
-    p = __double2float_rn(p64);
+    // (the comparison is made on the rounded result, in single precision: the
+    // threshold is a margin, not a boundary that has to be exact)
+    const float p_new = __double2float_rn(p64);
+    const bool cancelled = !(fabsf(p_new) >= __fmul_rn(fabsf(p), 0x1p-16f));
+    p = p_new;
     m = __double2float_rn(m64);
     v = __double2float_rn(v64);
     return cancelled;
