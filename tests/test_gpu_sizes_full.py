@@ -111,6 +111,22 @@ def test_sweep_one_bucket_per_combination(bucket_mi, grad_dtype):
     del opt
 
 
+def test_largest_bucket_the_library_accepts():
+    """bucket_elems = 2^30, the stated maximum: byte offsets inside a slot reach
+    2^32, tile counts 2^20 per slot.  Two buckets (the second partial, ending
+    off every grid), one undo slot: the first bucket is stepped speculatively,
+    the second scanned and stepped in place; both compared in full, with a clip."""
+    w = W.Workload(name="bucket_2p30", numel=[(1 << 30) + (3 << 20) + 5], bucket_elems=1 << 30,
+                   sigma_g=1e-3, steps=2, max_grad_norm=1.0,
+                   target_norm=lambda step: 0.5 if step == 1 else 3.0)
+    rep, opt = run_sampled(w, steps=2, pick_buckets=lambda s: [0, 1], undo_slots=1,
+                           expect_decisions=[C, R])
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+    write_report(w.name, rep, {"undo_slots": 1})
+    opt.close()
+    del opt
+
+
 # ---------------------------------------------------------------------------
 # the recipes at their full number of steps (config 2 and the 8-step recipe of
 # config 4 always; the 100-step recipe of config 3 and the long soaks, about
