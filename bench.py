@@ -164,6 +164,16 @@ def max_over_ranks(values, device):
     return [float(x) for x in t]
 
 
+def all_ranks_ok(ok: bool, device) -> bool:
+    """True only if `ok` holds on every rank of the default process group (a
+    leg with barriers inside must be entered by all ranks or by none)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([1.0 if ok else 0.0], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MIN)
+    return bool(t.item() == 1.0)
+
+
 def whole_job_value(world: int, params_per_replica: int, ms_per_step: float) -> float:
     """Replicas only: every rank steps its own copy of the workload, so the
     job's throughput is world x params over the slowest rank's step time."""
@@ -813,6 +823,9 @@ def main():
             host_g = host_p = None
             e2e = {"unavailable": f"could not pin {N * (gsz + 2)} bytes of host memory: "
                                   f"{str(exc).splitlines()[0][:120]}"}
+        if dist is not None and not all_ranks_ok(host_g is not None, "cuda") and host_g is not None:
+            host_g = host_p = None            # another rank could not pin its buffers: no rank runs the leg
+            e2e = {"unavailable": "a rank could not pin its host buffers"}
         if host_g is not None:
             for start, piece in W.iter_gradients(w, 1, device="cuda", loss_scale=w.loss_scale):
                 host_g[start:start + piece.numel()].copy_(piece)

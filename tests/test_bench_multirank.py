@@ -22,6 +22,9 @@ def _worker(rank, world, port, q):
     dist.init_process_group("gloo", rank=rank, world_size=world)
     mine = [10.0 + rank, 5.0 - rank]               # rank 1 is slower on the first timer
     got = bench.max_over_ranks(mine, "cpu")
+    # a leg is entered only if every rank can (rank 1 cannot here)
+    got.append(bench.all_ranks_ok(rank == 0, "cpu"))
+    got.append(bench.all_ranks_ok(True, "cpu"))
     dist.barrier()
     q.put((rank, got))
     dist.destroy_process_group()
@@ -39,7 +42,7 @@ def test_max_over_ranks_and_whole_job_value_with_two_gloo_ranks():
     for p in procs:
         p.join(timeout=60)
         assert p.exitcode == 0
-    assert results[0] == results[1] == [11.0, 5.0]
+    assert results[0] == results[1] == [11.0, 5.0, False, True]
     # two replicas of 1e9 parameters at 11 ms per step
     assert bench.whole_job_value(2, 10 ** 9, 11.0) == 2 * 10 ** 9 / 11e-3
 
