@@ -643,7 +643,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--step-variant", type=int, default=0,
-                    help="0: bulk-copy pipeline (default), 1: register-only step kernel")
+                    help="0: chosen by launch size (default), 1: register-only step kernel, "
+                         "2: bulk-copy pipeline")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -894,7 +895,9 @@ def main():
                               + ("at once" if (args.sync_verdict or args.order == "ste")
                                  else "one iteration late"),
                    "launch_mode": "per_bucket" if args.per_bucket else "batched",
-                   "step_kernel": "bulk_copy_pipeline" if args.step_variant == 0 else "registers",
+                   "step_kernel": {0: "by launch size: bulk-copy pipeline, register kernel for launches "
+                                       "of at most 3 Mi elements",
+                                    1: "registers", 2: "bulk_copy_pipeline"}[args.step_variant],
                    "parallelism": "replicas" if world > 1 else "single",
                    "l2": f"working set {16 * N / 1e6:.0f} MB resident + undo slots, "
                          "larger than the 126 MB L2; no flush"},

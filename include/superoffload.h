@@ -490,10 +490,13 @@ so_status so_debug_set_dry_run(so_ctx *ctx, int32_t on);
 so_status so_debug_set_bucket_stats(so_ctx *ctx, int32_t bucket, double sumsq,
                                     int32_t nonfinite);
 
-/* Which implementation of the fused step runs: 0 (default) stages bulk copies
- * through shared memory, 1 keeps everything in registers.  Both produce the
- * same bits; the switch exists for measurements and for testing them against
- * each other. */
+/* Which implementation of the fused step runs.  There are two kernels with the
+ * same results bit for bit: one stages bulk copies through shared memory (the
+ * fast one on anything large), one keeps everything in registers (lower fixed
+ * cost per launch).  0 (default): by launch size -- the register kernel for
+ * launches of at most 3 Mi elements, the pipeline otherwise; 1: always the
+ * register kernel; 2: always the pipeline.  1 and 2 exist for measurements and
+ * for testing the two against each other. */
 so_status so_debug_set_step_variant(so_ctx *ctx, int32_t variant);
 
 /* How many times the bulk-copy step kernel polls for a chunk's loads before it

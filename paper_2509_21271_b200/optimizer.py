@@ -22,15 +22,22 @@ class BucketedAdamW:
     """One optimizer context over a tensor list flattened into buckets."""
 
     GUARD = 4096            # bytes of sentinel before and after every arena
+    # step kernel when the constructor is not told: 0 = chosen by launch size
+    # (see so_debug_set_step_variant); the GPU tests set 2 so that the small
+    # cases they run still go through the bulk-copy pipeline
+    DEFAULT_STEP_VARIANT = 0
 
     def __init__(self, numel: Sequence[int], bucket_elems: int, grad_dtype: str = "bf16",
                  undo_slots: int = B.SO_ALL, device: str = "cuda", guard_bands: bool = False,
-                 step_variant: int = 0, param_dtype: str = "bf16"):
+                 step_variant: Optional[int] = None, param_dtype: str = "bf16"):
         self.device = torch.device(device)
         gd = {"bf16": B.SO_GRAD_BF16, "fp32": B.SO_GRAD_FP32, "fp16": B.SO_GRAD_FP16}[grad_dtype]
         self.ctx, self.info = B.so_layout_init(list(numel), bucket_elems, gd, undo_slots)
+        if step_variant is None:
+            step_variant = self.DEFAULT_STEP_VARIANT
         if step_variant:
             B.so_debug_set_step_variant(self.ctx, step_variant)
+        self.step_variant = step_variant
         self.grad_torch_dtype = {B.SO_GRAD_BF16: torch.bfloat16, B.SO_GRAD_FP32: torch.float32,
                                  B.SO_GRAD_FP16: torch.float16}[gd]
         self.guard_bands = guard_bands

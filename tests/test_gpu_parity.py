@@ -65,6 +65,39 @@ def test_register_variant_of_the_step_lockstep(name):
     assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
 
 
+@pytest.mark.parametrize("name", ["tiny", "tiny_ragged"])
+def test_step_kernel_chosen_by_launch_size_lockstep(name):
+    """The library's default: launches of at most 3 Mi elements take the register
+    kernel (every launch of these small cases)."""
+    rep, _ = run_lockstep(W.by_name(name), steps=8, step_variant=0)
+    assert rep.decisions[6] == S
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+
+
+def test_both_step_kernels_in_one_iteration_lockstep():
+    """Buckets stepped one by one under the library's choice of kernel: two
+    8 Mi-element buckets go through the bulk-copy pipeline, the last bucket
+    (1 Mi + 77 elements) through the register kernel; one undo slot short, so
+    one bucket is scanned and stepped in place; clip on the second step."""
+    w = W.by_name("tiny")
+    w.numel = [5 << 20, (12 << 20) + 77]
+    w.bucket_elems = 8 << 20
+    w.faults = ()
+    w.target_norm = lambda step: 0.5 if step % 2 == 1 else 3.0
+
+    def drive(opt, hp, stream, step):
+        for b in (2, 0, 1):
+            try:
+                opt.step_speculative(hp, b, stream)
+            except B.SuperOffloadError as e:
+                assert e.status == B.SO_ERR_UNDO_EXHAUSTED
+        return opt.validate(hp, stream)
+
+    rep, _ = run_lockstep(w, steps=3, undo_slots=2, step_variant=0, drive=drive)
+    assert rep.decisions == [C, R, C]
+    assert rep.n_diff["m"] == 0 and rep.n_diff["v"] == 0
+
+
 def test_tiny_without_clipping_commits():
     w = W.tiny()
     w.max_grad_norm = 0.0
@@ -118,7 +151,7 @@ def test_empty_model_binds_without_any_device_memory():
 # exactness of speculation (Section 4.4) and of the rollback
 # ---------------------------------------------------------------------------
 
-def _run_device_only(w, steps, undo_slots, speculative, bucket_order=None, step_variant=0):
+def _run_device_only(w, steps, undo_slots, speculative, bucket_order=None, step_variant=None):
     hp = hparams_of(w)
     stream = torch.cuda.current_stream()
     opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, undo_slots,
@@ -155,8 +188,10 @@ def test_speculative_flow_is_bitwise_the_check_first_flow(name):
     shuffled = _run_device_only(w, 9, undo_slots=3, speculative=True,
                                 bucket_order=[3, 0, 2, 1] if name == "tiny" else [4, 1, 0, 3, 2])
     registers = _run_device_only(w, 9, undo_slots=B.SO_ALL, speculative=True, step_variant=1)
-    assert ref[0] == full[0] == windowed[0] == shuffled[0] == registers[0]
-    assert ref[1] == full[1] == windowed[1] == shuffled[1] == registers[1]
+    # the kernel chosen by launch size (these launches are small: the register kernel)
+    by_size = _run_device_only(w, 9, undo_slots=2, speculative=True, step_variant=0)
+    assert ref[0] == full[0] == windowed[0] == shuffled[0] == registers[0] == by_size[0]
+    assert ref[1] == full[1] == windowed[1] == shuffled[1] == registers[1] == by_size[1]
 
 
 def test_repeat_runs_are_bitwise_identical():
@@ -587,7 +622,7 @@ def test_cancelling_update_stays_within_tolerance(t0, clip, dtype, undo):
     p0 = (u / (1 - hp.lr * hp.weight_decay) * (1 + delta)).astype(np.float32)
 
     stream = torch.cuda.current_stream()
-    for variant in (0, 1):
+    for variant in (2, 1):                 # the bulk-copy pipeline, the register kernel
         opt = BucketedAdamW([n], bucket, dtype, undo, step_variant=variant)
         opt.load_state(torch.from_numpy(p0).cuda(), torch.from_numpy(m0).cuda(),
                        torch.from_numpy(v0).cuda())
