@@ -359,11 +359,7 @@ def run_pack(args, torch):
 
     w = W.by_name("llama_1b" if args.workload == DEFAULT_WORKLOAD else args.workload)
     stream = torch.cuda.current_stream()
-    try:
-        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
-            peak, peak_kind = float(json.load(fh)["hbm_gbs"]), "of measured"
-    except Exception:
-        peak, peak_kind = 6650.0, "of fallback"
+    peak, peak_kind = _measured_peak()
     rows = []
     for off_grid in (False, True):
         opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, 0)
@@ -413,6 +409,47 @@ def run_pack(args, torch):
     print(json.dumps({"pack": rows, "workload": w.name, "tensors": len(w.numel), "params": w.total,
                       "peak_gbs": peak, "peak_kind": peak_kind,
                       "timing": "CUDA events around each call (pointer upload and launch included)"}))
+
+
+def run_scan(args, torch):
+    """`--scan`: time the stand-alone gradient check (`so_grad_check(SO_ALL)`:
+    one batched scan launch, the two-level reduction, the statistics sent to the
+    host) over the workload's gradients, CUDA events around the call (one JSON
+    line; algorithmic bytes = the gradient's element size x N)."""
+    from paper_2509_21271_b200 import binding as B
+    from paper_2509_21271_b200 import workloads as W
+    from paper_2509_21271_b200.optimizer import BucketedAdamW
+
+    w = W.by_name("llama_1b" if args.workload == DEFAULT_WORKLOAD else args.workload)
+    hp = _hparams(w)
+    stream = torch.cuda.current_stream()
+    peak, peak_kind = _measured_peak()
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, 0)
+    if w.grad_dtype == "fp16":
+        B.so_loss_scale_config(opt.ctx, w.loss_scale, w.ls_growth, w.ls_backoff, w.ls_interval)
+    opt.load_grads_stream(W.iter_gradients(w, 1, device="cuda", loss_scale=w.loss_scale))
+    torch.cuda.synchronize()
+    times, stats = [], None
+    for it in range(max(3, args.warmup) + max(5, args.steps)):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        stats = B.so_grad_check(opt.ctx, hp, B.SO_ALL, stream)
+        e1.record(stream)
+        B.so_abandon_iteration(opt.ctx, stream)        # close the iteration without stepping
+        torch.cuda.synchronize()
+        if it >= max(3, args.warmup):
+            times.append(e0.elapsed_time(e1))
+    times.sort()
+    med, best = times[len(times) // 2], times[0]
+    n_bytes = w.total * opt.grad.element_size()
+    print(json.dumps({"scan": {"ms_median": med, "ms_best": best, "gbs_median": n_bytes / med / 1e6,
+                               "gbs_best": n_bytes / best / 1e6, "frac": n_bytes / med / 1e6 / peak,
+                               "peak_gbs": peak, "peak_kind": peak_kind},
+                      "workload": w.name, "params": w.total, "grad_dtype": w.grad_dtype,
+                      "loss_scale": w.loss_scale, "norm": stats.norm,
+                      "timing": "CUDA events around so_grad_check(SO_ALL): scan launch, reduction, "
+                                "statistics to the host"}))
+    opt.close()
 
 
 def _hparams(w, oracle_mod=None):
@@ -633,6 +670,8 @@ def main():
     ap.add_argument("--placement", action="store_true",
                     help="measure this box's rates (fused step, pinned copies, all-cores oracle) and "
                          "print what the paper's placement models (Eq. 1-5) make of them")
+    ap.add_argument("--scan", action="store_true",
+                    help="time the stand-alone gradient check over the workload's gradients")
     ap.add_argument("--pack", action="store_true",
                     help="time the one-launch pack / unpack between per-tensor buffers and the arenas")
     ap.add_argument("--sharded", action="store_true",
@@ -676,9 +715,9 @@ def main():
     if dist is not None:
         dist.barrier()
 
-    if args.placement or args.pack:
+    if args.placement or args.pack or args.scan:
         if rank == 0:
-            (run_placement if args.placement else run_pack)(args, torch)
+            (run_placement if args.placement else run_pack if args.pack else run_scan)(args, torch)
         if dist is not None:
             dist.destroy_process_group()
         return

@@ -25,6 +25,7 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <type_traits>
 
 #include "so_types.h"
 
@@ -595,14 +596,25 @@ grad_check_kernel(const __grid_constant__ CheckArgs a)
     // times a power of two (the usual loss scales); with any other scale the
     // unscaled value has a full double mantissa and keeps the two separately
     // rounded operations.
+    // With a power-of-two scale the factor is also taken out of the loop: the
+    // stored values are squared and summed as they are and the tile's sum is
+    // multiplied by the scale's square once -- scaling every term of a sum by a
+    // power of two scales every rounding with it, so the bits are those of the
+    // sum of the unscaled squares.
     const bool exact_square = !kUnscale || (__double2loint(unscale) == 0 &&
                                             (__double2hiint(unscale) & 0x000FFFFF) == 0);
-    auto square_add = [&](float x, double &acc) {
-        const double gd = kUnscale ? __dmul_rn((double)x, unscale) : (double)x;
-        if (exact_square) acc = __fma_rn(gd, gd, acc);
-        else acc = __dadd_rn(acc, __dmul_rn(gd, gd));
-    };
-    auto consume = [&](const CheckTile &t, const Raw (&raw)[kRowsPerTile]) {
+    const double sum_scale = (kUnscale && exact_square) ? __dmul_rn(unscale, unscale) : 1.0;
+    // (the choice is made once per tile, outside the unrolled element loop)
+    auto consume_as = [&](auto exact, const CheckTile &t, const Raw (&raw)[kRowsPerTile]) {
+        constexpr bool kExact = decltype(exact)::value;
+        auto square_add = [&](double stored, double &acc) {
+            if constexpr (kExact) {
+                acc = __fma_rn(stored, stored, acc);
+            } else {
+                const double gd = __dmul_rn(stored, unscale);
+                acc = __dadd_rn(acc, __dmul_rn(gd, gd));
+            }
+        };
         double acc[4] = {0.0, 0.0, 0.0, 0.0};
         if (t.base + kTileElems <= t.n) {
             // the usual case, straight-line: no bounds to check
@@ -611,7 +623,7 @@ grad_check_kernel(const __grid_constant__ CheckArgs a)
                 float x[4];
                 unpack_quad<GradT>(raw[r], x);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) square_add(x[q], acc[q]);
+                for (int q = 0; q < 4; ++q) square_add((double)x[q], acc[q]);
             }
         } else {
             const GradT *g = grad + (int64_t)t.bucket * a.geo.stride;
@@ -622,11 +634,21 @@ grad_check_kernel(const __grid_constant__ CheckArgs a)
                 if (idx + 4 <= t.n) unpack_quad<GradT>(raw[r], x);
                 else load_quad(g, idx, t.n, x);                 // guarded: zeros past the end
 #pragma unroll
-                for (int q = 0; q < 4; ++q) square_add(x[q], acc[q]);
+                for (int q = 0; q < 4; ++q) square_add((double)x[q], acc[q]);
             }
         }
         const double tile_sum = tile_fold(acc);
-        if (lane == 0) a.partials[(int64_t)t.bucket * tps + t.base / kTileElems] = tile_sum;
+        if (lane == 0)
+            a.partials[(int64_t)t.bucket * tps + t.base / kTileElems] =
+                kUnscale ? __dmul_rn(tile_sum, sum_scale) : tile_sum;
+    };
+    auto consume = [&](const CheckTile &t, const Raw (&raw)[kRowsPerTile]) {
+        if constexpr (!kUnscale) {
+            consume_as(std::true_type{}, t, raw);
+        } else {
+            if (exact_square) consume_as(std::true_type{}, t, raw);
+            else consume_as(std::false_type{}, t, raw);
+        }
     };
 
     // Two register buffers used alternately: while one tile is summed the loads
