@@ -1,5 +1,5 @@
-// Fused AdamW step with bulk-copy (TMA) staging through shared memory and
-// dynamic tile scheduling.
+// Fused AdamW step with bulk-copy (TMA) staging of its inputs through shared
+// memory and dynamic tile scheduling.
 //
 // Same arithmetic, same tile/row/quad ownership and same summation order as
 // adamw_step_kernel; only the data movement and the work distribution differ.
@@ -10,12 +10,17 @@
 // (2 or 4 rows of a tile), consumed one row at a time:
 //
 //   global --cp.async.bulk--> shared (kStagesIn chunks ahead, completion on an
-//   mbarrier) --> registers --> fp64 AdamW --> shared --cp.async.bulk--> global
+//   mbarrier) --> registers --> fp64 AdamW --> 128-bit streaming stores --> global
 //
 // One lane issues the copies; the bytes in flight no longer depend on where
-// the warp is in its arithmetic, and stores leave through the async proxy as
-// well.  Pipelines are private to a warp, so there is no block-wide
-// synchronisation and the deterministic per-tile reduction is unchanged.
+// the warp is in its arithmetic.  The results leave straight from registers:
+// staging them through shared memory for bulk stores as well cost the issuing
+// lane four more copies, a commit and a wait per chunk (a tenth of all warp
+// instructions, executed with one lane active) and 70 KB of shared memory per
+// block, and was slower wherever a power cap holds the clock down (-1.1 % per
+// iteration on 8 B parameters, -1.3 % on 1.2 B, equal on 124 M).  Pipelines
+// are private to a warp, so there is no block-wide synchronisation and the
+// deterministic per-tile reduction is unchanged.
 // Bulk copies need 16-byte aligned addresses and sizes: slots are 256-byte
 // aligned and chunk starts are multiples of 128 elements, so only a chunk
 // whose valid length is not a multiple of 8 elements (the ragged end of a
@@ -41,14 +46,12 @@
 namespace so {
 
 // Shape of the per-warp pipeline: rows (of 128 elements) per chunk, warps per
-// block (one block per SM), chunks in flight ahead of the arithmetic, and
-// output staging buffers.
-template <int kRows_, int kWarps_, int kStagesIn_, int kStagesOut_>
+// block (one block per SM), chunks in flight ahead of the arithmetic.
+template <int kRows_, int kWarps_, int kStagesIn_>
 struct PipeShape {
     static constexpr int kRows = kRows_;
     static constexpr int kWarps = kWarps_;
     static constexpr int kStagesIn = kStagesIn_;
-    static constexpr int kStagesOut = kStagesOut_;
     static constexpr int kChunkElems = kRows_ * kRowElems;
     static constexpr int kChunksPerTile = kTileElems / kChunkElems;
     static constexpr int kThreads = kWarps_ * 32;
@@ -71,8 +74,7 @@ struct TmaLayout {
     static constexpr int kGradBytes = S::kChunkElems * (int)sizeof(GradT);
     static constexpr int kF32Bytes = S::kChunkElems * 4;
     static constexpr int kInStage = 3 * kF32Bytes + kGradBytes;            // p, m, v, g
-    static constexpr int kOutStage = 3 * kF32Bytes + S::kChunkElems * 2;   // p, m, v, bf16
-    static constexpr int kWarpBytes = S::kStagesIn * kInStage + S::kStagesOut * kOutStage;
+    static constexpr int kWarpBytes = S::kStagesIn * kInStage;
     // per warp and input stage: one mbarrier (8 B) and one descriptor (32 B);
     // then the launch's buckets with their slots resolved, and their count
     static constexpr int kEntriesOffset = S::kWarps * S::kStagesIn * 40;
@@ -137,25 +139,6 @@ __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, ui
         : "memory");
 }
 
-__device__ __forceinline__ void bulk_store(void *dst, uint32_t src_smem, uint32_t bytes,
-                                           uint64_t policy)
-{
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::
-                     "l"(dst),
-                 "r"(src_smem), "r"(bytes), "l"(policy)
-                 : "memory");
-}
-
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-
-template <int kPending>
-__device__ __forceinline__ void bulk_wait_read()
-{
-    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kPending) : "memory");
-}
-
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---- the kernel ---------------------------------------------------------------
@@ -165,7 +148,7 @@ __global__ void __launch_bounds__(S::kThreads, 1)
 adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, int pair)
 {
     using L = TmaLayout<GradT, S>;
-    constexpr int kStagesIn = S::kStagesIn, kStagesOut = S::kStagesOut;
+    constexpr int kStagesIn = S::kStagesIn;
     constexpr int kChunkRows = S::kRows, kTmaWarps = S::kWarps;
     extern __shared__ __align__(128) unsigned char smem[];
 
@@ -180,7 +163,6 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
     ResolvedEntry *entries = reinterpret_cast<ResolvedEntry *>(smem + L::kEntriesOffset);
     int32_t *n_active_smem = reinterpret_cast<int32_t *>(entries + kMaxBatch);
     unsigned char *wbase = smem + L::kHeaderBytes + wib * L::kWarpBytes;
-    unsigned char *out_base = wbase + kStagesIn * L::kInStage;
     uint32_t *next_tile = &ctrl->counters[pair][0];
     uint32_t *done_warps = &ctrl->counters[pair][1];
 
@@ -307,7 +289,7 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
     __syncwarp();
 
     uint32_t phases = 0;               // parity bit per input stage
-    int stage = 0, ostage = 0;
+    int stage = 0;
     double acc[4] = {0.0, 0.0, 0.0, 0.0};
     bool failed = false;
 
@@ -329,12 +311,10 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                 break;
             }
             phases ^= 1u << stage;
-            // the output stage is free once the bulk stores issued from it
-            // kStagesOut chunks ago have finished reading shared memory
-            if (lane == 0) bulk_wait_read<kStagesOut - 1>();
-            __syncwarp();
             const unsigned char *in = wbase + stage * L::kInStage;
-            unsigned char *out = out_base + ostage * L::kOutStage;
+            float *p_out = a.master + dst + start, *m_out = a.mom + dst + start,
+                  *v_out = a.var + dst + start;
+            uint16_t *lp_out = pb + start;
             // Two rows (8 elements per lane) in flight at a time: the eight
             // dependent chains of conversions, seeds and fp64 operations
             // interleave, which is what hides their latency with only ten warps
@@ -366,15 +346,16 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                     make_float4(m0[0], m0[1], m0[2], m0[3]), make_float4(v0[0], v0[1], v0[2], v0[3]), k,
                     scale);
             };
+            // (a chunk that takes this path starts on a 16-byte boundary in
+            // every arena and its valid length is a multiple of 8 elements, so
+            // every quad below it is whole and aligned)
             auto store_row = [&](uint32_t off, const float (&pq)[4], const float (&mq)[4],
                                  const float (&vq)[4]) {
-                *reinterpret_cast<float4 *>(out + off * 4) = make_float4(pq[0], pq[1], pq[2], pq[3]);
-                *reinterpret_cast<float4 *>(out + L::kF32Bytes + off * 4) =
-                    make_float4(mq[0], mq[1], mq[2], mq[3]);
-                *reinterpret_cast<float4 *>(out + 2 * L::kF32Bytes + off * 4) =
-                    make_float4(vq[0], vq[1], vq[2], vq[3]);
-                *reinterpret_cast<uint2 *>(out + 3 * L::kF32Bytes + off * 2) =
-                    make_uint2(pack_lp(pq[0], pq[1], fp16), pack_lp(pq[2], pq[3], fp16));
+                __stcs(reinterpret_cast<float4 *>(p_out + off), make_float4(pq[0], pq[1], pq[2], pq[3]));
+                __stcs(reinterpret_cast<float4 *>(m_out + off), make_float4(mq[0], mq[1], mq[2], mq[3]));
+                __stcs(reinterpret_cast<float4 *>(v_out + off), make_float4(vq[0], vq[1], vq[2], vq[3]));
+                __stcs(reinterpret_cast<uint2 *>(lp_out + off),
+                       make_uint2(pack_lp(pq[0], pq[1], fp16), pack_lp(pq[2], pq[3], fp16)));
             };
             constexpr int kAtOnce = 2;     // four at once spill (168 registers + 80 bytes of stack)
             static_assert(kChunkRows % kAtOnce == 0, "rows are taken in groups");
@@ -408,21 +389,9 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
                     }
                 }
             }
-            fence_async_smem();        // generic writes -> visible to the async proxy
-            // every lane is done with the input stage and has filled its part
-            // of the output stage: refill the one, drain the other
+            // every lane is done with the input stage: refill it
             __syncwarp();
-            if (lane == 0) {
-                produce(stage);
-                const uint32_t src_s = smem_u32(out);
-                const uint32_t fbytes = len * 4u;
-                bulk_store(a.master + dst + start, src_s, fbytes, policy);
-                bulk_store(a.mom + dst + start, src_s + L::kF32Bytes, fbytes, policy);
-                bulk_store(a.var + dst + start, src_s + 2 * L::kF32Bytes, fbytes, policy);
-                bulk_store(pb + start, src_s + 3 * L::kF32Bytes, len * 2u, policy);
-                bulk_commit();
-            }
-            ostage = (ostage + 1 == kStagesOut) ? 0 : ostage + 1;
+            if (lane == 0) produce(stage);
         } else {
             const GradT *g = static_cast<const GradT *>(a.grad) + (int64_t)d.bucket * stride;
             const int64_t src = (int64_t)d.src_slot * stride;
@@ -477,7 +446,6 @@ adamw_step_tma_kernel(const __grid_constant__ StepArgs a, ControlBlock *ctrl, in
         }
     }
     if (lane == 0) {
-        bulk_wait_all();
         // The last warp of the launch to get here re-arms the counters.  The
         // fence orders this warp's tile claims (including the look-ahead claim
         // whose value is never used) before its arrival, so no claim can land

@@ -297,13 +297,15 @@ cudaError_t launch_dependent(void (*kernel)(KArgs...), unsigned grid, unsigned b
 // crossover between 2 Mi and 4 Mi elements per launch).
 constexpr int64_t kSmallLaunchElems = (int64_t)3 << 20;
 
-// Shapes of the bulk-copy pipeline: rows per chunk, warps per block (one block
-// per SM), input stages, output stages.  They came out of a sweep on B200:
-// 512-element chunks halve the per-chunk bookkeeping, two input stages of 7 KB
-// per warp keep ~140 KB of loads in flight per SM, and ten warps are the most
-// that fit in shared memory (nine with fp32 gradients).
-using ShapeBf16 = PipeShape<4, 10, 2, 1>;
-using ShapeFp32 = PipeShape<4, 9, 2, 1>;
+// Shape of the bulk-copy pipeline: rows per chunk, warps per block (one block
+// per SM), input stages.  It came out of sweeps on B200: 512-element chunks
+// halve the per-chunk bookkeeping, and two input stages of 7 KB (8 KB with fp32
+// gradients) per warp keep 140-160 KB of loads in flight per SM.  Twelve warps,
+// or a third stage, fit as well since the results no longer pass through shared
+// memory; twelve warps measured 0.2 % better on 8 B parameters under the power
+// cap and 1 % worse on 124 M at full clock, a third stage 0.3-0.5 % worse on both.
+using ShapeBf16 = PipeShape<4, 10, 2>;
+using ShapeFp32 = PipeShape<4, 10, 2>;
 
 template <typename GradT, typename S>
 cudaError_t launch_tma(so_ctx *c, const StepArgs &a, int n, bool speculative, cudaStream_t stream)
@@ -385,7 +387,7 @@ so_status launch_steps(so_ctx *c, const std::vector<BucketEntry> &entries, const
             const int dt = c->grad_dtype;
             const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_step);
             // A small launch takes the register kernel: no pipeline to fill and
-            // drain, no 217 KB of shared memory per block to set up (a launch of
+            // drain, no 146 KB of shared memory per block to set up (a launch of
             // 1 Mi elements: 14 us against 17 us; from 4 Mi elements on the
             // pipeline is ahead, by 27 % at 8 Mi).
             int64_t launch_elems = 0;
