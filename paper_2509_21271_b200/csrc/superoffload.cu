@@ -388,8 +388,8 @@ so_status launch_steps(so_ctx *c, const std::vector<BucketEntry> &entries, const
             const unsigned grid = grid_for(c, (int64_t)n * geo.tiles_per_slot, c->occ_step);
             // A small launch takes the register kernel: no pipeline to fill and
             // drain, no 146 KB of shared memory per block to set up (a launch of
-            // 1 Mi elements: 14 us against 17 us; from 4 Mi elements on the
-            // pipeline is ahead, by 27 % at 8 Mi).
+            // 1 Mi elements: 14.3 us against 15.8 us; from 4 Mi elements on the
+            // pipeline is ahead, by 26 % at 8 Mi).
             int64_t launch_elems = 0;
             for (int i = 0; i < n; ++i) launch_elems += elems_of(c, a.e[i].bucket);
             const bool registers = c->step_variant == 1 ||
