@@ -7,7 +7,7 @@
 // Data movement.  The register version keeps a warp's loads in flight only
 // while that warp is not computing, which leaves both DRAM and the issue slots
 // half idle.  Here every warp runs a private software pipeline over *chunks*
-// (2 or 4 rows of a tile), consumed one row at a time:
+// (4 rows of a tile), consumed two rows at a time:
 //
 //   global --cp.async.bulk--> shared (kStagesIn chunks ahead, completion on an
 //   mbarrier) --> registers --> fp64 AdamW --> 128-bit streaming stores --> global
