@@ -14,6 +14,11 @@ fused step kernel, and the CPU oracle timed on a bounded sample.
 With N > 1 (launched by torchrun) every rank runs an independent replica of
 the workload on its own GPU -- the path has no exchange step on one node --
 and the value is N x params / max-over-ranks time.
+
+Side modes, each printing a JSON line of its own: --scan (the stand-alone
+gradient check), --pack (one-launch flattening between per-tensor buffers and
+the arenas), --placement (the paper's placement models fed with this box's
+rates), --sharded (optimizer states sharded by bucket ranges over the ranks).
 """
 from __future__ import annotations
 
