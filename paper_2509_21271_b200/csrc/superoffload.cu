@@ -1475,8 +1475,17 @@ so_status pack_or_unpack(so_ctx *c, const void *const *tensor_ptrs, bool pack, c
         if (!c->h_ptr_stage) {
             e = cudaHostAlloc(reinterpret_cast<void **>(&c->h_ptr_stage), nt * sizeof(uint64_t),
                               cudaHostAllocDefault);
-            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ptrs_uploaded, cudaEventDisableTiming);
-            if (e != cudaSuccess) return cuda_fail(c, e);
+            if (e != cudaSuccess) {
+                c->h_ptr_stage = nullptr;
+                return cuda_fail(c, e);
+            }
+            e = cudaEventCreateWithFlags(&c->ptrs_uploaded, cudaEventDisableTiming);
+            if (e != cudaSuccess) {             // all or nothing: the next call starts over
+                cudaFreeHost(c->h_ptr_stage);
+                c->h_ptr_stage = nullptr;
+                c->ptrs_uploaded = nullptr;
+                return cuda_fail(c, e);
+            }
         } else {
             // the staging buffer may still feed the previous call's upload
             // (only that copy is waited for, not the stream)
