@@ -396,7 +396,7 @@ def test_pipelined_host_fed_iterations_overwrite_no_gradient_still_in_use():
     assert torch.equal(host_p.view(torch.int16), opt.gather_param_bf16().cpu().view(torch.int16))
 
 
-@pytest.mark.parametrize("name,undo", [("tiny", B.SO_ALL), ("tiny_ragged", 2)])
+@pytest.mark.parametrize("name,undo", [("tiny", B.SO_ALL), ("tiny_ragged", 2), ("tiny_ragged", 0)])
 def test_pipelined_host_fed_iterations_are_bitwise_the_blocking_ones(name, undo):
     """so_iteration_host_pipelined does not wait at its end: the parameters that
     leave after the verdict travel while the next call's gradients arrive.
