@@ -433,6 +433,30 @@ def test_pipelined_host_fed_iterations_are_bitwise_the_blocking_ones(name, undo)
     assert torch.equal(host_p.view(torch.int16), opt.gather_param_bf16().cpu().view(torch.int16))
 
 
+def test_pipelined_host_fed_iterations_without_a_parameter_buffer():
+    """No outgoing copies at all (host_param_bf16 = NULL): the calls still
+    overlap their incoming copies with the previous iteration's follow-up, and
+    the final wait still waits for the stream."""
+    w = W.by_name("tiny_ragged")
+    hp = hparams_of(w)
+    stream = torch.cuda.current_stream()
+    ref = _run_device_only(w, 8, undo_slots=2, speculative=True)
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, 2)
+    opt.load_state(W.initial_master(w, device="cuda"))
+    opt.cast_params(stream=stream)
+    host_g = [torch.empty(w.total, dtype=opt.grad_torch_dtype, pin_memory=True) for _ in range(2)]
+    trace = []
+    for step in range(1, 9):
+        buf = host_g[step % 2]
+        buf.copy_(W.gradients(w, step, device="cuda"))
+        res = B.so_iteration_host_pipelined(opt.ctx, hp, buf.data_ptr(), 0, stream)
+        trace.append((res.decision, res.stats.sumsq, res.stats.norm, res.stats.clip_coef,
+                      res.stats.nonfinite, res.step_after))
+    B.so_iteration_host_wait(opt.ctx, stream)
+    assert trace == ref[0]
+    assert _state_bytes(opt) == ref[1]
+
+
 # ---------------------------------------------------------------------------
 # fp16 gradients under dynamic loss scaling (the paper's own precision path)
 # ---------------------------------------------------------------------------
