@@ -819,6 +819,47 @@ def test_a_kernel_that_gives_up_its_wait_ends_the_iteration_cleanly():
     assert opt.counters().timeouts == 1 and opt.guard_bands_intact()
 
 
+def test_a_give_up_inside_pipelined_host_fed_iterations_leaves_nothing_in_flight():
+    """The same bounded wait running out in the middle of overlapped host-fed
+    iterations: the failing call reports SO_ERR_TIMEOUT after waiting for every
+    copy it or its predecessor started, the committed state is the one before
+    it, and the iteration, given again, continues the sequence bit for bit."""
+    w = W.by_name("tiny_ragged")
+    hp = hparams_of(w)
+    stream = torch.cuda.current_stream()
+    ref = _run_device_only(w, 4, undo_slots=2, speculative=True)
+    opt = BucketedAdamW(w.numel, w.bucket_elems, w.grad_dtype, 2, guard_bands=True)
+    opt.load_state(W.initial_master(w, device="cuda"))
+    opt.cast_params(stream=stream)
+    host_g = [torch.empty(w.total, dtype=opt.grad_torch_dtype, pin_memory=True) for _ in range(2)]
+    host_p = torch.empty(w.total, dtype=torch.bfloat16, pin_memory=True)
+    trace = []
+
+    def call(step):
+        buf = host_g[step % 2]
+        buf.copy_(W.gradients(w, step, device="cuda"))
+        res = B.so_iteration_host_pipelined(opt.ctx, hp, buf.data_ptr(), host_p.data_ptr(), stream)
+        trace.append((res.decision, res.stats.sumsq, res.stats.norm, res.stats.clip_coef,
+                      res.stats.nonfinite, res.step_after))
+
+    call(1)
+    call(2)
+    B.so_debug_set_spin_limit(opt.ctx, 0)
+    with pytest.raises(B.SuperOffloadError) as err:
+        call(3)
+    assert err.value.status == B.SO_ERR_TIMEOUT
+    B.so_debug_set_spin_limit(opt.ctx, 1 << 20)
+    assert opt.step_count == 2 and opt.counters().timeouts == 1
+    B.so_iteration_host_wait(opt.ctx, stream)                 # nothing left to wait for
+    call(3)
+    call(4)
+    B.so_iteration_host_wait(opt.ctx, stream)
+    assert trace == ref[0]
+    assert _state_bytes(opt) == ref[1]
+    assert torch.equal(host_p.view(torch.int16), opt.gather_param_bf16().cpu().view(torch.int16))
+    assert opt.guard_bands_intact()
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "fp32"])
 def test_second_moments_that_overflow_fp32_follow_the_oracle(dtype):
     """Finite gradients around 1e21 with clipping off: (1 - beta2) g^2 exceeds
